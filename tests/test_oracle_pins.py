@@ -1,0 +1,418 @@
+"""Pins for the CPU oracle: closed forms on hand-built frames, brute force on tiny
+inputs, invariants, and library routines used as a third opinion.  None of these
+tests re-types the oracle's formulas; expected values come from construction."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import emc2_gen as gen
+
+F32 = np.float32
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def nxt(x, toward):
+    return np.nextafter(F32(x), F32(toward))
+
+
+# ------------------------------------------------------------------ O1 voxel coordinates
+# Grid whose numbers are exact in binary: min (-2, -4, 0), voxel (0.25, 0.5, 2), dims (16, 16, 4).
+BMIN, BVOX, BDIMS = (-2.0, -4.0, 0.0), (0.25, 0.5, 2.0), (16, 16, 4)
+
+
+def _pts(rows, C=4):
+    a = np.zeros((1, len(rows), C), F32)
+    for i, r in enumerate(rows):
+        a[0, i, :len(r)] = r
+    return a
+
+
+def test_coords_of_points_built_from_known_cells(oracle):
+    rng = np.random.default_rng(1)
+    cells = rng.integers(0, [16, 16, 4], size=(300, 3))
+    frac = rng.integers(0, 8, size=(300, 3)) / 8.0           # exactly representable offsets
+    p = np.array(BMIN) + (cells + frac) * np.array(BVOX)
+    pts = np.zeros((1, 300, 4), F32)
+    pts[0, :, :3] = p
+    r = oracle.voxelize(pts, BMIN, BVOX, BDIMS)
+    got = r["coords"][r["point_voxel"][0]]
+    assert (got[:, 0] == 0).all()
+    assert (got[:, 1:] == cells[:, ::-1]).all()               # columns are (b, z, y, x)
+
+
+@pytest.mark.parametrize("grid", [gen.KITTI_GRIDS[0], gen.KITTI_GRIDS[1], gen.NUSCENES_GRIDS[0],
+                                  gen.NUSCENES_GRIDS[1]])
+def test_voxel_centres_map_to_their_cell(oracle, grid):
+    rng = np.random.default_rng(2)
+    cells = rng.integers(0, grid.dims, size=(500, 3))
+    p = np.array(grid.min, np.float64) + (cells + 0.5) * np.array([F32(v) for v in grid.voxel], np.float64)
+    pts = np.zeros((1, 500, 4), F32)
+    pts[0, :, :3] = p
+    r = oracle.voxelize(pts, grid.min, grid.voxel, grid.dims)
+    pv = r["point_voxel"][0]
+    assert (pv >= 0).all()
+    assert (r["coords"][pv][:, 1:] == cells[:, ::-1]).all()
+
+
+def test_range_is_half_open_and_nonfinite_is_out(oracle):
+    rows = [(-2.0, -4.0, 0.0),                     # exactly min -> cell 0
+            (nxt(-2.0, -9), -4.0, 0.0),            # one ulp below min -> out
+            (2.0, 0.0, 0.0),                       # x == max -> out
+            (nxt(nxt(2.0, 0), 0), 0.0, 0.0),       # 2 ulps inside: p - min = 4 - 2^-22 exactly -> last cell
+            (0.0, 4.0, 0.0), (0.0, 0.0, 8.0),      # y == max, z == max -> out
+            (np.nan, 0.0, 0.0), (0.0, np.inf, 0.0), (0.0, 0.0, -np.inf),
+            (-0.0, 0.0, nxt(8.0, 0))]
+    r = oracle.voxelize(_pts(rows), BMIN, BVOX, BDIMS)
+    pv = r["point_voxel"][0]
+    assert list(pv >= 0) == [True, False, False, True, False, False, False, False, False, True]
+    c = r["coords"]
+    assert tuple(c[pv[0]]) == (0, 0, 0, 0)
+    assert tuple(c[pv[3]]) == (0, 0, 8, 15)
+    assert tuple(c[pv[9]]) == (0, 3, 8, 8)
+
+
+def test_scales_are_independent(oracle):
+    # z = 1.5 lies inside the pillar grid (z range [-3, 1) fails) -- use a point outside the
+    # fine grid's z range only by giving the fine grid a smaller z extent.
+    rows = [(0.1, 0.1, 3.0)]
+    fine = oracle.voxelize(_pts(rows), (0, 0, 0), (0.5, 0.5, 0.5), (4, 4, 4))
+    pillar = oracle.voxelize(_pts(rows), (0, 0, 0), (0.5, 0.5, 4.0), (4, 4, 1))
+    assert fine["num_voxels"] == 0 and fine["point_voxel"][0, 0] == -1
+    assert pillar["num_voxels"] == 1 and pillar["point_voxel"][0, 0] == 0
+
+
+# ------------------------------------------------------------------ O2 dedup
+def test_dedup_against_brute_force_on_tiny_inputs(oracle):
+    rng = np.random.default_rng(3)
+    for n in (1, 7, 64, 512):
+        B = 2
+        cells = rng.integers(0, [5, 4, 3], size=(B, n, 3))     # few cells -> many collisions
+        frac = rng.integers(1, 8, size=(B, n, 3)) / 8.0
+        pts = np.zeros((B, n, 4), F32)
+        pts[..., :3] = np.array(BMIN) + (cells + frac) * np.array(BVOX)
+        outside = rng.random((B, n)) < 0.2
+        pts[outside, 0] = 100.0
+        r = oracle.voxelize(pts, BMIN, BVOX, BDIMS)
+        # brute force: O(n^2) distinct list of (b, z, y, x) tuples, then sorted
+        seen = []
+        for b in range(B):
+            for i in range(n):
+                if outside[b, i]:
+                    continue
+                t = (b, int(cells[b, i, 2]), int(cells[b, i, 1]), int(cells[b, i, 0]))
+                if not any(t == s for s in seen):
+                    seen.append(t)
+        seen.sort()
+        assert r["num_voxels"] == len(seen)
+        assert [tuple(x) for x in r["coords"]] == seen
+        for b in range(B):
+            for i in range(n):
+                m = r["point_voxel"][b, i]
+                if outside[b, i]:
+                    assert m == -1
+                else:
+                    assert seen[m] == (b, int(cells[b, i, 2]), int(cells[b, i, 1]), int(cells[b, i, 0]))
+        # counts: number of points per tuple
+        for m, t in enumerate(seen):
+            k = sum(1 for b in range(B) for i in range(n) if not outside[b, i] and
+                    (b, int(cells[b, i, 2]), int(cells[b, i, 1]), int(cells[b, i, 0])) == t)
+            assert r["counts"][m] == k
+
+
+def test_dedup_invariants_and_torch_unique_on_generated_frame(oracle):
+    w = gen.TINY
+    pts = gen.make_points(w, 0)[None]
+    for g in w.grids:
+        r = oracle.voxelize(pts, g.min, g.voxel, g.dims, 0)
+        c = r["coords"].astype(np.int64)
+        key = ((c[:, 0] * g.dims[2] + c[:, 1]) * g.dims[1] + c[:, 2]) * g.dims[0] + c[:, 3]
+        assert (np.diff(key) > 0).all()                        # strictly ascending, hence unique
+        pv = r["point_voxel"][0]
+        assert r["counts"].sum() == (pv >= 0).sum()
+        # library third opinion: unique / inverse / counts of the per-point keys
+        pk = torch.from_numpy(key[pv[pv >= 0]])
+        u, inv, cnt = torch.unique(pk, sorted=True, return_inverse=True, return_counts=True)
+        assert np.array_equal(u.numpy(), key)
+        assert np.array_equal(inv.numpy(), pv[pv >= 0])
+        assert np.array_equal(cnt.numpy(), r["counts"])
+
+
+# ------------------------------------------------------------------ O3 counts and means
+def test_copies_of_one_point(oracle):
+    p = (0.3, -1.2, 0.7, 0.25)
+    for k, cap, want in ((5, 0, 5), (5, 8, 5), (40, 32, 32), (33, 32, 32)):
+        r = oracle.voxelize(_pts([p] * k), BMIN, BVOX, BDIMS, cap)
+        assert r["num_voxels"] == 1 and r["counts"][0] == want
+        assert np.array_equal(r["mean"][0], np.array(p, F32))
+        assert (r["point_voxel"][0] == 0).sum() == want
+        assert (r["point_voxel"][0][:want] == 0).all() and (r["point_voxel"][0][want:] == -1).all()
+
+
+def test_cap_keeps_lowest_indices(oracle):
+    # 40 points in one pillar; intensity (no range test) = index.
+    rows = [(0.1, 0.1, 0.5, float(i)) for i in range(40)]
+    r = oracle.voxelize(_pts(rows), BMIN, BVOX, BDIMS, 32)
+    assert r["counts"][0] == 32 and r["mean"][0, 3] == F32(15.5)      # mean of 0..31
+    r = oracle.voxelize(_pts(rows[::-1]), BMIN, BVOX, BDIMS, 32)
+    assert r["counts"][0] == 32 and r["mean"][0, 3] == F32(23.5)      # mean of 39..8
+    r = oracle.voxelize(_pts(rows), BMIN, BVOX, BDIMS, 0)
+    assert r["counts"][0] == 40 and r["mean"][0, 3] == F32(19.5)
+
+
+def test_means_against_index_add(oracle):
+    w = gen.NUSCENES.with_shape(1, 20000)
+    pts = gen.make_points(w, 0)[None]
+    g = w.grids[1]
+    r = oracle.voxelize(pts, g.min, g.voxel, g.dims, 0)
+    pv = torch.from_numpy(r["point_voxel"][0].astype(np.int64))
+    ok = pv >= 0
+    sums = torch.zeros(r["num_voxels"], w.C, dtype=torch.float64)
+    sums.index_add_(0, pv[ok], torch.from_numpy(pts[0]).double()[ok])
+    want = (sums / torch.from_numpy(r["counts"]).double()[:, None]).float().numpy()
+    assert np.abs(r["mean"] - want).max() <= 1e-6
+    # with the cap: sum over kept points only
+    r = oracle.voxelize(pts, g.min, g.voxel, g.dims, 4)
+    assert r["counts"].max() == 4
+    pv = r["point_voxel"][0]
+    tot = (r["mean"].astype(np.float64) * r["counts"][:, None]).sum(0)
+    assert np.allclose(tot, pts[0][pv >= 0].astype(np.float64).sum(0), rtol=1e-5)
+    # a kept point is among the first `cap` of its voxel: earlier same-voxel points are all kept
+    full = oracle.voxelize(pts, g.min, g.voxel, g.dims, 0)["point_voxel"][0]
+    seen = {}
+    for i, m in enumerate(full):
+        if m < 0:
+            continue
+        seen[m] = seen.get(m, 0) + 1
+        assert (pv[i] >= 0) == (seen[m] <= 4)
+
+
+# ------------------------------------------------------------------ O4 BEV
+def test_bev_cells(oracle):
+    w = gen.TINY
+    pts = gen.make_points(w, 0)[None].repeat(2, axis=0).copy()
+    pts[1, :, 0] += 0.2
+    g = w.grids[1]
+    r = oracle.voxelize(pts, g.min, g.voxel, g.dims, g.max_points)
+    img = oracle.bev(2, w.C, g.dims[1], g.dims[0], r["coords"], r["mean"])
+    assert img.shape == (2, 4, 500, 440)
+    c = r["coords"]
+    assert np.array_equal(img[c[:, 0], :, c[:, 2], c[:, 3]], r["mean"])      # bitwise
+    occ = np.zeros((2, 500, 440), bool)
+    occ[c[:, 0], c[:, 2], c[:, 3]] = True
+    assert not img[:, :, ~occ[0] & ~occ[1]].any()
+    assert (img[:, 0][occ] != 0).all()                                         # x means are non-zero
+    assert np.isclose(img.astype(np.float64).sum(), r["mean"].astype(np.float64).sum())
+
+
+# ------------------------------------------------------------------ O5 projection
+def _proj1(fx, fy, cx, cy, yaw=0.0, W=1280, H=512):
+    w = gen.TINY
+    from dataclasses import replace
+    w = replace(w, cameras=(gen.Camera(fx, fy, cx, cy, yaw),), img_w=W, img_h=H)
+    return gen.make_projection(w)[None], w
+
+
+def test_projection_closed_forms(oracle):
+    P, w = _proj1(512.0, 256.0, 640.0, 128.0)
+    d = 8.0
+    rows = [(d, 0, 0),                              # optical axis -> principal point
+            (d, -d * 64 / 512, -d * 32 / 256),      # -> (cx + 64, cy + 32)
+            (-d, 0, 0),                             # behind the camera
+            (2.0, 2.5, 0),                          # u == 0 exactly -> visible
+            (2.0, -2.5, 0),                         # u == W exactly -> not visible
+            (2.0, nxt(nxt(-2.5, 0), 0), 0),         # 2 ulps inside the right edge (1 ulp rounds onto it)
+            (4.0, 0, 2.0),                          # v == 0 exactly -> visible
+            (4.0, 0, nxt(2.0, 9)),                  # just above the top edge
+            (4.0, 0, -6.0),                         # v == H exactly -> not visible
+            (0.1, 0, 0),                            # depth == min_depth -> not visible
+            (nxt(0.1, 1), 0, 0)]
+    uvd, mask, cam = oracle.project(_pts(rows), P, 512, 1280, 0.1)
+    assert tuple(uvd[0, 0]) == (640.0, 128.0, 8.0)
+    assert tuple(uvd[0, 1]) == (704.0, 160.0, 8.0)
+    assert list(mask[0]) == [1, 1, 0, 1, 0, 1, 1, 0, 0, 0, 1]
+    assert list(cam[0]) == [0, 0, -1, 0, -1, 0, 0, -1, -1, -1, 0]
+    assert tuple(uvd[0, 3][:2]) == (0.0, 128.0) and tuple(uvd[0, 6][:2]) == (640.0, 0.0)
+    assert tuple(uvd[0, 2]) == (-1.0, -1.0, -8.0)       # invisible: (-1, -1, depth in camera 0)
+    assert tuple(uvd[0, 4]) == (-1.0, -1.0, 2.0)
+
+
+def test_projection_nonfinite_and_translation_column(oracle):
+    P, _ = _proj1(512.0, 256.0, 640.0, 128.0)
+    P[0, 0, :, 3] = (64.0, 32.0, 1.0)                   # t = (.., .., d + 1)
+    uvd, mask, cam = oracle.project(_pts([(7.0, 0, 0), (np.nan, 0, 0), (np.inf, 0, 0)]), P, 512, 1280, 0.1)
+    assert tuple(uvd[0, 0]) == ((640.0 * 7 + 64) / 8, (128.0 * 7 + 32) / 8, 8.0)
+    assert list(mask[0]) == [1, 0, 0] and list(cam[0]) == [0, -1, -1]
+    assert tuple(uvd[0, 1]) == (-1.0, -1.0, 0.0) and tuple(uvd[0, 2]) == (-1.0, -1.0, 0.0)
+
+
+def test_yawed_cameras_see_the_rotated_point_identically(oracle):
+    w = gen.NUSCENES
+    P = gen.make_projection(w)[None]
+    rng = np.random.default_rng(5)
+    base = np.stack([rng.uniform(10, 40, 200), rng.uniform(-3, 3, 200), rng.uniform(-2, 2, 200)], 1)
+    u0 = None
+    for k, camk in enumerate(w.cameras):
+        a = np.radians(camk.yaw_deg)
+        R = np.array([[np.cos(a), -np.sin(a), 0], [np.sin(a), np.cos(a), 0], [0, 0, 1]])
+        pts = np.zeros((1, 200, 5), F32)
+        pts[0, :, :3] = base @ R.T
+        uvd, mask, cam = oracle.project(pts, P, w.img_h, w.img_w, w.min_depth)
+        assert ((mask[0] >> k) & 1).all()
+        # lowest visible camera wins; for k > 0 a lower camera may also see the point
+        sel = cam[0] == k
+        assert sel.sum() > 50
+        if u0 is None:
+            u0 = uvd[0].copy()
+        assert np.allclose(uvd[0][sel], u0[sel], rtol=1e-5, atol=2e-3)
+
+
+def test_overlapping_cameras_lowest_index_wins(oracle):
+    w = gen.NUSCENES
+    P = gen.make_projection(w)[None]
+    a = np.radians(27.5)                                 # halfway between yaw 0 and yaw +55
+    pts = _pts([(20 * np.cos(a), 20 * np.sin(a), 0.0)], C=5)
+    uvd, mask, cam = oracle.project(pts, P, w.img_h, w.img_w, w.min_depth)
+    assert mask[0, 0] == 0b011 and cam[0, 0] == 0
+    assert uvd[0, 0, 0] < 800.0                          # left of camera 0's principal point
+    a = np.radians(145.0)                                # the gap between yaw 110 and yaw 180
+    _, mask, cam = oracle.project(_pts([(20 * np.cos(a), 20 * np.sin(a), 0.0)], C=5), P, w.img_h,
+                                  w.img_w, w.min_depth)
+    assert mask[0, 0] == 0 and cam[0, 0] == -1
+
+
+# ------------------------------------------------------------------ O6 bilinear gather
+def test_gather_at_texel_centres_and_zero_rows(oracle):
+    rng = np.random.default_rng(6)
+    feat = rng.standard_normal((1, 2, 6, 9, 5)).astype(F32)
+    uvd = np.array([[[4 * 3, 4 * 2, 1.0], [0, 0, 1.0], [4 * 8, 4 * 5, 1.0], [5.0, 5.0, 1.0]]], F32)
+    cam = np.array([[1, 0, 1, -1]], np.int8)
+    out = oracle.gather(uvd, cam, feat, 4)
+    assert np.array_equal(out[0, 0], feat[0, 1, 2, 3])
+    assert np.array_equal(out[0, 1], feat[0, 0, 0, 0])
+    assert np.array_equal(out[0, 2], feat[0, 1, 5, 8])   # last texel: neighbours clamp onto it
+    assert not out[0, 3].any()
+
+
+def test_gather_reproduces_affine_maps_and_clamps(oracle):
+    Hf, Wf, Cf, s = 12, 20, 3, 8
+    yy, xx = np.meshgrid(np.arange(Hf), np.arange(Wf), indexing="ij")
+    a, b, c = (0.5, -1.25, 2.0), (0.75, 0.5, -3.0), (1.0, -2.0, 0.25)
+    feat = np.stack([a[i] * xx + b[i] * yy + c[i] for i in range(3)], -1).astype(F32)[None, None]
+    rng = np.random.default_rng(7)
+    u = rng.uniform(0, (Wf - 1) * s, 300)
+    v = rng.uniform(0, (Hf - 1) * s, 300)
+    uvd = np.stack([u, v, np.ones(300)], 1).astype(F32)[None]
+    out = oracle.gather(uvd, np.zeros((1, 300), np.int8), feat, s)
+    fx, fy = uvd[0, :, 0].astype(np.float64) / s, uvd[0, :, 1].astype(np.float64) / s
+    want = np.stack([a[i] * fx + b[i] * fy + c[i] for i in range(3)], -1)
+    assert np.abs(out[0] - want).max() < 1e-5
+    # beyond the last texel centre the map is held constant along that axis (edge clamp)
+    uvd = np.array([[[(Wf - 1) * s + 5.0, 16.0, 1.0], [24.0, (Hf - 1) * s + 3.0, 1.0]]], F32)
+    out = oracle.gather(uvd, np.zeros((1, 2), np.int8), feat, s)
+    assert np.allclose(out[0, 0], [a[i] * (Wf - 1) + b[i] * 2 + c[i] for i in range(3)])
+    assert np.allclose(out[0, 1], [a[i] * 3 + b[i] * (Hf - 1) + c[i] for i in range(3)])
+
+
+def test_gather_against_grid_sample(oracle):
+    w = gen.TINY
+    rng = np.random.default_rng(8)
+    Hf, Wf, Cf, s = w.feat_h, w.feat_w, 8, w.feat_stride
+    feat = rng.standard_normal((1, 1, Hf, Wf, Cf)).astype(F32)
+    n = 2000
+    u = rng.uniform(0, w.img_w, n).astype(F32)
+    v = rng.uniform(0, w.img_h, n).astype(F32)
+    uvd = np.stack([u, v, np.ones(n, F32)], 1)[None]
+    out = oracle.gather(uvd, np.zeros((1, n), np.int8), feat, s)
+    gx = 2.0 * (u.astype(np.float64) / s) / (Wf - 1) - 1.0
+    gy = 2.0 * (v.astype(np.float64) / s) / (Hf - 1) - 1.0
+    grid = torch.from_numpy(np.stack([gx, gy], -1))[None, None]                 # [1,1,n,2]
+    img = torch.from_numpy(feat[0, 0]).double().permute(2, 0, 1)[None]          # [1,Cf,Hf,Wf]
+    ref = torch.nn.functional.grid_sample(img, grid, mode="bilinear", padding_mode="border",
+                                          align_corners=True)[0, :, 0].T.numpy()
+    assert np.abs(out[0] - ref).max() < 1e-5
+
+
+# ------------------------------------------------------------------ O7 routing
+def test_routing_boundaries_are_far(oracle):
+    lut = ((3, 3, 3), (0, 1, 2))
+    rows = [(12, 16), (nxt(12, 0), 16), (24, 32), (24, nxt(32, 0)), (0, 0), (100, 0), (-12, -16),
+            (np.nan, 0), (0, np.nan)]
+    ex = oracle.route(_pts(rows), np.ones((1, len(rows)), np.uint8), (20.0, 40.0), lut)
+    assert list(ex[0]) == [1, 0, 2, 1, 0, 2, 1, 0, 0]
+    ex = oracle.route(_pts(rows), np.zeros((1, len(rows)), np.uint8), (20.0, 40.0), lut)
+    assert (ex == 3).all()
+    lut2 = gen.LUT_NUSCENES
+    rows = [(21, 28), (nxt(21, 0), 28), (30, 40), (30, nxt(40, 0))]
+    ex = oracle.route(_pts(rows), np.ones((1, 4), np.uint8), (35.0, 50.0), lut2)
+    assert list(ex[0]) == [1, 0, 3, 1]
+    ex = oracle.route(_pts(rows), np.zeros((1, 4), np.uint8), (35.0, 50.0), lut2)
+    assert list(ex[0]) == [2, 2, 3, 2]
+
+
+def test_routing_uses_the_papers_thresholds(oracle):
+    vals = {}
+    with open(os.path.join(GOLDEN, "sad_thresholds.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                k, v = line.split()
+                vals[k] = float(v)
+    assert gen.NUSCENES.thresholds[0] == vals["D_nuscenes_m"]
+    for D in (vals["D_kitti_m"], vals["D_nuscenes_m"]):
+        rows = [(D, 0.0), (nxt(D, 0), 0.0), (0.0, -D)]
+        ex = oracle.route(_pts(rows), np.ones((1, 3), np.uint8), (D,), ((9, 9), (0, 1)))
+        assert list(ex[0]) == [1, 0, 1]                  # exactly at D -> the farther bucket
+
+
+def test_lut_is_enumerated_exhaustively(oracle):
+    th = (1.0, 2.0, 3.0, 4.0, 5.0, 6.0, 7.0)
+    lut = (tuple(range(8, 16)), tuple(range(0, 8)))
+    rows = [(t + 0.5, 0.0) for t in range(8)]
+    for vis in (0, 1, 0x20, 0xFF):
+        ex = oracle.route(_pts(rows), np.full((1, 8), vis, np.uint8), th, lut)
+        assert list(ex[0]) == [(0 if vis else 8) + d for d in range(8)]
+
+
+# ------------------------------------------------------------------ O8 dispatch
+def test_dispatch_against_python_stable_sort(oracle):
+    rng = np.random.default_rng(9)
+    B, N, C, Cf, E = 3, 777, 5, 6, 4
+    expert = rng.integers(0, E, size=(B, N)).astype(np.uint8)
+    expert[1] = 2                                         # all one expert
+    expert[2][expert[2] == 1] = 3                         # an empty expert
+    pts = rng.standard_normal((B, N, C)).astype(F32)
+    fts = rng.standard_normal((B, N, Cf)).astype(F32)
+    off, perm, pout, fout = oracle.dispatch(expert, pts, fts, E)
+    for b in range(B):
+        want = sorted(range(N), key=lambda i: expert[b, i])       # Python's sort is stable
+        assert list(perm[b]) == want
+        cnt = [int((expert[b] == e).sum()) for e in range(E)]
+        assert list(off[b]) == [sum(cnt[:e]) for e in range(E + 1)]
+        assert np.array_equal(pout[b], pts[b][want]) and np.array_equal(fout[b], fts[b][want])
+    assert list(off[1]) == [0, 0, 0, N, N]
+
+
+def test_dispatch_invariants_on_generated_batch(oracle):
+    w = gen.NUSCENES.with_shape(2, 5000)
+    r = oracle.bridge(w, gen.make_batch(w))
+    off, perm, ex = r["offsets"], r["perm"], r["expert"]
+    for b in range(2):
+        assert sorted(perm[b]) == list(range(w.N))
+        assert (np.diff(off[b]) >= 0).all() and off[b][0] == 0 and off[b][-1] == w.N
+        e_sorted = ex[b][perm[b]]
+        assert (np.diff(e_sorted.astype(int)) >= 0).all()
+        for e in range(w.num_experts):
+            seg = perm[b][off[b][e]:off[b][e + 1]]
+            assert (np.diff(seg) > 0).all() and (ex[b][seg] == e).all()
+    assert len(np.unique(ex)) == 4                        # every expert of the workload is exercised
+
+
+def test_dense_frame_recipe_hits_the_stated_occupancy(oracle):
+    w = gen.DENSE
+    pts = gen.make_points(w, 0)[None]
+    g = w.grids[1]
+    r = oracle.voxelize(pts, g.min, g.voxel, g.dims, 0)
+    assert 150 <= r["counts"].max() <= 300
+    capped = oracle.voxelize(pts, g.min, g.voxel, g.dims, g.max_points)
+    assert capped["counts"].max() == 32 and (r["counts"] > 32).sum() > 100
