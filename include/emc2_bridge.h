@@ -1,0 +1,169 @@
+/*
+ * emc2_bridge.h -- C ABI of the B200 (sm_100a) multimodal data bridge and dispatch.
+ *
+ * The library implements, as CUDA kernels, the non-learned work that runs on
+ * every frame before any expert model of EMC2 (arXiv 2507.04123):
+ *   - the Adaptive Multimodal Data Bridge's preprocessing (Sec. 3.1): LiDAR
+ *     voxelization at two grid scales with per-voxel counts and mean features,
+ *     the BEV pseudo-image the 2D expert consumes (Sec. 3.3), LiDAR-to-camera
+ *     projection and sampling of image features, with zero rows where a point
+ *     has no pixel (Fig. 5);
+ *   - the Scenario-Adaptive Dispatcher's distance rule (Sec. 3.2: "close" is
+ *     < D, "distant" is >= D), applied per point together with visibility;
+ *   - the dispatch of points and features into contiguous per-expert buffers,
+ *     indexed by prefix sums (Sec. 3.6).
+ *
+ * General rules
+ *   - Every pointer named d_* is DEVICE memory on the handle's device, owned by
+ *     the caller, contiguous, row-major and 16-byte aligned.  Pointers named
+ *     h_* or without prefix are HOST memory.  The library never frees or keeps
+ *     a caller pointer after the call has been enqueued.
+ *   - The three stage calls only enqueue kernels on `cuda_stream` (a
+ *     cudaStream_t passed as void*, NULL = legacy default stream).  They do not
+ *     allocate, do not synchronise and do not touch the host except to return.
+ *   - One handle serves one device and one stream at a time; it is not
+ *     thread-safe.  Calls on the same handle must be ordered on the stream.
+ *   - Errors are returned as negative emc2_status_t values.  Errors the host
+ *     can see (null or misaligned pointer, sizes over the configured maxima)
+ *     return at once and enqueue nothing.  Errors only the device can see
+ *     (more unique voxels than `capacity`) set a sticky status word that
+ *     emc2_bridge_status() reads.  Nothing aborts, traps or prints.
+ *   - There is no CPU fallback: without a CUDA device create() fails.
+ */
+#ifndef EMC2_BRIDGE_H
+#define EMC2_BRIDGE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    EMC2_OK = 0,
+    EMC2_ERR_INVALID_ARG = -1, /* null/misaligned pointer, B or N outside the configured maxima */
+    EMC2_ERR_BAD_CONFIG = -2,  /* emc2_config_t rejected by emc2_bridge_create */
+    EMC2_ERR_CUDA = -3,        /* a CUDA runtime call failed; see emc2_bridge_last_cuda_error */
+    EMC2_ERR_CAPACITY = -4,    /* more unique voxels than capacity[s] (device-detected, sticky) */
+    EMC2_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (device-detected, sticky) */
+    EMC2_ERR_INTERNAL = -6
+} emc2_status_t;
+
+#define EMC2_MAX_CAMERAS 8
+#define EMC2_MAX_THRESHOLDS 7
+#define EMC2_MAX_EXPERTS 16
+#define EMC2_MAX_BATCH 32
+
+typedef struct emc2_bridge emc2_bridge_t; /* opaque; owns scratch memory and the device status word */
+
+/* One voxel grid (Sec. 3.1 "multi-scale preprocessing").  A point p lies in cell
+ * i_d = floor((p_d - min[d]) / voxel[d]) (fp32 subtract, fp32 IEEE divide) and is inside the
+ * grid iff 0 <= i_d < dims[d] on all three axes; non-finite coordinates are outside. */
+typedef struct {
+    float min[3];       /* lower corner (x, y, z), metres */
+    float voxel[3];     /* cell size (x, y, z), metres, > 0 */
+    int32_t dims[3];    /* cells along (x, y, z) = (Gx, Gy, Gz) */
+    int32_t max_points; /* per-voxel cap; 0 = none.  With a cap a voxel keeps its max_points
+                           points of lowest index within the batch; the rest are dropped. */
+} emc2_grid_t;
+
+typedef struct {
+    int32_t device;       /* CUDA device ordinal */
+    int32_t max_batch;    /* largest B of any call, 1..EMC2_MAX_BATCH */
+    int32_t max_points;   /* largest N (points per frame) of any call */
+    int32_t point_floats; /* C: floats per point, 4 (x,y,z,intensity) or 5 (+ time lag) */
+    emc2_grid_t grid[2];  /* [0] fine voxels, [1] pillars (dims[2] == 1) */
+    int32_t num_cameras;  /* K, 1..EMC2_MAX_CAMERAS */
+    int32_t img_h, img_w; /* image size in pixels */
+    int32_t feat_h, feat_w, feat_c; /* feature map size; feat_c a multiple of 4 */
+    int32_t feat_stride;  /* s: texel (j, i) is the sample at pixel (j*s, i*s); a power of two */
+    float min_depth;      /* a point is visible only if its depth is > min_depth */
+    int32_t num_thresholds;                /* T, 0..EMC2_MAX_THRESHOLDS */
+    float thresholds[EMC2_MAX_THRESHOLDS]; /* ascending planar ranges in metres */
+    int32_t num_experts;                   /* E, 1..EMC2_MAX_EXPERTS */
+    uint8_t lut[2][8]; /* expert = lut[visible ? 1 : 0][number of thresholds reached]; < E */
+} emc2_config_t;
+
+/* Validates the configuration, selects the device and allocates all scratch memory the stage
+ * calls will ever need for (max_batch, max_points).  Returns EMC2_ERR_BAD_CONFIG for an
+ * unusable configuration (zero voxel size, more than 2^32 - 1 cells per batch, a cap on a grid
+ * too large for a direct count table, feat_c not a multiple of 4, stride not a power of two,
+ * lut entry >= num_experts, ...), EMC2_ERR_CUDA if the device or memory is unavailable. */
+int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out);
+
+/* Stage 1 (Sec. 3.1; BEV for the 2D expert of Sec. 3.3).  For each scale s in {0, 1}:
+ *   d_coords[s]      int32 [capacity[s], 4]  unique voxels as (b, z, y, x), ascending in that order
+ *   d_counts[s]      int32 [capacity[s]]     points kept in the voxel (<= max_points if capped)
+ *   d_mean[s]        float [capacity[s], C]  mean of the kept points over all C channels
+ *   d_point_voxel[s] int32 [B, N] or NULL    row of the point's voxel; -1 if outside the grid or
+ *                                            dropped by the cap
+ *   d_num_voxels     int32 [2]               number of unique voxels found per scale (true count
+ *                                            even when it exceeds capacity[s])
+ *   d_bev            float [B, C, Gy, Gx] of grid[1], or NULL: pillar means at (iy, ix), else 0
+ * d_points is float [B, N, C].  Rows past num_voxels are left untouched.  If a scale finds more
+ * voxels than capacity[s], rows past capacity are not written and EMC2_ERR_CAPACITY becomes
+ * sticky.  d_coords, d_counts, d_mean and capacity are HOST arrays of two entries. */
+int emc2_voxelize(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_points,
+                  int32_t* const d_coords[2], int32_t* const d_counts[2], float* const d_mean[2],
+                  int32_t* const d_point_voxel[2], const int32_t capacity[2], int32_t* d_num_voxels,
+                  float* d_bev, void* cuda_stream);
+
+/* Stage 2 (Sec. 3.1 projection "based on depth information"; Fig. 5 zero fill).
+ *   d_proj      float [B, K, 3, 4]  row-major; maps LiDAR-frame (x, y, z, 1) to (u*d, v*d, d)
+ *   d_feat      float [B, K, Hf, Wf, Cf]  channels-last feature maps
+ *   d_uvd       float [B, N, 3]   (u, v, depth) in the lowest-index camera that sees the point,
+ *                                 or (-1, -1, depth in camera 0 [0 if not finite]) if none does
+ *   d_vis_mask  uint8 [B, N]      bit k set iff depth_k > min_depth, 0 <= u < W and 0 <= v < H
+ *   d_cam       int8  [B, N]      that camera, or -1
+ *   d_gathered  float [B, N, Cf]  bilinear sample at (u/s, v/s), taps clamped to the map edge;
+ *                                 all zeros for points no camera sees */
+int emc2_project_gather(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_points,
+                        const float* d_proj, const float* d_feat, float* d_uvd, uint8_t* d_vis_mask,
+                        int8_t* d_cam, float* d_gathered, void* cuda_stream);
+
+/* Stages 3 and 4 (Sec. 3.2 distance rule; Sec. 3.6 prefix sums).  Per frame b:
+ *   d_expert      uint8 [B, N]     lut[vis_mask != 0][#{t : x*x + y*y >= thresholds[t]^2}]
+ *   d_offsets     int32 [B, E+1]   exclusive prefix sum of per-expert counts; offsets[b][E] = N
+ *   d_perm        int32 [B, N]     frame-local source index of output row j (stable: ascending
+ *                                  inside each expert's segment)
+ *   d_points_out  float [B, N, C]  points[b][perm[b][j]]
+ *   d_feat_out    float [B, N, Cf] gathered[b][perm[b][j]]
+ * d_vis_mask and d_gathered are the outputs of emc2_project_gather (or any buffers of that
+ * shape).  Outputs must not alias inputs. */
+int emc2_route_dispatch(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_points,
+                        const uint8_t* d_vis_mask, const float* d_gathered, uint8_t* d_expert,
+                        int32_t* d_offsets, int32_t* d_perm, float* d_points_out, float* d_feat_out,
+                        void* cuda_stream);
+
+/* Waits for `cuda_stream`, then returns and clears the sticky device status: EMC2_OK,
+ * EMC2_ERR_CAPACITY, EMC2_ERR_TIMEOUT or EMC2_ERR_CUDA. */
+int emc2_bridge_status(emc2_bridge_t* bridge, void* cuda_stream);
+
+/* Frees scratch memory.  The caller must have synchronised the streams it used.  NULL is OK. */
+int emc2_bridge_destroy(emc2_bridge_t* bridge);
+
+/* Text for a status code (static storage, never NULL). */
+const char* emc2_status_string(int status);
+
+/* cudaError_t of the last failed runtime call on this handle (0 if none). */
+int emc2_bridge_last_cuda_error(const emc2_bridge_t* bridge);
+
+/* Bytes of device scratch the handle owns. */
+size_t emc2_bridge_scratch_bytes(const emc2_bridge_t* bridge);
+
+/* Measurement aids (no paper counterpart).  The library counts its own kernel launches per
+ * kernel kind; with profiling enabled every launch is also bracketed by CUDA events on the
+ * launching stream.  emc2_bridge_profile_read() synchronises those events and fills, for
+ * kernel kind k in [0, emc2_bridge_kernel_kinds()), the launches and the summed device
+ * milliseconds since the last reset (ms only while profiling was enabled); it then resets
+ * the counters if `reset` is non-zero.  Arrays are HOST memory and may be NULL. */
+int emc2_bridge_kernel_kinds(void);
+const char* emc2_bridge_kernel_name(int kind);
+int emc2_bridge_profile_enable(emc2_bridge_t* bridge, int enable);
+int emc2_bridge_profile_read(emc2_bridge_t* bridge, int64_t* launches, double* ms, int reset);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EMC2_BRIDGE_H */

@@ -1,0 +1,282 @@
+"""Thin Python binding of libemc2_bridge.so (argument marshalling only).
+
+Every step of the path runs inside the CUDA library; this module allocates
+torch tensors for the outputs, passes ``data_ptr()`` values and the current
+CUDA stream through the C ABI declared in ``include/emc2_bridge.h`` and turns
+status codes into exceptions.  There is no CPU fallback: if the shared library
+is missing or no CUDA device is present, construction fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libemc2_bridge.so")
+
+EMC2_OK = 0
+EMC2_ERR_INVALID_ARG = -1
+EMC2_ERR_BAD_CONFIG = -2
+EMC2_ERR_CUDA = -3
+EMC2_ERR_CAPACITY = -4
+EMC2_ERR_TIMEOUT = -5
+EMC2_ERR_INTERNAL = -6
+
+# Every symbol include/emc2_bridge.h declares.
+ABI_SYMBOLS = (
+    "emc2_bridge_create", "emc2_voxelize", "emc2_project_gather", "emc2_route_dispatch",
+    "emc2_bridge_status", "emc2_bridge_destroy", "emc2_status_string", "emc2_bridge_last_cuda_error",
+    "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
+    "emc2_bridge_profile_enable", "emc2_bridge_profile_read",
+)
+
+
+class Emc2Grid(ctypes.Structure):
+    _fields_ = [("min", ctypes.c_float * 3), ("voxel", ctypes.c_float * 3),
+                ("dims", ctypes.c_int32 * 3), ("max_points", ctypes.c_int32)]
+
+
+class Emc2Config(ctypes.Structure):
+    _fields_ = [("device", ctypes.c_int32), ("max_batch", ctypes.c_int32),
+                ("max_points", ctypes.c_int32), ("point_floats", ctypes.c_int32),
+                ("grid", Emc2Grid * 2),
+                ("num_cameras", ctypes.c_int32), ("img_h", ctypes.c_int32), ("img_w", ctypes.c_int32),
+                ("feat_h", ctypes.c_int32), ("feat_w", ctypes.c_int32), ("feat_c", ctypes.c_int32),
+                ("feat_stride", ctypes.c_int32), ("min_depth", ctypes.c_float),
+                ("num_thresholds", ctypes.c_int32), ("thresholds", ctypes.c_float * 7),
+                ("num_experts", ctypes.c_int32), ("lut", (ctypes.c_uint8 * 8) * 2)]
+
+
+class Emc2Error(RuntimeError):
+    def __init__(self, status: int, where: str, text: str):
+        super().__init__(f"{where}: {text} (status {status})")
+        self.status = status
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with paper_2507_04123_b200.build.build(); "
+                           "there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, P = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER
+    lib.emc2_bridge_create.argtypes = [P(Emc2Config), P(vp)]
+    lib.emc2_voxelize.argtypes = [vp, i32, i32, vp, P(vp), P(vp), P(vp), P(vp), P(i32), vp, vp, vp]
+    lib.emc2_project_gather.argtypes = [vp, i32, i32] + [vp] * 8
+    lib.emc2_route_dispatch.argtypes = [vp, i32, i32] + [vp] * 9
+    lib.emc2_bridge_status.argtypes = [vp, vp]
+    lib.emc2_bridge_destroy.argtypes = [vp]
+    lib.emc2_status_string.argtypes = [ctypes.c_int]
+    lib.emc2_status_string.restype = ctypes.c_char_p
+    lib.emc2_bridge_last_cuda_error.argtypes = [vp]
+    lib.emc2_bridge_scratch_bytes.argtypes = [vp]
+    lib.emc2_bridge_scratch_bytes.restype = ctypes.c_size_t
+    lib.emc2_bridge_kernel_name.argtypes = [ctypes.c_int]
+    lib.emc2_bridge_kernel_name.restype = ctypes.c_char_p
+    lib.emc2_bridge_profile_enable.argtypes = [vp, ctypes.c_int]
+    lib.emc2_bridge_profile_read.argtypes = [vp, P(ctypes.c_int64), P(ctypes.c_double), ctypes.c_int]
+    _lib = lib
+    return lib
+
+
+def make_config(*, device: int, max_batch: int, max_points: int, point_floats: int, grids,
+                num_cameras: int, img_h: int, img_w: int, feat_h: int, feat_w: int, feat_c: int,
+                feat_stride: int, min_depth: float, thresholds: Sequence[float], num_experts: int,
+                lut: Sequence[Sequence[int]]) -> Emc2Config:
+    """Fills an emc2_config_t.  ``grids`` is two objects with min, voxel, dims, max_points."""
+    c = Emc2Config()
+    c.device, c.max_batch, c.max_points, c.point_floats = device, max_batch, max_points, point_floats
+    for s in range(2):
+        g = grids[s]
+        for d in range(3):
+            c.grid[s].min[d] = g.min[d]
+            c.grid[s].voxel[d] = g.voxel[d]
+            c.grid[s].dims[d] = g.dims[d]
+        c.grid[s].max_points = g.max_points
+    c.num_cameras, c.img_h, c.img_w = num_cameras, img_h, img_w
+    c.feat_h, c.feat_w, c.feat_c, c.feat_stride = feat_h, feat_w, feat_c, feat_stride
+    c.min_depth = min_depth
+    c.num_thresholds = len(thresholds)
+    for t, v in enumerate(thresholds):
+        c.thresholds[t] = v
+    c.num_experts = num_experts
+    for v in range(2):
+        row = list(lut[v])[:8]
+        for d, e in enumerate(row):
+            c.lut[v][d] = e
+    return c
+
+
+def config_from_workload(w, device: int = 0, max_batch: Optional[int] = None,
+                         max_points: Optional[int] = None) -> Emc2Config:
+    """emc2_config_t for a workload description with the fields of emc2_gen.Workload."""
+    return make_config(device=device, max_batch=max_batch or w.B, max_points=max_points or w.N,
+                       point_floats=w.C, grids=w.grids, num_cameras=w.K, img_h=w.img_h, img_w=w.img_w,
+                       feat_h=w.feat_h, feat_w=w.feat_w, feat_c=w.feat_c, feat_stride=w.feat_stride,
+                       min_depth=w.min_depth, thresholds=w.thresholds, num_experts=w.num_experts,
+                       lut=w.lut)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _check(t: torch.Tensor, dtype, shape, name: str, device) -> None:
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous() or t.device != device:
+        raise ValueError(f"{name}: expected contiguous {dtype} {tuple(shape)} on {device}, "
+                         f"got {t.dtype} {tuple(t.shape)} on {t.device}")
+
+
+class Bridge:
+    """One emc2_bridge_t handle.  Methods mirror the C entry points."""
+
+    def __init__(self, config: Emc2Config):
+        if not torch.cuda.is_available():
+            raise RuntimeError("emc2 bridge needs a CUDA device; there is no CPU path")
+        self.lib = load_library()
+        self.cfg = config
+        self.device = torch.device("cuda", config.device)
+        self._h = ctypes.c_void_p()
+        rc = self.lib.emc2_bridge_create(ctypes.byref(config), ctypes.byref(self._h))
+        self._raise(rc, "emc2_bridge_create")
+
+    # ------------------------------------------------------------------ helpers
+    def _raise(self, rc: int, where: str) -> None:
+        if rc != EMC2_OK:
+            raise Emc2Error(rc, where, self.lib.emc2_status_string(rc).decode())
+
+    def _stream(self) -> int:
+        return torch.cuda.current_stream(self.device).cuda_stream
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            torch.cuda.synchronize(self.device)
+            self.lib.emc2_bridge_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def scratch_bytes(self) -> int:
+        return int(self.lib.emc2_bridge_scratch_bytes(self._h))
+
+    # ------------------------------------------------------------------ stage calls
+    def voxelize(self, points: torch.Tensor, capacity: Optional[Sequence[int]] = None,
+                 want_point_voxel: bool = True, want_bev: bool = True,
+                 out: Optional[Dict[str, object]] = None) -> Dict[str, object]:
+        """emc2_voxelize.  Returns device tensors; rows past num_voxels[s] are unspecified."""
+        B, N, C = points.shape
+        _check(points, torch.float32, (B, N, self.cfg.point_floats), "points", self.device)
+        cap = list(capacity) if capacity is not None else [B * N, B * N]
+        dev = self.device
+        if out is None:
+            out = {
+                "coords": [torch.empty((max(cap[s], 1), 4), dtype=torch.int32, device=dev) for s in range(2)],
+                "counts": [torch.empty((max(cap[s], 1),), dtype=torch.int32, device=dev) for s in range(2)],
+                "mean": [torch.empty((max(cap[s], 1), C), dtype=torch.float32, device=dev) for s in range(2)],
+                "point_voxel": [torch.empty((B, N), dtype=torch.int32, device=dev) for _ in range(2)]
+                if want_point_voxel else None,
+                "num_voxels": torch.empty((2,), dtype=torch.int32, device=dev),
+                "bev": torch.empty((B, C, self.cfg.grid[1].dims[1], self.cfg.grid[1].dims[0]),
+                                   dtype=torch.float32, device=dev) if want_bev else None,
+            }
+        arr = ctypes.c_void_p * 2
+        pv = out["point_voxel"]
+        rc = self.lib.emc2_voxelize(
+            self._h, B, N, points.data_ptr(),
+            arr(*[t.data_ptr() for t in out["coords"]]), arr(*[t.data_ptr() for t in out["counts"]]),
+            arr(*[t.data_ptr() for t in out["mean"]]),
+            arr(*[t.data_ptr() for t in pv]) if pv is not None else None,
+            (ctypes.c_int32 * 2)(*cap), out["num_voxels"].data_ptr(), _ptr(out["bev"]), self._stream())
+        self._raise(rc, "emc2_voxelize")
+        return out
+
+    def project_gather(self, points: torch.Tensor, proj: torch.Tensor, feat: torch.Tensor,
+                       out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        """emc2_project_gather."""
+        B, N, C = points.shape
+        c = self.cfg
+        _check(points, torch.float32, (B, N, c.point_floats), "points", self.device)
+        _check(proj, torch.float32, (B, c.num_cameras, 3, 4), "proj", self.device)
+        _check(feat, torch.float32, (B, c.num_cameras, c.feat_h, c.feat_w, c.feat_c), "feat", self.device)
+        if out is None:
+            dev = self.device
+            out = {"uvd": torch.empty((B, N, 3), dtype=torch.float32, device=dev),
+                   "vis_mask": torch.empty((B, N), dtype=torch.uint8, device=dev),
+                   "cam": torch.empty((B, N), dtype=torch.int8, device=dev),
+                   "gathered": torch.empty((B, N, c.feat_c), dtype=torch.float32, device=dev)}
+        rc = self.lib.emc2_project_gather(self._h, B, N, points.data_ptr(), proj.data_ptr(), feat.data_ptr(),
+                                          out["uvd"].data_ptr(), out["vis_mask"].data_ptr(),
+                                          out["cam"].data_ptr(), out["gathered"].data_ptr(), self._stream())
+        self._raise(rc, "emc2_project_gather")
+        return out
+
+    def route_dispatch(self, points: torch.Tensor, vis_mask: torch.Tensor, gathered: torch.Tensor,
+                       out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        """emc2_route_dispatch."""
+        B, N, C = points.shape
+        c = self.cfg
+        _check(points, torch.float32, (B, N, c.point_floats), "points", self.device)
+        _check(vis_mask, torch.uint8, (B, N), "vis_mask", self.device)
+        _check(gathered, torch.float32, (B, N, c.feat_c), "gathered", self.device)
+        if out is None:
+            dev = self.device
+            out = {"expert": torch.empty((B, N), dtype=torch.uint8, device=dev),
+                   "offsets": torch.empty((B, c.num_experts + 1), dtype=torch.int32, device=dev),
+                   "perm": torch.empty((B, N), dtype=torch.int32, device=dev),
+                   "points_out": torch.empty_like(points),
+                   "feat_out": torch.empty_like(gathered)}
+        rc = self.lib.emc2_route_dispatch(self._h, B, N, points.data_ptr(), vis_mask.data_ptr(),
+                                          gathered.data_ptr(), out["expert"].data_ptr(),
+                                          out["offsets"].data_ptr(), out["perm"].data_ptr(),
+                                          out["points_out"].data_ptr(), out["feat_out"].data_ptr(),
+                                          self._stream())
+        self._raise(rc, "emc2_route_dispatch")
+        return out
+
+    def status(self, raise_on_error: bool = True) -> int:
+        """emc2_bridge_status: waits for the current stream, returns the sticky device status."""
+        rc = self.lib.emc2_bridge_status(self._h, self._stream())
+        if raise_on_error:
+            self._raise(rc, "emc2_bridge_status")
+        return rc
+
+    # ------------------------------------------------------------------ whole path
+    def run(self, points: torch.Tensor, proj: torch.Tensor, feat: torch.Tensor,
+            bufs: Optional[Dict[str, object]] = None) -> Dict[str, object]:
+        """The three stage calls back to back on the current stream (no host sync)."""
+        bufs = bufs if bufs is not None else {}
+        bufs["vox"] = self.voxelize(points, out=bufs.get("vox"))
+        bufs["pg"] = self.project_gather(points, proj, feat, out=bufs.get("pg"))
+        pg = bufs["pg"]
+        bufs["rd"] = self.route_dispatch(points, pg["vis_mask"], pg["gathered"], out=bufs.get("rd"))
+        return bufs
+
+    # ------------------------------------------------------------------ measurement aids
+    def kernel_names(self) -> List[str]:
+        n = self.lib.emc2_bridge_kernel_kinds()
+        return [self.lib.emc2_bridge_kernel_name(k).decode() for k in range(n)]
+
+    def profile_enable(self, enable: bool) -> None:
+        self._raise(self.lib.emc2_bridge_profile_enable(self._h, int(enable)), "emc2_bridge_profile_enable")
+
+    def profile_read(self, reset: bool = True) -> Dict[str, Tuple[int, float]]:
+        n = self.lib.emc2_bridge_kernel_kinds()
+        launches = (ctypes.c_int64 * n)()
+        ms = (ctypes.c_double * n)()
+        self._raise(self.lib.emc2_bridge_profile_read(self._h, launches, ms, int(reset)),
+                    "emc2_bridge_profile_read")
+        return {name: (int(launches[k]), float(ms[k])) for k, name in enumerate(self.kernel_names())}

@@ -1,0 +1,322 @@
+// Handle management and the extern "C" entry points of the bridge library.
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "bridge_internal.cuh"
+
+namespace emc2 {
+
+static const char* const kKernelNames[K_KINDS] = {
+    "vox_mark", "vox_reduce", "vox_blockscan", "vox_emit", "vox_accum", "vox_overflow", "vox_finalize",
+    "vox_clean", "bev_zero", "project_gather", "route_hist", "route_scan", "dispatch_scatter"};
+
+int check_cuda(emc2_bridge* h, cudaError_t e) {
+    if (e == cudaSuccess) return EMC2_OK;
+    if (h) h->last_cuda_error = (int)e;
+    return EMC2_ERR_CUDA;
+}
+
+LaunchScope::LaunchScope(emc2_bridge* h_, int kind_, cudaStream_t st_) : h(h_), kind(kind_), st(st_) {
+    h->launches[kind] += 1;
+    if (!h->profiling) return;
+    for (cudaEvent_t* e : {&a, &b}) {
+        if (!h->event_pool.empty()) {
+            *e = h->event_pool.back();
+            h->event_pool.pop_back();
+        } else if (cudaEventCreate(e) != cudaSuccess) {
+            *e = nullptr;
+        }
+    }
+    if (a) cudaEventRecord(a, st);
+}
+
+LaunchScope::~LaunchScope() {
+    if (!h->profiling || !a || !b) return;
+    cudaEventRecord(b, st);
+    h->recs.push_back({kind, a, b});
+}
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() {
+        int cur;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int validate(const emc2_config_t& c) {
+    if (c.device < 0) return EMC2_ERR_BAD_CONFIG;
+    if (c.max_batch < 1 || c.max_batch > EMC2_MAX_BATCH) return EMC2_ERR_BAD_CONFIG;
+    if (c.max_points < 1) return EMC2_ERR_BAD_CONFIG;
+    if ((int64_t)c.max_batch * c.max_points > (int64_t)1 << 30) return EMC2_ERR_BAD_CONFIG;
+    if (c.point_floats != 4 && c.point_floats != 5) return EMC2_ERR_BAD_CONFIG;
+    for (int s = 0; s < 2; ++s) {
+        const emc2_grid_t& g = c.grid[s];
+        uint64_t cells = 1;
+        for (int d = 0; d < 3; ++d) {
+            if (!(g.voxel[d] > 0.0f) || !std::isfinite(g.voxel[d]) || !std::isfinite(g.min[d]))
+                return EMC2_ERR_BAD_CONFIG;
+            if (g.dims[d] < 1 || g.dims[d] > (1 << 24)) return EMC2_ERR_BAD_CONFIG;
+            cells *= (uint64_t)g.dims[d];
+            if (cells > 0xFFFFFFFFull) return EMC2_ERR_BAD_CONFIG;
+        }
+        if (cells * (uint64_t)c.max_batch > 0xFFFFFF00ull) return EMC2_ERR_BAD_CONFIG;
+        if (g.max_points < 0) return EMC2_ERR_BAD_CONFIG;
+        // The per-voxel cap needs the per-cell point count, which only the count table holds.
+        if (g.max_points > 0 && cells * (uint64_t)c.max_batch > (uint64_t)kMaxTableCells)
+            return EMC2_ERR_BAD_CONFIG;
+    }
+    if (c.grid[1].dims[2] != 1) return EMC2_ERR_BAD_CONFIG;
+    if (c.num_cameras < 1 || c.num_cameras > EMC2_MAX_CAMERAS) return EMC2_ERR_BAD_CONFIG;
+    if (c.img_h < 1 || c.img_w < 1 || c.feat_h < 1 || c.feat_w < 1) return EMC2_ERR_BAD_CONFIG;
+    if (c.feat_c < 4 || (c.feat_c & 3)) return EMC2_ERR_BAD_CONFIG;
+    if (!is_pow2(c.feat_stride)) return EMC2_ERR_BAD_CONFIG;
+    // Every visible pixel must fall inside the map: (dim - 1) / stride <= feat_dim - 1.
+    if ((c.img_h - 1) / c.feat_stride > c.feat_h - 1 || (c.img_w - 1) / c.feat_stride > c.feat_w - 1)
+        return EMC2_ERR_BAD_CONFIG;
+    if ((uint64_t)c.max_batch * c.num_cameras * c.feat_h * c.feat_w * (uint64_t)(c.feat_c / 4) > 0xFFFFFFFFFFFFull)
+        return EMC2_ERR_BAD_CONFIG;
+    if (!(c.min_depth >= 0.0f)) return EMC2_ERR_BAD_CONFIG;
+    if (c.num_thresholds < 0 || c.num_thresholds > EMC2_MAX_THRESHOLDS) return EMC2_ERR_BAD_CONFIG;
+    for (int t = 0; t < c.num_thresholds; ++t) {
+        if (!(c.thresholds[t] >= 0.0f) || !std::isfinite(c.thresholds[t])) return EMC2_ERR_BAD_CONFIG;
+        if (t && !(c.thresholds[t] >= c.thresholds[t - 1])) return EMC2_ERR_BAD_CONFIG;
+    }
+    if (c.num_experts < 1 || c.num_experts > EMC2_MAX_EXPERTS) return EMC2_ERR_BAD_CONFIG;
+    for (int v = 0; v < 2; ++v)
+        for (int d = 0; d <= c.num_thresholds; ++d)
+            if (c.lut[v][d] >= c.num_experts) return EMC2_ERR_BAD_CONFIG;
+    return EMC2_OK;
+}
+
+struct SlabPlan {
+    size_t off = 0;
+    size_t take(size_t bytes) {
+        const size_t o = off;
+        off += (bytes + 255) & ~(size_t)255;
+        return o;
+    }
+};
+
+}  // namespace
+}  // namespace emc2
+
+using namespace emc2;
+
+extern "C" {
+
+int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
+    if (!config || !out) return EMC2_ERR_INVALID_ARG;
+    *out = nullptr;
+    int rc = validate(*config);
+    if (rc != EMC2_OK) return rc;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || config->device >= ndev) return EMC2_ERR_CUDA;
+    emc2_bridge* h = new (std::nothrow) emc2_bridge();
+    if (!h) return EMC2_ERR_INTERNAL;
+    h->cfg = *config;
+    DeviceGuard guard(config->device);
+    if (!guard.ok) { delete h; return EMC2_ERR_CUDA; }
+
+    const emc2_config_t& c = h->cfg;
+    const size_t maxpts = (size_t)c.max_batch * c.max_points;
+    for (int t = 0; t < EMC2_MAX_THRESHOLDS; ++t)
+        h->thr2[t] = t < c.num_thresholds ? c.thresholds[t] * c.thresholds[t] : 0.0f;
+
+    // Plan the slab: everything the stage calls need, allocated once.
+    SlabPlan plan;
+    size_t o_store[2], o_summary[2], o_prefix[2], o_sums[2], o_bs[2], o_bo[2], o_ovf[2][4], o_tot[2];
+    for (int s = 0; s < 2; ++s) {
+        ScaleDev& d = h->scale[s];
+        const emc2_grid_t& g = c.grid[s];
+        for (int k = 0; k < 3; ++k) { d.mn[k] = g.min[k]; d.vs[k] = g.voxel[k]; d.dims[k] = g.dims[k]; }
+        d.cap = g.max_points;
+        d.cells = (uint32_t)((uint64_t)g.dims[0] * g.dims[1] * g.dims[2]);
+        const uint64_t total_cells = (uint64_t)d.cells * c.max_batch;
+        d.mode = total_cells <= (uint64_t)kMaxTableCells ? MODE_TABLE : MODE_BITMAP;
+        const uint64_t per_chunk = d.mode == MODE_BITMAP ? 256 : 8;
+        d.nchunks = (uint32_t)((total_cells + per_chunk - 1) / per_chunk);
+        d.nsumwords = (d.nchunks + 31) / 32;
+        d.scan_blocks = (int)((d.nsumwords + kThreads - 1) / kThreads);
+        o_store[s] = plan.take((size_t)d.nsumwords * 32 * kChunkBytes);
+        o_summary[s] = plan.take((size_t)d.nsumwords * 4);
+        o_prefix[s] = plan.take((size_t)d.nsumwords * 32 * 4);
+        o_sums[s] = plan.take(maxpts * c.point_floats * sizeof(double));
+        o_bs[s] = plan.take((size_t)d.scan_blocks * 3 * sizeof(int));
+        o_bo[s] = plan.take((size_t)d.scan_blocks * 3 * sizeof(int));
+        for (int k = 0; k < 4; ++k) o_ovf[s][k] = d.cap > 0 ? plan.take(maxpts * sizeof(int)) : 0;
+        o_tot[s] = plan.take(4 * sizeof(int));
+    }
+    h->max_tiles = (c.max_points + kTile - 1) / kTile;
+    const size_t tile_ints = (size_t)c.max_batch * h->max_tiles * c.num_experts;
+    const size_t o_tc = plan.take(tile_ints * sizeof(int));
+    const size_t o_tb = plan.take(tile_ints * sizeof(int));
+    const size_t o_status = plan.take(sizeof(int));
+
+    h->slab_bytes = plan.off;
+    cudaError_t e = cudaMalloc(&h->slab, h->slab_bytes);
+    if (e != cudaSuccess) { h->slab = nullptr; delete h; return EMC2_ERR_CUDA; }
+    // The voxel stores and summaries must be all-zero between calls; every call restores that.
+    e = cudaMemset(h->slab, 0, h->slab_bytes);
+    if (e != cudaSuccess) { cudaFree(h->slab); delete h; return EMC2_ERR_CUDA; }
+    char* base = static_cast<char*>(h->slab);
+    for (int s = 0; s < 2; ++s) {
+        ScaleDev& d = h->scale[s];
+        d.store = reinterpret_cast<uint32_t*>(base + o_store[s]);
+        d.summary = reinterpret_cast<uint32_t*>(base + o_summary[s]);
+        d.chunk_prefix = reinterpret_cast<uint32_t*>(base + o_prefix[s]);
+        d.sums = reinterpret_cast<double*>(base + o_sums[s]);
+        d.blk_sums = reinterpret_cast<int*>(base + o_bs[s]);
+        d.blk_offs = reinterpret_cast<int*>(base + o_bo[s]);
+        d.ovf_off = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][0]) : nullptr;
+        d.ovf_cursor = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][1]) : nullptr;
+        d.ovf_vox = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][2]) : nullptr;
+        d.ovf_list = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][3]) : nullptr;
+        d.totals = reinterpret_cast<int*>(base + o_tot[s]);
+    }
+    h->d_tile_counts = reinterpret_cast<int*>(base + o_tc);
+    h->d_tile_base = reinterpret_cast<int*>(base + o_tb);
+    h->d_status = reinterpret_cast<int*>(base + o_status);
+    *out = h;
+    return EMC2_OK;
+}
+
+static int check_call(emc2_bridge* h, int32_t B, int32_t N) {
+    if (!h) return EMC2_ERR_INVALID_ARG;
+    if (B < 0 || N < 0 || B > h->cfg.max_batch || N > h->cfg.max_points) return EMC2_ERR_INVALID_ARG;
+    return EMC2_OK;
+}
+
+int emc2_voxelize(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points,
+                  int32_t* const d_coords[2], int32_t* const d_counts[2], float* const d_mean[2],
+                  int32_t* const d_point_voxel[2], const int32_t capacity[2], int32_t* d_num_voxels,
+                  float* d_bev, void* cuda_stream) {
+    int rc = check_call(h, B, N);
+    if (rc != EMC2_OK) return rc;
+    if (!d_points || !d_coords || !d_counts || !d_mean || !capacity || !d_num_voxels) return EMC2_ERR_INVALID_ARG;
+    if (!aligned16(d_points) || (d_bev && !aligned16(d_bev))) return EMC2_ERR_INVALID_ARG;
+    for (int s = 0; s < 2; ++s) {
+        if (!d_coords[s] || !d_counts[s] || !d_mean[s] || capacity[s] < 0) return EMC2_ERR_INVALID_ARG;
+        if (!aligned16(d_coords[s])) return EMC2_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity,
+                           d_num_voxels, d_bev, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int emc2_project_gather(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points, const float* d_proj,
+                        const float* d_feat, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
+                        float* d_gathered, void* cuda_stream) {
+    int rc = check_call(h, B, N);
+    if (rc != EMC2_OK) return rc;
+    if (!d_points || !d_proj || !d_feat || !d_uvd || !d_vis_mask || !d_cam || !d_gathered)
+        return EMC2_ERR_INVALID_ARG;
+    if (!aligned16(d_points) || !aligned16(d_feat) || !aligned16(d_gathered)) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_project_gather(h, B, N, d_points, d_proj, d_feat, d_uvd, d_vis_mask, d_cam, d_gathered,
+                                 static_cast<cudaStream_t>(cuda_stream));
+}
+
+int emc2_route_dispatch(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points,
+                        const uint8_t* d_vis_mask, const float* d_gathered, uint8_t* d_expert,
+                        int32_t* d_offsets, int32_t* d_perm, float* d_points_out, float* d_feat_out,
+                        void* cuda_stream) {
+    int rc = check_call(h, B, N);
+    if (rc != EMC2_OK) return rc;
+    if (!d_points || !d_vis_mask || !d_gathered || !d_expert || !d_offsets || !d_perm || !d_points_out ||
+        !d_feat_out)
+        return EMC2_ERR_INVALID_ARG;
+    if (!aligned16(d_points) || !aligned16(d_gathered) || !aligned16(d_feat_out)) return EMC2_ERR_INVALID_ARG;
+    if (d_points_out == d_points || d_feat_out == d_gathered) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_route_dispatch(h, B, N, d_points, d_vis_mask, d_gathered, d_expert, d_offsets, d_perm,
+                                 d_points_out, d_feat_out, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int emc2_bridge_status(emc2_bridge_t* h, void* cuda_stream) {
+    if (!h) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, h->d_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->d_status, 0, sizeof(int), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return check_cuda(h, e);
+    if (word & 2) return EMC2_ERR_TIMEOUT;
+    if (word & 1) return EMC2_ERR_CAPACITY;
+    return EMC2_OK;
+}
+
+int emc2_bridge_destroy(emc2_bridge_t* h) {
+    if (!h) return EMC2_OK;
+    DeviceGuard guard(h->cfg.device);
+    int rc = EMC2_OK;
+    for (ProfRec& r : h->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (cudaEvent_t e : h->event_pool) cudaEventDestroy(e);
+    if (h->slab && cudaFree(h->slab) != cudaSuccess) rc = EMC2_ERR_CUDA;
+    delete h;
+    return rc;
+}
+
+const char* emc2_status_string(int status) {
+    switch (status) {
+        case EMC2_OK: return "ok";
+        case EMC2_ERR_INVALID_ARG: return "invalid argument";
+        case EMC2_ERR_BAD_CONFIG: return "bad configuration";
+        case EMC2_ERR_CUDA: return "CUDA runtime error";
+        case EMC2_ERR_CAPACITY: return "more unique voxels than capacity";
+        case EMC2_ERR_TIMEOUT: return "bounded device wait timed out";
+        case EMC2_ERR_INTERNAL: return "internal error";
+        default: return "unknown status";
+    }
+}
+
+int emc2_bridge_last_cuda_error(const emc2_bridge_t* h) { return h ? h->last_cuda_error : 0; }
+size_t emc2_bridge_scratch_bytes(const emc2_bridge_t* h) { return h ? h->slab_bytes : 0; }
+
+int emc2_bridge_kernel_kinds(void) { return K_KINDS; }
+const char* emc2_bridge_kernel_name(int kind) { return kind >= 0 && kind < K_KINDS ? kKernelNames[kind] : ""; }
+
+int emc2_bridge_profile_enable(emc2_bridge_t* h, int enable) {
+    if (!h) return EMC2_ERR_INVALID_ARG;
+    h->profiling = enable != 0;
+    return EMC2_OK;
+}
+
+int emc2_bridge_profile_read(emc2_bridge_t* h, int64_t* launches, double* ms, int reset) {
+    if (!h) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    int rc = EMC2_OK;
+    for (ProfRec& r : h->recs) {
+        float t = 0.f;
+        cudaError_t e = cudaEventSynchronize(r.b);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&t, r.a, r.b);
+        if (e == cudaSuccess) h->ms[r.kind] += t; else rc = check_cuda(h, e);
+        h->event_pool.push_back(r.a);
+        h->event_pool.push_back(r.b);
+    }
+    h->recs.clear();
+    for (int k = 0; k < K_KINDS; ++k) {
+        if (launches) launches[k] = h->launches[k];
+        if (ms) ms[k] = h->ms[k];
+        if (reset) { h->launches[k] = 0; h->ms[k] = 0.0; }
+    }
+    return rc;
+}
+
+}  // extern "C"

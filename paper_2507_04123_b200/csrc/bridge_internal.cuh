@@ -1,0 +1,146 @@
+// Internal declarations shared by the bridge's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "emc2_bridge.h"
+
+namespace emc2 {
+
+constexpr int kTile = 256;           // points per CTA tile in the per-point kernels
+constexpr int kThreads = 256;
+constexpr int kChunkBytes = 32;      // one L2 sector: 256 bitmap cells or 8 table cells
+constexpr int kMaxTableCells = 1 << 26;  // direct count table up to 64 Mi cells per batch
+
+// Kernel kinds, for the launch counters and the optional event timing.
+enum KernelKind {
+    K_VOX_MARK = 0,
+    K_VOX_REDUCE,
+    K_VOX_BLOCKSCAN,
+    K_VOX_EMIT,
+    K_VOX_ACCUM,
+    K_VOX_OVERFLOW,
+    K_VOX_FINALIZE,
+    K_VOX_CLEAN,
+    K_BEV_ZERO,
+    K_PROJECT_GATHER,
+    K_ROUTE_HIST,
+    K_ROUTE_SCAN,
+    K_DISPATCH_SCATTER,
+    K_KINDS
+};
+
+enum ScaleMode { MODE_BITMAP = 0, MODE_TABLE = 1 };
+
+// Per-scale grid description and scratch pointers, passed to kernels by value.
+struct ScaleDev {
+    float mn[3];
+    float vs[3];
+    int dims[3];            // Gx, Gy, Gz
+    int cap;                // 0 = none
+    int mode;               // ScaleMode
+    uint32_t cells;         // cells per frame
+    uint32_t nchunks;       // 32-byte chunks of `store` for the largest batch
+    uint32_t nsumwords;     // 32-bit words of `summary`
+    uint32_t* store;        // bitmap words, or int32 counts
+    uint32_t* summary;      // one bit per chunk: chunk has an occupied cell
+    uint32_t* chunk_prefix; // voxels before the chunk (valid for flagged chunks)
+    double* sums;           // [max voxels, C]
+    int* blk_sums;          // [scan blocks, 3]
+    int* blk_offs;          // [scan blocks, 3]
+    int* ovf_off;           // per voxel: start in ovf_list, -1 = not overflowing (capped scales)
+    int* ovf_cursor;        // per voxel: points appended so far
+    int* ovf_vox;           // list of overflowing voxels
+    int* ovf_list;          // global point indices of overflowing voxels
+    int* totals;            // [0] voxels, [1] overflowing voxels, [2] overflowing points
+    int scan_blocks;
+};
+
+struct ProfRec {
+    int kind;
+    cudaEvent_t a, b;
+};
+
+}  // namespace emc2
+
+struct emc2_bridge {
+    emc2_config_t cfg;
+    emc2::ScaleDev scale[2];
+    float thr2[EMC2_MAX_THRESHOLDS];
+    void* slab = nullptr;
+    size_t slab_bytes = 0;
+    int* d_status = nullptr;       // sticky device status word
+    int* d_tile_counts = nullptr;  // [B, tiles per frame, E]
+    int* d_tile_base = nullptr;    // same shape, exclusive bases
+    int max_tiles = 0;
+    int last_cuda_error = 0;
+    bool profiling = false;
+    int64_t launches[emc2::K_KINDS] = {0};
+    double ms[emc2::K_KINDS] = {0};
+    std::vector<emc2::ProfRec> recs;
+    std::vector<cudaEvent_t> event_pool;
+};
+
+namespace emc2 {
+
+// Brackets a launch with events when profiling; always counts it.
+struct LaunchScope {
+    emc2_bridge* h;
+    int kind;
+    cudaStream_t st;
+    cudaEvent_t a = nullptr, b = nullptr;
+    LaunchScope(emc2_bridge* h_, int kind_, cudaStream_t st_);
+    ~LaunchScope();
+};
+
+int check_cuda(emc2_bridge* h, cudaError_t e);
+
+int launch_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* const d_coords[2],
+                    int32_t* const d_counts[2], float* const d_mean[2], int32_t* const d_point_voxel[2],
+                    const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st);
+int launch_project_gather(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj,
+                          const float* d_feat, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
+                          float* d_gathered, cudaStream_t st);
+int launch_route_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const uint8_t* d_vis_mask,
+                          const float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
+                          float* d_points_out, float* d_feat_out, cudaStream_t st);
+
+// ---------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+
+// Loads `nfloats` consecutive floats starting at a 16-byte aligned address into shared
+// memory with 128-bit loads (scalar loads for a ragged tail).
+__device__ __forceinline__ void load_tile_f32(const float* __restrict__ src, int nfloats, float* smem) {
+    const int nvec = nfloats >> 2;
+    const float4* s4 = reinterpret_cast<const float4*>(src);
+    float4* d4 = reinterpret_cast<float4*>(smem);
+    for (int i = threadIdx.x; i < nvec; i += blockDim.x) d4[i] = __ldg(s4 + i);
+    for (int i = (nvec << 2) + threadIdx.x; i < nfloats; i += blockDim.x) smem[i] = __ldg(src + i);
+}
+
+// Cell index along one axis: one fp32 subtract, one IEEE fp32 divide, floor.  -1 if outside.
+__device__ __forceinline__ int axis_cell(float p, float mn, float vs, int dim) {
+    float q = __fdiv_rn(__fsub_rn(p, mn), vs);
+    float f = floorf(q);
+    // NaN fails both comparisons; +-inf fails one of them.
+    if (!(f >= 0.0f) || !(f < (float)dim)) return -1;
+    return (int)f;
+}
+
+// Cell id of a point inside the whole batch, or 0xFFFFFFFF if outside the grid.
+__device__ __forceinline__ uint32_t cell_of(const ScaleDev& g, float x, float y, float z, int b) {
+    int ix = axis_cell(x, g.mn[0], g.vs[0], g.dims[0]);
+    int iy = axis_cell(y, g.mn[1], g.vs[1], g.dims[1]);
+    int iz = axis_cell(z, g.mn[2], g.vs[2], g.dims[2]);
+    if ((ix | iy | iz) < 0) return 0xFFFFFFFFu;
+    return (((uint32_t)b * g.dims[2] + iz) * g.dims[1] + iy) * g.dims[0] + ix;
+}
+
+__device__ __forceinline__ int warp_sum(int v) { return __reduce_add_sync(0xFFFFFFFFu, v); }
+
+#endif  // __CUDACC__
+
+}  // namespace emc2

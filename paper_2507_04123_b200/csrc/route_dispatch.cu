@@ -1,0 +1,210 @@
+// Stages 3 and 4 of the bridge: per-point expert id from distance and visibility buckets
+// (Scenario-Adaptive Dispatcher, Sec. 3.2: near is < D, far is >= D), then a stable
+// counting-sort partition of point rows and feature rows into per-expert segments whose
+// offsets are exclusive prefix sums (Sec. 3.6).
+//
+// Three launches: (1) expert ids plus one histogram per 256-point tile, counted with warp
+// ballots; (2) a small scan that turns tile histograms into per-frame expert offsets and
+// per-tile bases; (3) one CTA per tile ranks its points inside the tile with ballots and
+// popcounts, writes the permutation and moves the 16/20-byte point rows and the 256/320-byte
+// feature rows with coalesced 128-bit accesses.
+#include "bridge_internal.cuh"
+
+namespace emc2 {
+namespace {
+
+struct RouteArgs {
+    const float* pts;
+    const uint8_t* vis;
+    uint8_t* expert;
+    int* tile_counts;     // [B, tiles, E]
+    int N, tiles, E, T;
+    float thr2[EMC2_MAX_THRESHOLDS];
+    uint8_t lut[16];
+};
+
+// grid = (tiles per frame, B); tiles never straddle frames.
+template <int C>
+__global__ void __launch_bounds__(kThreads) route_hist_kernel(RouteArgs a) {
+    __shared__ __align__(16) float sp[kTile * C];
+    __shared__ int hist[EMC2_MAX_EXPERTS];
+    const int b = blockIdx.y, tile = blockIdx.x, t = threadIdx.x;
+    const int i0 = tile * kTile;
+    const int npts = min(kTile, a.N - i0);
+    const size_t g0 = (size_t)b * a.N + i0;
+    // Frames start on a 16-byte boundary only if N*C is a multiple of 4 floats.
+    const float* src = a.pts + g0 * C;
+    if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+        load_tile_f32(src, npts * C, sp);
+    } else {
+        for (int i = t; i < npts * C; i += kThreads) sp[i] = __ldg(src + i);
+    }
+    if (t < EMC2_MAX_EXPERTS) hist[t] = 0;
+    __syncthreads();
+    int e = -1;
+    if (t < npts) {
+        const float x = sp[t * C], y = sp[t * C + 1];
+        const float r2 = __fmaf_rn(x, x, __fmul_rn(y, y));
+        int bucket = 0;
+        for (int k = 0; k < a.T; ++k) bucket += (r2 >= a.thr2[k]) ? 1 : 0;
+        e = a.lut[(a.vis[g0 + t] != 0 ? 8 : 0) + bucket];
+        a.expert[g0 + t] = (uint8_t)e;
+    }
+    const int lane = t & 31;
+    for (int k = 0; k < a.E; ++k) {
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
+        if (lane == 0 && m) atomicAdd(&hist[k], __popc(m));
+    }
+    __syncthreads();
+    if (t < a.E) a.tile_counts[((size_t)b * a.tiles + tile) * a.E + t] = hist[t];
+}
+
+// One CTA per frame.  For each expert: exclusive scan of its tile counts.  Then offsets.
+__global__ void __launch_bounds__(kThreads)
+route_scan_kernel(const int* __restrict__ tile_counts, int* __restrict__ tile_base, int32_t* offsets,
+                  int tiles, int E, int N) {
+    __shared__ int wsum[kThreads / 32];
+    __shared__ int carry;
+    __shared__ int etot[EMC2_MAX_EXPERTS + 1];
+    const int b = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int* cnt = tile_counts + (size_t)b * tiles * E;
+    int* base = tile_base + (size_t)b * tiles * E;
+    for (int e = 0; e < E; ++e) {
+        if (t == 0) carry = 0;
+        __syncthreads();
+        for (int s = 0; s < tiles; s += kThreads) {
+            const int i = s + t;
+            const int v = i < tiles ? cnt[(size_t)i * E + e] : 0;
+            int x = v;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
+                if (lane >= d) x += y;
+            }
+            if (lane == 31) wsum[warp] = x;
+            __syncthreads();
+            int wb = 0;
+            for (int w = 0; w < warp; ++w) wb += wsum[w];
+            const int c0 = carry;
+            if (i < tiles) base[(size_t)i * E + e] = c0 + wb + x - v;   // still relative to the expert
+            __syncthreads();
+            if (t == kThreads - 1) carry = c0 + wb + x;
+            __syncthreads();
+        }
+        if (t == 0) etot[e] = carry;
+        __syncthreads();
+    }
+    if (t == 0) {
+        int run = 0;
+        for (int e = 0; e < E; ++e) { const int c = etot[e]; etot[e] = run; run += c; }
+        etot[E] = run;
+    }
+    __syncthreads();
+    if (t <= E) offsets[(size_t)b * (E + 1) + t] = etot[t];
+    for (int i = t; i < tiles * E; i += kThreads) base[i] += etot[i % E];
+}
+
+struct ScatterArgs {
+    const float* pts;
+    const float4* feat;
+    const uint8_t* expert;
+    const int* tile_base;
+    int32_t* perm;
+    float* pts_out;
+    float4* feat_out;
+    int N, tiles, E, cf4;
+};
+
+template <int C, int CF4>
+__global__ void __launch_bounds__(kThreads) dispatch_scatter_kernel(ScatterArgs a) {
+    __shared__ int sdest[kTile];
+    __shared__ int wcnt[kThreads / 32][EMC2_MAX_EXPERTS];
+    const int b = blockIdx.y, tile = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int i0 = tile * kTile;
+    const int npts = min(kTile, a.N - i0);
+    const size_t f0 = (size_t)b * a.N;        // first row of the frame
+    const size_t g0 = f0 + i0;
+    const int cf4 = CF4 > 0 ? CF4 : a.cf4;
+
+    const int e = t < npts ? (int)a.expert[g0 + t] : -1;
+    int rank = 0;
+    for (int k = 0; k < a.E; ++k) {
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
+        if (e == k) rank = __popc(m & ((1u << lane) - 1u));
+        if (lane == 0) wcnt[warp][k] = __popc(m);
+    }
+    __syncthreads();
+    if (t < npts) {
+        int before = 0;
+        for (int w = 0; w < warp; ++w) before += wcnt[w][e];
+        const int d = a.tile_base[((size_t)b * a.tiles + tile) * a.E + e] + before + rank;
+        sdest[t] = d;
+        a.perm[f0 + d] = i0 + t;
+    }
+    __syncthreads();
+
+    // Point rows: the tile's source floats are contiguous.
+    const float* psrc = a.pts + g0 * C;
+    float* pdst = a.pts_out + f0 * C;
+    for (int i = t; i < npts * C; i += kThreads) {
+        const int r = i / C, c = i - r * C;
+        pdst[(size_t)sdest[r] * C + c] = __ldg(psrc + i);
+    }
+    // Feature rows: read the tile as a flat float4 stream, write whole rows to their slots.
+    const float4* fsrc = a.feat + g0 * cf4;
+    float4* fdst = a.feat_out + f0 * cf4;
+    const int items = npts * cf4;
+#pragma unroll 5
+    for (int i = t; i < items; i += kThreads) {
+        const int r = i / cf4, c = i - r * cf4;
+        const float4 v = __ldcs(fsrc + i);
+        __stcs(fdst + (size_t)sdest[r] * cf4 + c, v);
+    }
+}
+
+template <int C>
+void launch_scatter(emc2_bridge* h, const ScatterArgs& a, dim3 grid, cudaStream_t st) {
+    LaunchScope ls(h, K_DISPATCH_SCATTER, st);
+    switch (a.cf4) {
+        case 16: dispatch_scatter_kernel<C, 16><<<grid, kThreads, 0, st>>>(a); break;
+        case 20: dispatch_scatter_kernel<C, 20><<<grid, kThreads, 0, st>>>(a); break;
+        default: dispatch_scatter_kernel<C, 0><<<grid, kThreads, 0, st>>>(a); break;
+    }
+}
+
+}  // namespace
+
+int launch_route_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const uint8_t* d_vis_mask,
+                          const float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
+                          float* d_points_out, float* d_feat_out, cudaStream_t st) {
+    const emc2_config_t& c = h->cfg;
+    const int tiles = (N + kTile - 1) / kTile;
+    const int E = c.num_experts;
+    if (B == 0) return EMC2_OK;
+    const dim3 grid(tiles > 0 ? tiles : 1, B);
+    RouteArgs ra;
+    ra.pts = d_points; ra.vis = d_vis_mask; ra.expert = d_expert; ra.tile_counts = h->d_tile_counts;
+    ra.N = N; ra.tiles = tiles; ra.E = E; ra.T = c.num_thresholds;
+    for (int k = 0; k < EMC2_MAX_THRESHOLDS; ++k) ra.thr2[k] = h->thr2[k];
+    for (int k = 0; k < 16; ++k) ra.lut[k] = c.lut[k >> 3][k & 7];
+    if (tiles > 0) {
+        LaunchScope ls(h, K_ROUTE_HIST, st);
+        if (c.point_floats == 4) route_hist_kernel<4><<<grid, kThreads, 0, st>>>(ra);
+        else route_hist_kernel<5><<<grid, kThreads, 0, st>>>(ra);
+    }
+    {
+        LaunchScope ls(h, K_ROUTE_SCAN, st);
+        route_scan_kernel<<<B, kThreads, 0, st>>>(h->d_tile_counts, h->d_tile_base, d_offsets, tiles, E, N);
+    }
+    if (tiles > 0) {
+        ScatterArgs sa;
+        sa.pts = d_points; sa.feat = reinterpret_cast<const float4*>(d_gathered); sa.expert = d_expert;
+        sa.tile_base = h->d_tile_base; sa.perm = d_perm; sa.pts_out = d_points_out;
+        sa.feat_out = reinterpret_cast<float4*>(d_feat_out);
+        sa.N = N; sa.tiles = tiles; sa.E = E; sa.cf4 = c.feat_c / 4;
+        if (c.point_floats == 4) launch_scatter<4>(h, sa, grid, st); else launch_scatter<5>(h, sa, grid, st);
+    }
+    return check_cuda(h, cudaGetLastError());
+}
+
+}  // namespace emc2

@@ -1,0 +1,136 @@
+"""CUDA library vs CPU oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import emc2_gen as gen
+from parity import compare_bridge, np_, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def b200():
+    import paper_2507_04123_b200 as pkg
+    from paper_2507_04123_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+    return pkg
+
+
+def run_case(pkg, oracle, w, batch=None, repeat=1):
+    batch = batch if batch is not None else gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    br = pkg.Bridge(pkg.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = None
+    for _ in range(repeat):                      # a second call must see clean scratch
+        bufs = br.run(d["points"], d["proj"], d["feat"], bufs)
+    br.status()
+    compare_bridge(w, ref, bufs)
+    br.close()
+    return ref, bufs
+
+
+@pytest.mark.parametrize("cid", [0, 1, 2, 3])
+def test_benchmark_configs_match_the_oracle(b200, oracle, cid):
+    run_case(b200, oracle, gen.workload(cid), repeat=2)
+
+
+@pytest.mark.parametrize("B,N", [(1, 1), (1, 255), (2, 257), (3, 1000), (2, 4099), (5, 777)])
+def test_ragged_shapes(b200, oracle, B, N):
+    for base in (gen.KITTI, gen.NUSCENES):
+        run_case(b200, oracle, base.with_shape(B, N), repeat=2)
+
+
+def test_sweep_cell_with_six_cameras(b200, oracle):
+    run_case(b200, oracle, gen.SWEEP.with_shape(2, 65536))
+
+
+def test_degenerate_frames(b200, oracle):
+    w = gen.NUSCENES.with_shape(2, 3000)
+    batch = gen.make_batch(w)
+    p = batch["points"]
+    p[0, :, :3] = (1.0, 2.0, 0.5)                # every point of frame 0 in one voxel (cap binds)
+    p[1, :1000, 0] = 500.0                       # outside both grids, beyond every threshold
+    p[1, 1000:1100, 1] = np.nan                  # non-finite coordinates
+    p[1, 1100:1200, 2] = np.inf
+    run_case(b200, oracle, w, batch)
+    q = gen.make_batch(w)
+    q["points"][..., :3] = 1e6                   # nothing in range, nothing visible: zero voxels
+    ref, bufs = run_case(b200, oracle, w, q)
+    assert ref["vox0"]["num_voxels"] == 0 and ref["vox1"]["num_voxels"] == 0
+    assert not np_(bufs["vox"]["bev"]).any()
+
+
+def test_single_expert_and_empty_expert(b200, oracle):
+    from dataclasses import replace
+    w = replace(gen.KITTI.with_shape(2, 5000), lut=((2, 2, 2, 0, 0, 0, 0, 0), (2, 2, 2, 0, 0, 0, 0, 0)))
+    ref, _ = run_case(b200, oracle, w)
+    assert (ref["offsets"][:, 2] == 0).all() and (ref["offsets"][:, 3] == w.N).all()
+
+
+def test_empty_inputs(b200):
+    w = gen.KITTI.with_shape(2, 64)
+    br = b200.Bridge(b200.config_from_workload(w))
+    for B, N in ((0, 64), (2, 0)):
+        pts = torch.zeros((B, N, 4), device="cuda")
+        proj = torch.zeros((B, 1, 3, 4), device="cuda")
+        feat = torch.zeros((B, 1, w.feat_h, w.feat_w, w.feat_c), device="cuda")
+        bufs = br.run(pts, proj, feat)
+        br.status()
+        assert np_(bufs["vox"]["num_voxels"]).tolist() == [0, 0]
+        if B:
+            assert (np_(bufs["rd"]["offsets"]) == 0).all()
+    br.close()
+
+
+def test_capacity_overflow_is_reported_and_handle_recovers(b200, oracle):
+    w = gen.TINY
+    batch = gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    cap = [1000, 500]
+    out = br.voxelize(d["points"], capacity=cap)
+    assert br.status(raise_on_error=False) == b200.bridge.EMC2_ERR_CAPACITY
+    nv = np_(out["num_voxels"])
+    assert nv[0] == ref["vox0"]["num_voxels"] and nv[1] == ref["vox1"]["num_voxels"]   # true counts
+    for s in range(2):
+        assert np.array_equal(np_(out["coords"][s])[:cap[s]], ref[f"vox{s}"]["coords"][:cap[s]])
+        assert np.array_equal(np_(out["counts"][s])[:cap[s]], ref[f"vox{s}"]["counts"][:cap[s]])
+    assert br.status(raise_on_error=False) == 0                   # sticky word was cleared
+    bufs = br.run(d["points"], d["proj"], d["feat"])              # scratch is clean again
+    br.status()
+    compare_bridge(w, ref, bufs)
+    br.close()
+
+
+def test_integer_outputs_are_deterministic(b200):
+    w = gen.DENSE
+    d = to_dev(gen.make_batch(w))
+    br = b200.Bridge(b200.config_from_workload(w))
+    runs = []
+    for _ in range(2):
+        bufs = br.run(d["points"], d["proj"], d["feat"])
+        br.status()
+        nv = np_(bufs["vox"]["num_voxels"])
+        runs.append([np_(bufs["vox"]["coords"][1])[:nv[1]].copy(), np_(bufs["vox"]["counts"][1])[:nv[1]].copy(),
+                     np_(bufs["vox"]["point_voxel"][1]).copy(), np_(bufs["rd"]["perm"]).copy(),
+                     np_(bufs["pg"]["vis_mask"]).copy()])
+    for a, b in zip(*runs):
+        assert np.array_equal(a, b)
+    br.close()
+
+
+def test_host_detected_errors(b200):
+    w = gen.TINY
+    br = b200.Bridge(b200.config_from_workload(w))
+    pts = torch.zeros((1, w.N + 1, 4), device="cuda")
+    with pytest.raises(b200.Emc2Error) as e:
+        br.voxelize(pts)
+    assert e.value.status == b200.bridge.EMC2_ERR_INVALID_ARG
+    pts = torch.zeros((1, 65, 4), device="cuda").view(-1)[1:257].view(1, 64, 4)   # misaligned view
+    with pytest.raises((b200.Emc2Error, ValueError)):
+        br.voxelize(pts)
+    br.close()
