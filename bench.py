@@ -1,0 +1,394 @@
+#!/usr/bin/env python
+"""Benchmark of the EMC2 data bridge + dispatch on B200.
+
+A step is one pass of the whole hot path (emc2_voxelize, emc2_project_gather,
+emc2_route_dispatch back to back on one stream) over one batch of synthetic
+frames.  Default workload: the nuScenes-shaped 6-camera batch (4 frames of
+300,000 points), the configuration the roofline target is quoted on.
+
+    python bench.py --gpus 1 --steps 20 --warmup 5
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   (replicas, weak scaling)
+    python bench.py --impl reference      (the CPU oracle on the host cores)
+    python bench.py --config 1            (another workload; --sweep for the throughput grid)
+
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import emc2_gen as gen
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126e6
+
+
+# ----------------------------------------------------------------------------- helpers
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(w, B, N, m0, m1, texels):
+    """Bytes the staged ABI must move: every input read once per call, every output written once."""
+    pb, fb, C = 4 * w.C, 4 * w.feat_c, w.C
+    g1 = w.grids[1]
+    vox = B * N * pb + B * N * 8 + (m0 + m1) * (16 + 4 + pb) + B * C * g1.dims[1] * g1.dims[0] * 4
+    pg = B * N * pb + B * w.K * 48 + fb * texels + B * N * (12 + 1 + 1 + fb)
+    rd = B * N * (pb + 1 + fb) + B * N * (1 + 4 + pb + fb) + B * (w.num_experts + 1) * 4
+    return {"voxelize": vox, "project_gather": pg, "route_dispatch": rd, "total": vox + pg + rd}
+
+
+def kernel_bytes(w, B, N, texels):
+    """Algorithmic bytes of the two row-moving kernels, per launch."""
+    pb, fb = 4 * w.C, 4 * w.feat_c
+    return {"project_gather": B * N * pb + B * w.K * 48 + fb * texels + B * N * (12 + 1 + 1 + fb),
+            "dispatch_scatter": B * N * (1 + pb + fb) + B * N * (4 + pb + fb)}
+
+
+def distinct_texels(w, pg):
+    """Distinct feature texels the gather touches, from the library's own uvd/cam outputs."""
+    uvd, cam = pg["uvd"], pg["cam"]
+    B, N = cam.shape
+    vis = cam >= 0
+    fx = (uvd[..., 0] / w.feat_stride)[vis]
+    fy = (uvd[..., 1] / w.feat_stride)[vis]
+    b = torch.arange(B, device=cam.device)[:, None].expand(B, N)[vis].long()
+    k = cam[vis].long()
+    x0, y0 = fx.floor().long(), fy.floor().long()
+    keys = []
+    for dy in (0, 1):
+        for dx in (0, 1):
+            x = (x0 + dx).clamp(max=w.feat_w - 1)
+            y = (y0 + dy).clamp(max=w.feat_h - 1)
+            keys.append(((b * w.K + k) * w.feat_h + y) * w.feat_w + x)
+    return int(torch.unique(torch.cat(keys)).numel())
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                   "samples": len(sm)}
+        return out
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ----------------------------------------------------------------------------- reference arm (CPU oracle)
+def oracle_rate(w, target_s=12.0, max_steps=None):
+    """Times the oracle, as it stands, single-threaded on the host, on one-frame samples."""
+    import oracle
+    oracle.build()
+    w1 = w.with_shape(1, w.N)
+    batch = gen.make_batch(w1, frames=[0])
+    oracle.bridge(w1, batch)                               # warm the caches / page in
+    times = []
+    t_all = time.perf_counter()
+    while True:
+        t0 = time.perf_counter()
+        oracle.bridge(w1, batch)
+        times.append(time.perf_counter() - t0)
+        if max_steps is not None and len(times) >= max_steps:
+            break
+        if max_steps is None and time.perf_counter() - t_all > target_s and len(times) >= 3:
+            break
+    return times
+
+
+def run_reference(args, w):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    steps = args.steps
+    times = oracle_rate(w, max_steps=args.warmup + steps)[args.warmup:]
+    per = float(np.median(times))
+    fps = 1.0 / per
+    line = {
+        "impl": "reference", "metric": "bridge frames/s", "value": fps, "unit": "frames/s",
+        "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": per * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "points_per_frame": w.N, "cameras": w.K, "feat_c": w.feat_c,
+                   "step": "one frame through the single-threaded C++ oracle"},
+        "mpoints_per_s": fps * w.N / 1e6,
+        "cpu_baseline": {"value": fps, "unit": "frames/s", "cores": 1, "kind": "oracle",
+                         "sample": f"1 frame of {w.N} points per step, median of {steps} steps",
+                         "host_cores_available": os.cpu_count()},
+        "e2e": {"value": fps, "unit": "frames/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- our arm
+def time_steps(fn, steps, stream_sync, barrier):
+    barrier()
+    stream_sync()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        fn()
+    b.record()
+    stream_sync()
+    barrier()
+    return a.elapsed_time(b) / 1e3
+
+
+def run_ours(args, w):
+    import paper_2507_04123_b200 as pkg
+    from paper_2507_04123_b200 import build as cuda_build
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the bridge has no CPU path")
+    if not os.path.exists(pkg.LIB_PATH):
+        cuda_build.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if use_dist:
+            dist.barrier()
+
+    def max_over_ranks(x):
+        if not use_dist:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    B, N = w.B, w.N
+    frames = list(range(rank * B, rank * B + B))           # every rank owns its own frames
+    batch = gen.make_batch(w, frames=frames, feature_frames=args.feature_frames)
+    host = {k: torch.from_numpy(v).pin_memory() for k, v in batch.items()}
+    d = {k: v.to(dev, non_blocking=True) for k, v in host.items()}
+    br = pkg.Bridge(pkg.config_from_workload(w, device=local_rank))
+    sync = lambda: torch.cuda.synchronize(dev)
+
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    br.status()
+    nv = bufs["vox"]["num_voxels"].cpu().numpy()
+    texels = distinct_texels(w, bufs["pg"])
+    abytes = algorithmic_bytes(w, B, N, int(nv[0]), int(nv[1]), texels)
+
+    def step():
+        br.run(d["points"], d["proj"], d["feat"], bufs)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sync()
+    br.profile_read(reset=True)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        time.sleep(0.3)
+    secs = max_over_ranks(time_steps(step, args.steps, sync, barrier))
+    launches = sum(n for n, _ in br.profile_read(reset=True).values())
+    br.status()
+
+    # End to end: pinned host inputs copied in every step, small results read back every step.
+    e2e_in = {k: torch.empty_like(v) for k, v in d.items()}
+    off_host = torch.empty((B, w.num_experts + 1), dtype=torch.int32).pin_memory()
+    nv_host = torch.empty((2,), dtype=torch.int32).pin_memory()
+    e2e_bufs = bufs
+
+    def e2e_step():
+        for k in ("points", "proj", "feat"):
+            e2e_in[k].copy_(host[k], non_blocking=True)
+        br.run(e2e_in["points"], e2e_in["proj"], e2e_in["feat"], e2e_bufs)
+        off_host.copy_(e2e_bufs["rd"]["offsets"], non_blocking=True)
+        nv_host.copy_(e2e_bufs["vox"]["num_voxels"], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for _ in range(2):
+        e2e_step()
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_secs = max_over_ranks(time_steps(e2e_step, e2e_steps, sync, barrier))
+    clocks = sampler.stop() if sampler else None
+    h2d = sum(int(host[k].numel() * host[k].element_size()) for k in ("points", "proj", "feat"))
+    d2h = int(off_host.numel() * 4 + nv_host.numel() * 4)
+
+    # Per-kernel device time (events around every launch), outside the timed region.
+    br.profile_read(reset=True)
+    br.profile_enable(True)
+    prof_steps = max(3, min(args.steps, 10))
+    for _ in range(prof_steps):
+        step()
+    sync()
+    prof = br.profile_read(reset=True)
+    br.profile_enable(False)
+    kb = kernel_bytes(w, B, N, texels)
+    per_kernel = {k: {"launches": n, "ms_per_launch": (ms / n if n else 0.0)} for k, (n, ms) in prof.items() if n}
+    dom = max((k for k in per_kernel if k in kb), key=lambda k: per_kernel[k]["ms_per_launch"] * per_kernel[k]["launches"])
+    peak, peak_kind = measured_peak()
+    dom_ms = per_kernel[dom]["ms_per_launch"]
+    achieved = kb[dom] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
+    traffic = None
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            t = json.load(f).get(dom)
+            if t:
+                traffic = t["dram_bytes_per_point"] * B * N
+    except Exception:
+        pass
+
+    if rank != 0:
+        if use_dist:
+            dist.destroy_process_group()
+        return
+
+    ms_step = secs / args.steps * 1e3
+    fps = world * B * args.steps / secs
+    total_gbs = abytes["total"] / (ms_step * 1e-3) / 1e9
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        times = oracle_rate(w, target_s=12.0)
+        per = float(np.median(times))
+        cpu = {"value": 1.0 / per, "unit": "frames/s", "cores": 1, "kind": "oracle",
+               "sample": f"{len(times)} single-frame passes ({w.N} points each), median; host has {os.cpu_count()} cores",
+               "ms_per_frame": per * 1e3}
+    line = {
+        "metric": "bridge frames/s", "value": fps, "unit": "frames/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "frames_per_step_per_gpu": B, "points_per_frame": N, "point_floats": w.C,
+                   "cameras": w.K, "feat_c": w.feat_c, "parallelism": f"replicas x{world} (frames sharded, no collective)",
+                   "l2": "inputs and outputs of a step exceed L2 (no flush)" if abytes["total"] > 2 * L2_BYTES
+                         else "working set fits in L2 (latency-bound workload, no flush)"},
+        "mpoints_per_s": fps * N / 1e6,
+        "bridge_algorithmic_bytes_per_step": abytes,
+        "bridge_gbs": total_gbs, "bridge_frac_of_8tbs": total_gbs / NOMINAL_HBM_GBS,
+        f"bridge_frac_of_{peak_kind}_copy": total_gbs / peak,
+        "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_source": peak_kind,
+                     "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+                     "algorithmic_bytes_per_launch": kb[dom], "ms_per_launch": dom_ms},
+        "kernels": per_kernel,
+        "e2e": {"value": world * B * e2e_steps / e2e_secs, "unit": "frames/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_secs / e2e_steps * 1e3},
+        "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
+        "unique_voxels": [int(nv[0]), int(nv[1])], "distinct_texels": texels,
+    }
+    print(json.dumps(line), flush=True)
+    if use_dist:
+        dist.destroy_process_group()
+
+
+def run_sweep(args):
+    """Throughput grid: points per frame x batch through the six-camera projection (1 GPU)."""
+    import paper_2507_04123_b200 as pkg
+    dev = torch.device("cuda", 0)
+    rows = []
+    for N in gen.SWEEP_POINTS:
+        for B in gen.SWEEP_BATCH:
+            w = gen.SWEEP.with_shape(B, N)
+            batch = gen.make_batch(w, feature_frames=1)
+            d = {k: torch.from_numpy(v).to(dev) for k, v in batch.items()}
+            br = pkg.Bridge(pkg.config_from_workload(w))
+            bufs = br.run(d["points"], d["proj"], d["feat"])
+            br.status()
+            nv = bufs["vox"]["num_voxels"].cpu().numpy()
+            ab = algorithmic_bytes(w, B, N, int(nv[0]), int(nv[1]), distinct_texels(w, bufs["pg"]))
+            step = lambda: br.run(d["points"], d["proj"], d["feat"], bufs)
+            for _ in range(5):
+                step()
+            steps = 20 if B * N < 4_000_000 else 8
+            secs = time_steps(step, steps, lambda: torch.cuda.synchronize(dev), lambda: None)
+            ms = secs / steps * 1e3
+            gbs = ab["total"] / (ms * 1e-3) / 1e9
+            rows.append({"N": N, "B": B, "ms_per_step": ms, "frames_per_s": B / (ms * 1e-3),
+                         "mpoints_per_s": B * N / (ms * 1e-3) / 1e6, "gbs": gbs, "frac_of_8tbs": gbs / NOMINAL_HBM_GBS,
+                         "bytes_per_point": ab["total"] / (B * N)})
+            br.close()
+            del d, bufs
+            torch.cuda.empty_cache()
+            print(json.dumps(rows[-1]), flush=True)
+    return rows
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload id 0..3 (default: nuScenes-shaped)")
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--points", type=int, default=None)
+    ap.add_argument("--feature-frames", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true")
+    args = ap.parse_args()
+    w = gen.workload(args.config)
+    if args.batch or args.points:
+        w = w.with_shape(args.batch or w.B, args.points or w.N)
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

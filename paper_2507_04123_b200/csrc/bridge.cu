@@ -136,7 +136,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
 
     // Plan the slab: everything the stage calls need, allocated once.
     SlabPlan plan;
-    size_t o_store[2], o_summary[2], o_prefix[2], o_sums[2], o_bs[2], o_bo[2], o_ovf[2][4], o_tot[2];
+    size_t o_store[2], o_summary[2], o_prefix[2], o_covf[2], o_sums[2], o_bs[2], o_bo[2], o_ovf[2][4], o_tot[2];
     for (int s = 0; s < 2; ++s) {
         ScaleDev& d = h->scale[s];
         const emc2_grid_t& g = c.grid[s];
@@ -148,14 +148,17 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         const uint64_t per_chunk = d.mode == MODE_BITMAP ? 256 : 8;
         d.nchunks = (uint32_t)((total_cells + per_chunk - 1) / per_chunk);
         d.nsumwords = (d.nchunks + 31) / 32;
-        d.scan_blocks = (int)((d.nsumwords + kThreads - 1) / kThreads);
+        d.scan_blocks = (int)((d.nchunks + kThreads - 1) / kThreads);
+        d.max_ovf = d.cap > 0 ? (uint32_t)(maxpts / ((size_t)d.cap + 1) + 1) : 0;
         o_store[s] = plan.take((size_t)d.nsumwords * 32 * kChunkBytes);
         o_summary[s] = plan.take((size_t)d.nsumwords * 4);
         o_prefix[s] = plan.take((size_t)d.nsumwords * 32 * 4);
+        o_covf[s] = d.cap > 0 ? plan.take((size_t)d.nsumwords * 32 * 4) : 0;
         o_sums[s] = plan.take(maxpts * c.point_floats * sizeof(double));
         o_bs[s] = plan.take((size_t)d.scan_blocks * 3 * sizeof(int));
         o_bo[s] = plan.take((size_t)d.scan_blocks * 3 * sizeof(int));
-        for (int k = 0; k < 4; ++k) o_ovf[s][k] = d.cap > 0 ? plan.take(maxpts * sizeof(int)) : 0;
+        for (int k = 0; k < 3; ++k) o_ovf[s][k] = d.cap > 0 ? plan.take((size_t)d.max_ovf * sizeof(int)) : 0;
+        o_ovf[s][3] = d.cap > 0 ? plan.take(maxpts * sizeof(int)) : 0;
         o_tot[s] = plan.take(4 * sizeof(int));
     }
     h->max_tiles = (c.max_points + kTile - 1) / kTile;
@@ -176,6 +179,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         d.store = reinterpret_cast<uint32_t*>(base + o_store[s]);
         d.summary = reinterpret_cast<uint32_t*>(base + o_summary[s]);
         d.chunk_prefix = reinterpret_cast<uint32_t*>(base + o_prefix[s]);
+        d.chunk_ovf = d.cap > 0 ? reinterpret_cast<uint32_t*>(base + o_covf[s]) : nullptr;
         d.sums = reinterpret_cast<double*>(base + o_sums[s]);
         d.blk_sums = reinterpret_cast<int*>(base + o_bs[s]);
         d.blk_offs = reinterpret_cast<int*>(base + o_bo[s]);
@@ -204,7 +208,9 @@ int emc2_voxelize(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points,
                   float* d_bev, void* cuda_stream) {
     int rc = check_call(h, B, N);
     if (rc != EMC2_OK) return rc;
-    if (!d_points || !d_coords || !d_counts || !d_mean || !capacity || !d_num_voxels) return EMC2_ERR_INVALID_ARG;
+    const bool empty = B == 0 || N == 0;   // zero-sized buffers may be null
+    if ((!d_points && !empty) || !d_coords || !d_counts || !d_mean || !capacity || !d_num_voxels)
+        return EMC2_ERR_INVALID_ARG;
     if (!aligned16(d_points) || (d_bev && !aligned16(d_bev))) return EMC2_ERR_INVALID_ARG;
     for (int s = 0; s < 2; ++s) {
         if (!d_coords[s] || !d_counts[s] || !d_mean[s] || capacity[s] < 0) return EMC2_ERR_INVALID_ARG;
@@ -221,6 +227,7 @@ int emc2_project_gather(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_p
                         float* d_gathered, void* cuda_stream) {
     int rc = check_call(h, B, N);
     if (rc != EMC2_OK) return rc;
+    if (B == 0 || N == 0) return EMC2_OK;   // nothing to write
     if (!d_points || !d_proj || !d_feat || !d_uvd || !d_vis_mask || !d_cam || !d_gathered)
         return EMC2_ERR_INVALID_ARG;
     if (!aligned16(d_points) || !aligned16(d_feat) || !aligned16(d_gathered)) return EMC2_ERR_INVALID_ARG;
@@ -236,11 +243,13 @@ int emc2_route_dispatch(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_p
                         void* cuda_stream) {
     int rc = check_call(h, B, N);
     if (rc != EMC2_OK) return rc;
-    if (!d_points || !d_vis_mask || !d_gathered || !d_expert || !d_offsets || !d_perm || !d_points_out ||
-        !d_feat_out)
+    if (B == 0) return EMC2_OK;             // nothing to write
+    if (!d_offsets) return EMC2_ERR_INVALID_ARG;
+    if (N > 0 && (!d_points || !d_vis_mask || !d_gathered || !d_expert || !d_perm || !d_points_out ||
+                  !d_feat_out))
         return EMC2_ERR_INVALID_ARG;
     if (!aligned16(d_points) || !aligned16(d_gathered) || !aligned16(d_feat_out)) return EMC2_ERR_INVALID_ARG;
-    if (d_points_out == d_points || d_feat_out == d_gathered) return EMC2_ERR_INVALID_ARG;
+    if (N > 0 && (d_points_out == d_points || d_feat_out == d_gathered)) return EMC2_ERR_INVALID_ARG;
     DeviceGuard guard(h->cfg.device);
     if (!guard.ok) return EMC2_ERR_CUDA;
     return launch_route_dispatch(h, B, N, d_points, d_vis_mask, d_gathered, d_expert, d_offsets, d_perm,

@@ -45,16 +45,18 @@ struct ScaleDev {
     uint32_t cells;         // cells per frame
     uint32_t nchunks;       // 32-byte chunks of `store` for the largest batch
     uint32_t nsumwords;     // 32-bit words of `summary`
+    uint32_t max_ovf;       // most voxels that can exceed the cap
     uint32_t* store;        // bitmap words, or int32 counts
     uint32_t* summary;      // one bit per chunk: chunk has an occupied cell
     uint32_t* chunk_prefix; // voxels before the chunk (valid for flagged chunks)
+    uint32_t* chunk_ovf;    // overflowing voxels before the chunk (capped scales)
     double* sums;           // [max voxels, C]
     int* blk_sums;          // [scan blocks, 3]
     int* blk_offs;          // [scan blocks, 3]
-    int* ovf_off;           // per voxel: start in ovf_list, -1 = not overflowing (capped scales)
-    int* ovf_cursor;        // per voxel: points appended so far
-    int* ovf_vox;           // list of overflowing voxels
-    int* ovf_list;          // global point indices of overflowing voxels
+    int* ovf_off;           // per overflowing voxel j: start of its points in ovf_list
+    int* ovf_cursor;        // per overflowing voxel j: points appended so far
+    int* ovf_vox;           // per overflowing voxel j: its row m in the unique list
+    int* ovf_list;          // global point indices of the points in overflowing voxels
     int* totals;            // [0] voxels, [1] overflowing voxels, [2] overflowing points
     int scan_blocks;
 };

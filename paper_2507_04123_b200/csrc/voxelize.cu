@@ -16,6 +16,7 @@ namespace emc2 {
 namespace {
 
 constexpr int kStatusCapacity = 1;
+constexpr int kEmitWindow = 2048;   // voxels a CTA stages in shared memory per emission round
 
 // ------------------------------------------------------------------ block-level helpers
 // Exclusive scan of three counters across the CTA; returns CTA totals in tot[].
@@ -84,17 +85,9 @@ __device__ __forceinline__ void chunk_stats(const ScaleDev& g, const Chunk& c, i
     }
 }
 
-__device__ __forceinline__ void word_stats(const ScaleDev& g, uint32_t sumword, uint32_t wi, int s[3]) {
-    while (sumword) {
-        int bit = __ffs(sumword) - 1;
-        sumword &= sumword - 1;
-        Chunk c = load_chunk(g.store, wi * 32u + bit);
-        chunk_stats(g, c, s);
-    }
-}
-
-// Rank of an occupied cell among all occupied cells of the batch (ascending cell id).
-__device__ __forceinline__ uint32_t rank_of(const ScaleDev& g, uint32_t cell, int* n_in_cell) {
+// Rank of an occupied cell among all occupied cells of the batch (ascending cell id).  For a
+// count table also returns the cell's point count and its rank among overflowing cells.
+__device__ __forceinline__ uint32_t rank_of(const ScaleDev& g, uint32_t cell, int* n_in_cell, int* ovf_rank) {
     if (g.mode == MODE_BITMAP) {
         const uint32_t chunk = cell >> 8, w = (cell >> 5) & 7u, bit = cell & 31u;
         Chunk c = load_chunk(g.store, chunk);
@@ -105,14 +98,21 @@ __device__ __forceinline__ uint32_t rank_of(const ScaleDev& g, uint32_t cell, in
             r += __popc(c.w[i] & m);
         }
         *n_in_cell = 0;
+        *ovf_rank = -1;
         return r;
     } else {
         const uint32_t chunk = cell >> 3, w = cell & 7u;
         Chunk c = load_chunk(g.store, chunk);
         uint32_t r = g.chunk_prefix[chunk];
+        int before_ovf = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) r += (i < (int)w && c.w[i] != 0u) ? 1u : 0u;
-        *n_in_cell = (int)c.w[w];
+        for (int i = 0; i < 8; ++i) {
+            r += (i < (int)w && c.w[i] != 0u) ? 1u : 0u;
+            before_ovf += (i < (int)w && g.cap > 0 && (int)c.w[i] > g.cap) ? 1 : 0;
+        }
+        const int n = (int)c.w[w];
+        *n_in_cell = n;
+        *ovf_rank = (g.cap > 0 && n > g.cap) ? (int)g.chunk_ovf[chunk] + before_ovf : -1;
         return r;
     }
 }
@@ -151,24 +151,28 @@ vox_mark_kernel(const float* __restrict__ pts, long long total, int N, ScaleDev 
 // ------------------------------------------------------------------ pass 2: ranks
 struct ScanArgs {
     ScaleDev s[2];
-    uint32_t nsum_used[2];   // summary words covering this call's B frames
+    uint32_t nchunks_used[2];   // chunks covering this call's B frames
     int capacity[2];
     int32_t* coords[2];
     int32_t* counts[2];
     int32_t* num_voxels;
     int* status;
-    int C;
 };
 
+__device__ __forceinline__ bool chunk_flagged(const ScaleDev& g, uint32_t chunk, uint32_t nchunks) {
+    return chunk < nchunks && ((g.summary[chunk >> 5] >> (chunk & 31u)) & 1u);
+}
+
+// One thread per chunk; per-CTA totals of (voxels, overflowing voxels, overflowing points).
 __global__ void __launch_bounds__(kThreads) vox_reduce_kernel(ScanArgs a) {
     __shared__ int sm[kThreads / 32][3];
     const int sc = blockIdx.y;
     const ScaleDev& g = a.s[sc];
-    const uint32_t nblk = (a.nsum_used[sc] + kThreads - 1) / kThreads;
+    const uint32_t nblk = (a.nchunks_used[sc] + kThreads - 1) / kThreads;
     if (blockIdx.x >= nblk) return;
-    const uint32_t wi = blockIdx.x * kThreads + threadIdx.x;
+    const uint32_t chunk = blockIdx.x * kThreads + threadIdx.x;
     int s[3] = {0, 0, 0};
-    if (wi < a.nsum_used[sc]) word_stats(g, g.summary[wi], wi, s);
+    if (chunk_flagged(g, chunk, a.nchunks_used[sc])) chunk_stats(g, load_chunk(g.store, chunk), s);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int k = 0; k < 3; ++k) {
@@ -189,7 +193,7 @@ __global__ void __launch_bounds__(1024) vox_blockscan_kernel(ScanArgs a) {
     __shared__ int carry[3];
     const int sc = blockIdx.x;
     const ScaleDev& g = a.s[sc];
-    const int nblk = (int)((a.nsum_used[sc] + kThreads - 1) / kThreads);
+    const int nblk = (int)((a.nchunks_used[sc] + kThreads - 1) / kThreads);
     if (threadIdx.x < 3) carry[threadIdx.x] = 0;
     __syncthreads();
     for (int base = 0; base < nblk; base += blockDim.x) {
@@ -215,76 +219,94 @@ __global__ void __launch_bounds__(1024) vox_blockscan_kernel(ScanArgs a) {
     }
 }
 
+// One thread per chunk finds the rank of its first voxel; the CTA then stages its voxels'
+// cell ids in shared memory, window by window, and writes the rows of the unique list
+// (coords, count, zeroed sums) with consecutive threads on consecutive rows.
 template <int C>
 __global__ void __launch_bounds__(kThreads) vox_emit_kernel(ScanArgs a) {
     __shared__ int sm[kThreads / 32][3];
+    __shared__ uint32_t wcell[kEmitWindow];
+    __shared__ int wn[kEmitWindow];
     const int sc = blockIdx.y;
     const ScaleDev& g = a.s[sc];
-    const uint32_t nblk = (a.nsum_used[sc] + kThreads - 1) / kThreads;
+    const uint32_t nblk = (a.nchunks_used[sc] + kThreads - 1) / kThreads;
     if (blockIdx.x >= nblk) return;
-    const uint32_t wi = blockIdx.x * kThreads + threadIdx.x;
-    uint32_t sumword = wi < a.nsum_used[sc] ? g.summary[wi] : 0u;
+    const uint32_t chunk = blockIdx.x * kThreads + threadIdx.x;
+    const bool flagged = chunk_flagged(g, chunk, a.nchunks_used[sc]);
+    Chunk c;
     int run[3] = {0, 0, 0}, tot[3];
-    word_stats(g, sumword, wi, run);
-    block_excl_scan3(run, tot, sm);
-    run[0] += g.blk_offs[blockIdx.x * 3];
-    run[1] += g.blk_offs[blockIdx.x * 3 + 1];
-    run[2] += g.blk_offs[blockIdx.x * 3 + 2];
+    if (flagged) {
+        c = load_chunk(g.store, chunk);
+        chunk_stats(g, c, run);
+    }
+    block_excl_scan3(run, tot, sm);       // run[] = exclusive offsets inside the CTA
+    const int m0 = g.blk_offs[blockIdx.x * 3];
+    const bool table = g.mode == MODE_TABLE;
+    if (flagged) {
+        g.chunk_prefix[chunk] = (uint32_t)(m0 + run[0]);
+        if (table && g.cap > 0) {
+            int j = g.blk_offs[blockIdx.x * 3 + 1] + run[1];
+            int off = g.blk_offs[blockIdx.x * 3 + 2] + run[2];
+            g.chunk_ovf[chunk] = (uint32_t)j;
+            int m = m0 + run[0];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int n = (int)c.w[i];
+                if (n > g.cap) {
+                    g.ovf_vox[j] = m;
+                    g.ovf_off[j] = off;
+                    g.ovf_cursor[j] = 0;
+                    j += 1;
+                    off += n;
+                }
+                m += n > 0;
+            }
+        }
+    }
     const int cap_rows = a.capacity[sc];
-    int32_t* coords = a.coords[sc];
-    int32_t* counts = a.counts[sc];
     const uint32_t gx = g.dims[0], gy = g.dims[1], gz = g.dims[2];
-    while (sumword) {
-        const int cb = __ffs(sumword) - 1;
-        sumword &= sumword - 1;
-        const uint32_t chunk = wi * 32u + cb;
-        const Chunk c = load_chunk(g.store, chunk);
-        g.chunk_prefix[chunk] = (uint32_t)run[0];
+    for (int wb = 0; wb < tot[0]; wb += kEmitWindow) {
+        if (flagged) {
+            int local = run[0] - wb;          // window slot of this chunk's next voxel
+            if (table) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            uint32_t word = c.w[i];
-            if (g.mode == MODE_BITMAP) {
-                while (word) {
-                    const int bit = __ffs(word) - 1;
-                    word &= word - 1;
-                    const int m = run[0]++;
-                    if (m < cap_rows) {
-                        uint32_t cell = chunk * 256u + i * 32u + bit;
-                        const uint32_t x = cell % gx; cell /= gx;
-                        const uint32_t y = cell % gy; cell /= gy;
-                        const uint32_t z = cell % gz; cell /= gz;
-                        reinterpret_cast<int4*>(coords)[m] = make_int4((int)cell, (int)z, (int)y, (int)x);
-                        counts[m] = 0;
-#pragma unroll
-                        for (int k = 0; k < C; ++k) g.sums[(size_t)m * C + k] = 0.0;
+                for (int i = 0; i < 8; ++i) {
+                    if (c.w[i]) {
+                        if (local >= 0 && local < kEmitWindow) { wcell[local] = chunk * 8u + i; wn[local] = (int)c.w[i]; }
+                        local += 1;
                     }
                 }
-            } else if (word) {
-                const int n = (int)word;
-                const int m = run[0]++;
-                const bool ovf = g.cap > 0 && n > g.cap;
-                if (m < cap_rows) {
-                    uint32_t cell = chunk * 8u + i;
-                    const uint32_t x = cell % gx; cell /= gx;
-                    const uint32_t y = cell % gy; cell /= gy;
-                    const uint32_t z = cell % gz; cell /= gz;
-                    reinterpret_cast<int4*>(coords)[m] = make_int4((int)cell, (int)z, (int)y, (int)x);
-                    counts[m] = ovf ? g.cap : n;
+            } else if (local < kEmitWindow) {
 #pragma unroll
-                    for (int k = 0; k < C; ++k) g.sums[(size_t)m * C + k] = 0.0;
-                }
-                if (g.cap > 0) {
-                    // ovf_* arrays are sized for every point of the batch, so m is in range.
-                    g.ovf_off[m] = ovf ? run[2] : -1;
-                    g.ovf_cursor[m] = 0;
-                    if (ovf) {
-                        g.ovf_vox[run[1]] = m;
-                        run[1] += 1;
-                        run[2] += n;
+                for (int i = 0; i < 8; ++i) {
+                    uint32_t word = c.w[i];
+                    while (word) {
+                        const int bit = __ffs(word) - 1;
+                        word &= word - 1;
+                        if (local >= 0 && local < kEmitWindow) wcell[local] = chunk * 256u + i * 32u + bit;
+                        local += 1;
                     }
                 }
             }
         }
+        __syncthreads();
+        const int nw = min(kEmitWindow, tot[0] - wb);
+        for (int i = threadIdx.x; i < nw; i += kThreads) {
+            const int m = m0 + wb + i;
+            if (m < cap_rows) {
+                uint32_t cell = wcell[i];
+                const uint32_t x = cell % gx; cell /= gx;
+                const uint32_t y = cell % gy; cell /= gy;
+                const uint32_t z = cell % gz; cell /= gz;
+                reinterpret_cast<int4*>(a.coords[sc])[m] = make_int4((int)cell, (int)z, (int)y, (int)x);
+                int cnt = 0;
+                if (table) cnt = (g.cap > 0 && wn[i] > g.cap) ? g.cap : wn[i];
+                a.counts[sc][m] = cnt;
+#pragma unroll
+                for (int k = 0; k < C; ++k) g.sums[(size_t)m * C + k] = 0.0;
+            }
+        }
+        __syncthreads();
     }
 }
 
@@ -295,12 +317,11 @@ __device__ __forceinline__ void accum_point(const ScaleDev& g, const float* p, i
     const uint32_t cell = cell_of(g, p[0], p[1], p[2], b);
     int pv = -1;
     if (cell != 0xFFFFFFFFu) {
-        int n;
-        const int m = (int)rank_of(g, cell, &n);
-        const bool ovf = g.mode == MODE_TABLE && g.cap > 0 && n > g.cap;
-        if (ovf) {
+        int n, j;
+        const int m = (int)rank_of(g, cell, &n, &j);
+        if (j >= 0) {
             // Which of this voxel's points survive the cap is decided by vox_overflow_kernel.
-            const int slot = g.ovf_off[m] + atomicAdd(&g.ovf_cursor[m], 1);
+            const int slot = g.ovf_off[j] + atomicAdd(&g.ovf_cursor[j], 1);
             g.ovf_list[slot] = (int)gi;
             return;
         }
@@ -357,9 +378,8 @@ vox_overflow_kernel(const float* __restrict__ pts, long long total, AccumArgs a,
     int32_t* pv = a.point_voxel[sc];
     for (int j = warp; j < novf; j += nwarps) {
         const int m = g.ovf_vox[j];
-        const int off = g.ovf_off[m];
-        const int n = g.ovf_cursor[m];
-        const int* list = g.ovf_list + off;
+        const int n = g.ovf_cursor[j];
+        const int* list = g.ovf_list + g.ovf_off[j];
         // Smallest t with #{v <= t} >= cap, by bisection on the index value.
         long long lo = -1, hi = total - 1;
         while (hi - lo > 1) {
@@ -421,8 +441,9 @@ __global__ void __launch_bounds__(kThreads) vox_finalize_kernel(AccumArgs a, int
 __global__ void __launch_bounds__(kThreads) vox_clean_kernel(ScanArgs a) {
     const int sc = blockIdx.y;
     const ScaleDev& g = a.s[sc];
+    const uint32_t nwords = (a.nchunks_used[sc] + 31) / 32;
     const uint32_t wi = blockIdx.x * kThreads + threadIdx.x;
-    if (wi >= a.nsum_used[sc]) return;
+    if (wi >= nwords) return;
     uint32_t sumword = g.summary[wi];
     if (!sumword) return;
     g.summary[wi] = 0u;
@@ -450,15 +471,15 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     const int ptiles = (int)((total + kTile - 1) / kTile);
     ScanArgs sa;
     AccumArgs aa;
-    int scan_blocks = 1;
+    int scan_blocks = 1, clean_blocks = 1;
     for (int s = 0; s < 2; ++s) {
         sa.s[s] = h->scale[s];
         aa.s[s] = h->scale[s];
         const uint64_t cells = (uint64_t)B * h->scale[s].cells;
         const uint64_t per_chunk = h->scale[s].mode == MODE_BITMAP ? 256 : 8;
-        const uint64_t chunks = (cells + per_chunk - 1) / per_chunk;
-        sa.nsum_used[s] = (uint32_t)((chunks + 31) / 32);
-        scan_blocks = max(scan_blocks, (int)((sa.nsum_used[s] + kThreads - 1) / kThreads));
+        sa.nchunks_used[s] = (uint32_t)((cells + per_chunk - 1) / per_chunk);
+        scan_blocks = max(scan_blocks, (int)((sa.nchunks_used[s] + kThreads - 1) / kThreads));
+        clean_blocks = max(clean_blocks, (int)(((sa.nchunks_used[s] + 31) / 32 + kThreads - 1) / kThreads));
         sa.capacity[s] = aa.capacity[s] = capacity[s];
         sa.coords[s] = d_coords[s];
         sa.counts[s] = aa.counts[s] = d_counts[s];
@@ -468,11 +489,10 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     }
     sa.num_voxels = d_num_voxels;
     sa.status = h->d_status;
-    sa.C = C;
     aa.bev = d_bev;
     aa.B = B;
 
-    if (d_bev) {
+    if (d_bev && B > 0) {
         const size_t n = (size_t)B * C * h->scale[1].dims[1] * h->scale[1].dims[0];
         LaunchScope ls(h, K_BEV_ZERO, st);
         if ((n & 3) == 0) {
@@ -517,7 +537,7 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     }
     {
         LaunchScope ls(h, K_VOX_CLEAN, st);
-        vox_clean_kernel<<<dim3(scan_blocks, 2), kThreads, 0, st>>>(sa);
+        vox_clean_kernel<<<dim3(clean_blocks, 2), kThreads, 0, st>>>(sa);
     }
     return check_cuda(h, cudaGetLastError());
 }
