@@ -9,7 +9,7 @@ namespace emc2 {
 
 static const char* const kKernelNames[K_KINDS] = {
     "vox_mark", "vox_reduce", "vox_blockscan", "vox_emit", "vox_accum", "vox_overflow", "vox_finalize",
-    "vox_clean", "bev_zero", "project_gather", "route_hist", "route_scan", "dispatch_scatter"};
+    "project_gather", "route_hist", "route_scan", "dispatch_scatter"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
     if (e == cudaSuccess) return EMC2_OK;
@@ -85,7 +85,8 @@ int validate(const emc2_config_t& c) {
     // Every visible pixel must fall inside the map: (dim - 1) / stride <= feat_dim - 1.
     if ((c.img_h - 1) / c.feat_stride > c.feat_h - 1 || (c.img_w - 1) / c.feat_stride > c.feat_w - 1)
         return EMC2_ERR_BAD_CONFIG;
-    if ((uint64_t)c.max_batch * c.num_cameras * c.feat_h * c.feat_w * (uint64_t)(c.feat_c / 4) > 0xFFFFFFFFFFFFull)
+    // Tap addresses are 32-bit float4 indices into the feature buffer.
+    if ((uint64_t)c.max_batch * c.num_cameras * c.feat_h * c.feat_w * (uint64_t)(c.feat_c / 4) > 0xFFFFFFF0ull)
         return EMC2_ERR_BAD_CONFIG;
     if (!(c.min_depth >= 0.0f)) return EMC2_ERR_BAD_CONFIG;
     if (c.num_thresholds < 0 || c.num_thresholds > EMC2_MAX_THRESHOLDS) return EMC2_ERR_BAD_CONFIG;
@@ -136,7 +137,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
 
     // Plan the slab: everything the stage calls need, allocated once.
     SlabPlan plan;
-    size_t o_store[2], o_summary[2], o_prefix[2], o_covf[2], o_sums[2], o_bs[2], o_bo[2], o_ovf[2][4], o_tot[2];
+    size_t o_store[2], o_summary[2], o_prefix[2], o_covf[2], o_sums[2], o_arr[2], o_cl[2], o_bs[2], o_bo[2], o_ovf[2][4], o_tot[2];
     for (int s = 0; s < 2; ++s) {
         ScaleDev& d = h->scale[s];
         const emc2_grid_t& g = c.grid[s];
@@ -155,6 +156,8 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         o_prefix[s] = plan.take((size_t)d.nsumwords * 32 * 4);
         o_covf[s] = d.cap > 0 ? plan.take((size_t)d.nsumwords * 32 * 4) : 0;
         o_sums[s] = plan.take(maxpts * c.point_floats * sizeof(double));
+        o_arr[s] = plan.take(maxpts * sizeof(int));
+        o_cl[s] = plan.take(maxpts * sizeof(uint32_t));
         o_bs[s] = plan.take((size_t)d.scan_blocks * 3 * sizeof(int));
         o_bo[s] = plan.take((size_t)d.scan_blocks * 3 * sizeof(int));
         for (int k = 0; k < 3; ++k) o_ovf[s][k] = d.cap > 0 ? plan.take((size_t)d.max_ovf * sizeof(int)) : 0;
@@ -170,7 +173,8 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     h->slab_bytes = plan.off;
     cudaError_t e = cudaMalloc(&h->slab, h->slab_bytes);
     if (e != cudaSuccess) { h->slab = nullptr; delete h; return EMC2_ERR_CUDA; }
-    // The voxel stores and summaries must be all-zero between calls; every call restores that.
+    // The voxel stores, summaries, sums and arrival counters must be all-zero between calls;
+    // every call restores that.
     e = cudaMemset(h->slab, 0, h->slab_bytes);
     if (e != cudaSuccess) { cudaFree(h->slab); delete h; return EMC2_ERR_CUDA; }
     char* base = static_cast<char*>(h->slab);
@@ -181,6 +185,8 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         d.chunk_prefix = reinterpret_cast<uint32_t*>(base + o_prefix[s]);
         d.chunk_ovf = d.cap > 0 ? reinterpret_cast<uint32_t*>(base + o_covf[s]) : nullptr;
         d.sums = reinterpret_cast<double*>(base + o_sums[s]);
+        d.arrivals = reinterpret_cast<int*>(base + o_arr[s]);
+        d.cell_list = reinterpret_cast<uint32_t*>(base + o_cl[s]);
         d.blk_sums = reinterpret_cast<int*>(base + o_bs[s]);
         d.blk_offs = reinterpret_cast<int*>(base + o_bo[s]);
         d.ovf_off = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][0]) : nullptr;

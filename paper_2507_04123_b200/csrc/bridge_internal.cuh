@@ -24,8 +24,6 @@ enum KernelKind {
     K_VOX_ACCUM,
     K_VOX_OVERFLOW,
     K_VOX_FINALIZE,
-    K_VOX_CLEAN,
-    K_BEV_ZERO,
     K_PROJECT_GATHER,
     K_ROUTE_HIST,
     K_ROUTE_SCAN,
@@ -50,7 +48,9 @@ struct ScaleDev {
     uint32_t* summary;      // one bit per chunk: chunk has an occupied cell
     uint32_t* chunk_prefix; // voxels before the chunk (valid for flagged chunks)
     uint32_t* chunk_ovf;    // overflowing voxels before the chunk (capped scales)
-    double* sums;           // [max voxels, C]
+    double* sums;           // [max voxels, C] fp64 sums of all but the first point; zero between calls
+    int* arrivals;          // [max voxels] points accumulated so far; zero between calls
+    uint32_t* cell_list;    // [max voxels] cell id of each unique voxel
     int* blk_sums;          // [scan blocks, 3]
     int* blk_offs;          // [scan blocks, 3]
     int* ovf_off;           // per overflowing voxel j: start of its points in ovf_list

@@ -4,9 +4,11 @@
 //
 // One CTA owns a tile of 256 consecutive points.  Phase 1: one thread per point projects into
 // all K cameras (fp32 fma chain and IEEE divide, so the mask is reproducible bit for bit),
-// writes uvd / mask / camera, and leaves the four tap addresses and two weights in shared
-// memory.  Phase 2: the CTA walks the tile's output rows as a flat array of float4, so every
-// 128-bit store is coalesced and each thread keeps several independent 4-tap loads in flight.
+// writes uvd / mask / camera, and leaves one 16-byte record per point in shared memory: the
+// address of tap (y0, x0), two clamp flags and the two weights.  Phase 2: the CTA is laid out
+// as 16 rows x (Cf/4) columns of threads; every thread keeps its float4 column and walks the
+// tile's rows 16 at a time, so a warp's 128-bit loads and stores cover whole contiguous rows,
+// no index division is needed, and each thread has 16 independent tap loads in flight.
 #include "bridge_internal.cuh"
 
 namespace emc2 {
@@ -25,20 +27,25 @@ struct PgArgs {
     float min_depth, inv_stride;
 };
 
-struct Tap {
-    uint32_t base;   // float4 index of tap (y0, x0) inside the whole feat buffer / 1; 0xFFFFFFFF = zero row
-    uint32_t dx;     // float4 offset to x1 (0 when clamped)
-    uint32_t dy;     // float4 offset to y1 (0 when clamped)
-    float wx, wy;
-};
+constexpr uint32_t kZeroRow = 0xFFFFFFFFu;
 
+__device__ __forceinline__ float4 blend(const float4& f00, const float4& f01, const float4& f10, const float4& f11,
+                                        float wx, float wy) {
+    const float ax = 1.0f - wx, ay = 1.0f - wy;
+    float4 o;
+    o.x = ay * (ax * f00.x + wx * f01.x) + wy * (ax * f10.x + wx * f11.x);
+    o.y = ay * (ax * f00.y + wx * f01.y) + wy * (ax * f10.y + wx * f11.y);
+    o.z = ay * (ax * f00.z + wx * f01.z) + wy * (ax * f10.z + wx * f11.z);
+    o.w = ay * (ax * f00.w + wx * f01.w) + wy * (ax * f10.w + wx * f11.w);
+    return o;
+}
+
+// CF4 > 0: Cf/4 known at compile time, blockDim.x == 16 * CF4.  CF4 == 0: any Cf, 256 threads.
 template <int C, int CF4>
-__global__ void __launch_bounds__(kThreads) project_gather_kernel(PgArgs a) {
+__global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) project_gather_kernel(PgArgs a) {
     __shared__ __align__(16) float sp[kTile * C];
     __shared__ float suvd[kTile * 3];
-    __shared__ uint64_t sbase[kTile];
-    __shared__ uint32_t sdx[kTile], sdy[kTile];
-    __shared__ float swx[kTile], swy[kTile];
+    __shared__ uint4 srow[kTile];          // {tap (y0,x0) as a float4 index, clamp flags, wx, wy}
 
     const long long g0 = (long long)blockIdx.x * kTile;
     const int npts = (int)min((long long)kTile, a.total - g0);
@@ -71,48 +78,60 @@ __global__ void __launch_bounds__(kThreads) project_gather_kernel(PgArgs a) {
         suvd[t * 3] = bu; suvd[t * 3 + 1] = bv; suvd[t * 3 + 2] = bd;
         a.vis[gi] = (uint8_t)mask;
         a.cam[gi] = (int8_t)best;
+        uint4 rec = make_uint4(kZeroRow, 0u, 0u, 0u);
         if (best >= 0) {
             // Texel coordinates: stride is a power of two, so the scaling is exact.
             const float fx = bu * a.inv_stride, fy = bv * a.inv_stride;
             const float flx = floorf(fx), fly = floorf(fy);
             int x0 = (int)flx, y0 = (int)fly;
-            swx[t] = fx - flx;
-            swy[t] = fy - fly;
             const int x1 = min(x0 + 1, a.Wf - 1), y1 = min(y0 + 1, a.Hf - 1);
             x0 = min(x0, a.Wf - 1);
             y0 = min(y0, a.Hf - 1);
-            const uint64_t map = ((uint64_t)b * a.K + best) * a.Hf;
-            sbase[t] = ((map + y0) * a.Wf + x0) * (uint64_t)cf4;
-            sdx[t] = (uint32_t)(x1 - x0) * cf4;
-            sdy[t] = (uint32_t)(y1 - y0) * a.Wf * cf4;
-        } else {
-            sbase[t] = ~0ull;
+            const uint32_t map = ((uint32_t)b * a.K + best) * a.Hf;
+            rec.x = ((map + y0) * a.Wf + x0) * (uint32_t)cf4;
+            rec.y = (uint32_t)(x1 - x0) | ((uint32_t)(y1 - y0) << 1);
+            rec.z = __float_as_uint(fx - flx);
+            rec.w = __float_as_uint(fy - fly);
         }
+        srow[t] = rec;
     }
     __syncthreads();
 
     // uvd: the tile's 3*npts floats are contiguous in global memory.
-    for (int i = t; i < npts * 3; i += kThreads) a.uvd[g0 * 3 + i] = suvd[i];
+    for (int i = t; i < npts * 3; i += blockDim.x) a.uvd[g0 * 3 + i] = suvd[i];
 
-    const int items = npts * cf4;
     float4* out = a.out + (size_t)g0 * cf4;
+    const uint32_t dyv = (uint32_t)a.Wf * cf4;
+    if (CF4 > 0) {
+        const int c = t % CF4, r0 = t / CF4;
 #pragma unroll 4
-    for (int i = t; i < items; i += kThreads) {
-        const int r = i / cf4, c = i - r * cf4;
-        const uint64_t base = sbase[r];
-        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (base != ~0ull) {
-            const float4* p = a.feat + base + c;
-            const uint32_t dx = sdx[r], dy = sdy[r];
-            const float4 f00 = __ldg(p), f01 = __ldg(p + dx), f10 = __ldg(p + dy), f11 = __ldg(p + dy + dx);
-            const float wx = swx[r], wy = swy[r];
-            const float ax = 1.0f - wx, ay = 1.0f - wy;
-            o.x = ay * (ax * f00.x + wx * f01.x) + wy * (ax * f10.x + wx * f11.x);
-            o.y = ay * (ax * f00.y + wx * f01.y) + wy * (ax * f10.y + wx * f11.y);
-            o.z = ay * (ax * f00.z + wx * f01.z) + wy * (ax * f10.z + wx * f11.z);
-            o.w = ay * (ax * f00.w + wx * f01.w) + wy * (ax * f10.w + wx * f11.w);
+        for (int j = 0; j < kTile / 16; ++j) {
+            const int r = r0 + 16 * j;
+            if (r >= npts) break;
+            const uint4 rec = srow[r];
+            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (rec.x != kZeroRow) {
+                const float4* p = a.feat + rec.x + c;
+                const uint32_t dx = (rec.y & 1u) ? (uint32_t)CF4 : 0u, dy = (rec.y & 2u) ? dyv : 0u;
+                const float4 f00 = __ldg(p), f01 = __ldg(p + dx), f10 = __ldg(p + dy), f11 = __ldg(p + dy + dx);
+                o = blend(f00, f01, f10, f11, __uint_as_float(rec.z), __uint_as_float(rec.w));
+            }
+            __stcs(out + r * CF4 + c, o);
         }
-        out[i] = o;
+    } else {
+        const int items = npts * cf4;
+        for (int i = t; i < items; i += blockDim.x) {
+            const int r = i / cf4, c = i - r * cf4;
+            const uint4 rec = srow[r];
+            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (rec.x != kZeroRow) {
+                const float4* p = a.feat + rec.x + c;
+                const uint32_t dx = (rec.y & 1u) ? (uint32_t)cf4 : 0u, dy = (rec.y & 2u) ? dyv : 0u;
+                const float4 f00 = __ldg(p), f01 = __ldg(p + dx), f10 = __ldg(p + dy), f11 = __ldg(p + dy + dx);
+                o = blend(f00, f01, f10, f11, __uint_as_float(rec.z), __uint_as_float(rec.w));
+            }
+            __stcs(out + i, o);
+        }
     }
 }
 
@@ -120,8 +139,8 @@ template <int C>
 void launch_c(emc2_bridge* h, const PgArgs& a, int tiles, cudaStream_t st) {
     LaunchScope ls(h, K_PROJECT_GATHER, st);
     switch (a.cf4) {
-        case 16: project_gather_kernel<C, 16><<<tiles, kThreads, 0, st>>>(a); break;
-        case 20: project_gather_kernel<C, 20><<<tiles, kThreads, 0, st>>>(a); break;
+        case 16: project_gather_kernel<C, 16><<<tiles, 16 * 16, 0, st>>>(a); break;
+        case 20: project_gather_kernel<C, 20><<<tiles, 16 * 20, 0, st>>>(a); break;
         default: project_gather_kernel<C, 0><<<tiles, kThreads, 0, st>>>(a); break;
     }
 }

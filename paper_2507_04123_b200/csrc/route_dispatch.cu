@@ -115,10 +115,11 @@ struct ScatterArgs {
     int N, tiles, E, cf4;
 };
 
+// CF4 > 0: Cf/4 known at compile time, blockDim.x == 16 * CF4.  CF4 == 0: any Cf, 256 threads.
 template <int C, int CF4>
-__global__ void __launch_bounds__(kThreads) dispatch_scatter_kernel(ScatterArgs a) {
+__global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) dispatch_scatter_kernel(ScatterArgs a) {
     __shared__ int sdest[kTile];
-    __shared__ int wcnt[kThreads / 32][EMC2_MAX_EXPERTS];
+    __shared__ int wcnt[kTile / 32][EMC2_MAX_EXPERTS];
     const int b = blockIdx.y, tile = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int i0 = tile * kTile;
     const int npts = min(kTile, a.N - i0);
@@ -126,12 +127,16 @@ __global__ void __launch_bounds__(kThreads) dispatch_scatter_kernel(ScatterArgs 
     const size_t g0 = f0 + i0;
     const int cf4 = CF4 > 0 ? CF4 : a.cf4;
 
-    const int e = t < npts ? (int)a.expert[g0 + t] : -1;
-    int rank = 0;
-    for (int k = 0; k < a.E; ++k) {
-        const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
-        if (e == k) rank = __popc(m & ((1u << lane) - 1u));
-        if (lane == 0) wcnt[warp][k] = __popc(m);
+    // Stable rank inside the tile: ballots per expert (warps past the tile only take part in
+    // the barriers).
+    int e = -1, rank = 0;
+    if (t < kTile) {
+        e = t < npts ? (int)a.expert[g0 + t] : -1;
+        for (int k = 0; k < a.E; ++k) {
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
+            if (e == k) rank = __popc(m & ((1u << lane) - 1u));
+            if (lane == 0) wcnt[warp][k] = __popc(m);
+        }
     }
     __syncthreads();
     if (t < npts) {
@@ -146,19 +151,36 @@ __global__ void __launch_bounds__(kThreads) dispatch_scatter_kernel(ScatterArgs 
     // Point rows: the tile's source floats are contiguous.
     const float* psrc = a.pts + g0 * C;
     float* pdst = a.pts_out + f0 * C;
-    for (int i = t; i < npts * C; i += kThreads) {
+    for (int i = t; i < npts * C; i += blockDim.x) {
         const int r = i / C, c = i - r * C;
         pdst[(size_t)sdest[r] * C + c] = __ldg(psrc + i);
     }
-    // Feature rows: read the tile as a flat float4 stream, write whole rows to their slots.
+    // Feature rows: 16 rows x Cf/4 columns of threads; each thread keeps its column, reads
+    // eight rows (eight independent 128-bit streaming loads), then writes them to their slots.
     const float4* fsrc = a.feat + g0 * cf4;
     float4* fdst = a.feat_out + f0 * cf4;
-    const int items = npts * cf4;
-#pragma unroll 5
-    for (int i = t; i < items; i += kThreads) {
-        const int r = i / cf4, c = i - r * cf4;
-        const float4 v = __ldcs(fsrc + i);
-        __stcs(fdst + (size_t)sdest[r] * cf4 + c, v);
+    if (CF4 > 0) {
+        const int c = t % CF4, r0 = t / CF4;
+#pragma unroll
+        for (int j0 = 0; j0 < kTile / 16; j0 += 8) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int r = r0 + 16 * (j0 + u);
+                if (r < npts) v[u] = __ldcs(fsrc + r * CF4 + c);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int r = r0 + 16 * (j0 + u);
+                if (r < npts) __stcs(fdst + (size_t)sdest[r] * CF4 + c, v[u]);
+            }
+        }
+    } else {
+        const int items = npts * cf4;
+        for (int i = t; i < items; i += blockDim.x) {
+            const int r = i / cf4, c = i - r * cf4;
+            __stcs(fdst + (size_t)sdest[r] * cf4 + c, __ldcs(fsrc + i));
+        }
     }
 }
 
@@ -166,8 +188,8 @@ template <int C>
 void launch_scatter(emc2_bridge* h, const ScatterArgs& a, dim3 grid, cudaStream_t st) {
     LaunchScope ls(h, K_DISPATCH_SCATTER, st);
     switch (a.cf4) {
-        case 16: dispatch_scatter_kernel<C, 16><<<grid, kThreads, 0, st>>>(a); break;
-        case 20: dispatch_scatter_kernel<C, 20><<<grid, kThreads, 0, st>>>(a); break;
+        case 16: dispatch_scatter_kernel<C, 16><<<grid, 16 * 16, 0, st>>>(a); break;
+        case 20: dispatch_scatter_kernel<C, 20><<<grid, 16 * 20, 0, st>>>(a); break;
         default: dispatch_scatter_kernel<C, 0><<<grid, kThreads, 0, st>>>(a); break;
     }
 }

@@ -39,7 +39,7 @@ def test_status_strings(pkg):
     lib = pkg.load_library()
     texts = {lib.emc2_status_string(s).decode() for s in range(0, -7, -1)}
     assert len(texts) == 7 and "ok" in texts
-    assert lib.emc2_bridge_kernel_kinds() == len({lib.emc2_bridge_kernel_name(k) for k in range(13)})
+    assert lib.emc2_bridge_kernel_kinds() == len({lib.emc2_bridge_kernel_name(k) for k in range(lib.emc2_bridge_kernel_kinds())})
 
 
 def _create(pkg, cfg):
