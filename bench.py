@@ -261,10 +261,12 @@ def run_ours(args, w):
         nv_host.copy_(e2e_bufs["vox"]["num_voxels"], non_blocking=True)
         torch.cuda.current_stream().synchronize()
 
-    for _ in range(2):
-        e2e_step()
     e2e_steps = max(3, min(args.steps, 10))
-    e2e_secs = max_over_ranks(time_steps(e2e_step, e2e_steps, sync, barrier))
+    e2e_secs = None
+    if not args.no_e2e:
+        for _ in range(2):
+            e2e_step()
+        e2e_secs = max_over_ranks(time_steps(e2e_step, e2e_steps, sync, barrier))
     clocks = sampler.stop() if sampler else None
     h2d = sum(int(host[k].numel() * host[k].element_size()) for k in ("points", "proj", "feat"))
     d2h = int(off_host.numel() * 4 + nv_host.numel() * 4)
@@ -325,7 +327,7 @@ def run_ours(args, w):
                      "algorithmic_bytes_per_launch": kb[dom], "ms_per_launch": dom_ms},
         "kernels": per_kernel,
         "e2e": {"value": world * B * e2e_steps / e2e_secs, "unit": "frames/s", "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_secs / e2e_steps * 1e3},
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_secs / e2e_steps * 1e3} if e2e_secs else None,
         "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
         "unique_voxels": [int(nv[0]), int(nv[1])], "distinct_texels": texels,
     }
@@ -377,6 +379,7 @@ def main():
     ap.add_argument("--points", type=int, default=None)
     ap.add_argument("--feature-frames", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--sweep", action="store_true")
     args = ap.parse_args()
     w = gen.workload(args.config)
