@@ -212,15 +212,13 @@ def run_ours(args, w):
         if use_dist:
             dist.barrier()
 
+    from paper_2507_04123_b200 import sharding
+
     def max_over_ranks(x):
-        if not use_dist:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return sharding.max_over_ranks(x, dev)
 
     B, N = w.B, w.N
-    frames = list(range(rank * B, rank * B + B))           # every rank owns its own frames
+    frames = sharding.frames_for_rank(rank, world, B)      # every rank owns its own frames
     batch = gen.make_batch(w, frames=frames, feature_frames=args.feature_frames)
     host = {k: torch.from_numpy(v).pin_memory() for k, v in batch.items()}
     d = {k: v.to(dev, non_blocking=True) for k, v in host.items()}
