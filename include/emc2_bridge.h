@@ -47,7 +47,8 @@ typedef enum {
     EMC2_ERR_CUDA = -3,        /* a CUDA runtime call failed; see emc2_bridge_last_cuda_error */
     EMC2_ERR_CAPACITY = -4,    /* more unique voxels than capacity[s] (device-detected, sticky) */
     EMC2_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (device-detected, sticky) */
-    EMC2_ERR_INTERNAL = -6
+    EMC2_ERR_INTERNAL = -6,
+    EMC2_ERR_TOO_LARGE = -7    /* the call needs more scratch than a fixed-size scratch area holds */
 } emc2_status_t;
 
 #define EMC2_MAX_CAMERAS 8
@@ -135,6 +136,37 @@ int emc2_route_dispatch(emc2_bridge_t* bridge, int32_t B, int32_t N, const float
                         const uint8_t* d_vis_mask, const float* d_gathered, uint8_t* d_expert,
                         int32_t* d_offsets, int32_t* d_perm, float* d_points_out, float* d_feat_out,
                         void* cuda_stream);
+
+/* Stages 3 and 4 for callers that must not allocate device memory (the paper has no counterpart;
+ * this is a packaging variant of emc2_route_dispatch).
+ *
+ * emc2_bridge_create() obtains its scratch with cudaMalloc.  Some hosts cannot do that at the point
+ * where they need the dispatch: a plug-in running inside an engine that owns the whole device heap
+ * and forbids allocation outside its own pool, or a real-time loop that may not take the driver's
+ * allocation lock.  This entry point needs no handle and calls no allocator of any kind: its only
+ * scratch (the per-tile expert histograms and their prefix sums) lives in a fixed array that is
+ * part of the library image, EMC2_STATIC_SCRATCH_BYTES in size, which every device that loads the
+ * library holds from load until the process exits.
+ *
+ * Arguments and outputs are exactly those of emc2_route_dispatch; in place of the handle it reads,
+ * from `config` (HOST memory), only device, point_floats, feat_c, num_thresholds, thresholds,
+ * num_experts and lut (other fields are ignored).  All buffers are the caller's.
+ *   - Size limit: B * ceil(N / 256) * num_experts must not exceed EMC2_STATIC_SCRATCH_ENTRIES;
+ *     a larger call returns EMC2_ERR_TOO_LARGE and enqueues nothing (B <= EMC2_MAX_BATCH still
+ *     applies; there is no max_points).
+ *   - The first call on each device looks up the array's device address (one runtime query, no
+ *     allocation); make that first call outside any stream capture.
+ *   - The array is shared by every call in the process and keeps whatever the previous call left;
+ *     each call overwrites all entries it later reads, so nothing has to be cleared.  Two calls
+ *     whose kernels can overlap on the same device (different streams) race on it: order them.
+ * Errors: EMC2_ERR_INVALID_ARG, EMC2_ERR_BAD_CONFIG (of the fields listed), EMC2_ERR_TOO_LARGE,
+ * EMC2_ERR_CUDA. */
+#define EMC2_STATIC_SCRATCH_ENTRIES (1 << 18)
+#define EMC2_STATIC_SCRATCH_BYTES (2 * EMC2_STATIC_SCRATCH_ENTRIES * 4)
+int emc2_route_dispatch_static(const emc2_config_t* config, int32_t B, int32_t N, const float* d_points,
+                               const uint8_t* d_vis_mask, const float* d_gathered, uint8_t* d_expert,
+                               int32_t* d_offsets, int32_t* d_perm, float* d_points_out,
+                               float* d_feat_out, void* cuda_stream);
 
 /* Waits for `cuda_stream`, then returns and clears the sticky device status: EMC2_OK,
  * EMC2_ERR_CAPACITY, EMC2_ERR_TIMEOUT or EMC2_ERR_CUDA. */

@@ -24,13 +24,15 @@ EMC2_ERR_CUDA = -3
 EMC2_ERR_CAPACITY = -4
 EMC2_ERR_TIMEOUT = -5
 EMC2_ERR_INTERNAL = -6
+EMC2_ERR_TOO_LARGE = -7
+STATIC_SCRATCH_ENTRIES = 1 << 18
 
 # Every symbol include/emc2_bridge.h declares.
 ABI_SYMBOLS = (
     "emc2_bridge_create", "emc2_voxelize", "emc2_project_gather", "emc2_route_dispatch",
     "emc2_bridge_status", "emc2_bridge_destroy", "emc2_status_string", "emc2_bridge_last_cuda_error",
     "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
-    "emc2_bridge_profile_enable", "emc2_bridge_profile_read",
+    "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
 )
 
 
@@ -73,6 +75,7 @@ def load_library() -> ctypes.CDLL:
     lib.emc2_voxelize.argtypes = [vp, i32, i32, vp, P(vp), P(vp), P(vp), P(vp), P(i32), vp, vp, vp]
     lib.emc2_project_gather.argtypes = [vp, i32, i32] + [vp] * 8
     lib.emc2_route_dispatch.argtypes = [vp, i32, i32] + [vp] * 9
+    lib.emc2_route_dispatch_static.argtypes = [P(Emc2Config), i32, i32] + [vp] * 9
     lib.emc2_bridge_status.argtypes = [vp, vp]
     lib.emc2_bridge_destroy.argtypes = [vp]
     lib.emc2_status_string.argtypes = [ctypes.c_int]
@@ -134,6 +137,37 @@ def _check(t: torch.Tensor, dtype, shape, name: str, device) -> None:
     if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous() or t.device != device:
         raise ValueError(f"{name}: expected contiguous {dtype} {tuple(shape)} on {device}, "
                          f"got {t.dtype} {tuple(t.shape)} on {t.device}")
+
+
+def route_dispatch_static(config: Emc2Config, points: torch.Tensor, vis_mask: torch.Tensor,
+                          gathered: torch.Tensor, out: Dict[str, torch.Tensor]) -> Dict[str, torch.Tensor]:
+    """emc2_route_dispatch_static: stages 3 and 4 without a handle and without any allocation.
+
+    For hosts that may not allocate device memory where they dispatch (an engine plug-in confined
+    to the engine's pool, a real-time loop).  The library's only scratch is a fixed array inside
+    its image, so the call is limited to B * ceil(N / 256) * num_experts <= STATIC_SCRATCH_ENTRIES
+    and calls that can overlap on one device must be ordered by the caller.  ``out`` must hold the
+    five preallocated output tensors of :meth:`Bridge.route_dispatch`; nothing is allocated here.
+    """
+    lib = load_library()
+    B, N, C = points.shape
+    dev = points.device
+    _check(points, torch.float32, (B, N, config.point_floats), "points", dev)
+    _check(vis_mask, torch.uint8, (B, N), "vis_mask", dev)
+    _check(gathered, torch.float32, (B, N, config.feat_c), "gathered", dev)
+    _check(out["expert"], torch.uint8, (B, N), "expert", dev)
+    _check(out["offsets"], torch.int32, (B, config.num_experts + 1), "offsets", dev)
+    _check(out["perm"], torch.int32, (B, N), "perm", dev)
+    _check(out["points_out"], torch.float32, (B, N, C), "points_out", dev)
+    _check(out["feat_out"], torch.float32, (B, N, config.feat_c), "feat_out", dev)
+    rc = lib.emc2_route_dispatch_static(ctypes.byref(config), B, N, points.data_ptr(), vis_mask.data_ptr(),
+                                        gathered.data_ptr(), out["expert"].data_ptr(),
+                                        out["offsets"].data_ptr(), out["perm"].data_ptr(),
+                                        out["points_out"].data_ptr(), out["feat_out"].data_ptr(),
+                                        torch.cuda.current_stream(dev).cuda_stream)
+    if rc != EMC2_OK:
+        raise Emc2Error(rc, "emc2_route_dispatch_static", lib.emc2_status_string(rc).decode())
+    return out
 
 
 class Bridge:

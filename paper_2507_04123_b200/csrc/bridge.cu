@@ -297,6 +297,7 @@ const char* emc2_status_string(int status) {
         case EMC2_ERR_CAPACITY: return "more unique voxels than capacity";
         case EMC2_ERR_TIMEOUT: return "bounded device wait timed out";
         case EMC2_ERR_INTERNAL: return "internal error";
+        case EMC2_ERR_TOO_LARGE: return "call exceeds the fixed scratch area";
         default: return "unknown status";
     }
 }

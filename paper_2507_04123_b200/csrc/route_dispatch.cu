@@ -8,6 +8,9 @@
 // per-tile bases; (3) one CTA per tile ranks its points inside the tile with ballots and
 // popcounts, writes the permutation and moves the 16/20-byte point rows and the 256/320-byte
 // feature rows with coalesced 128-bit accesses.
+#include <cmath>
+#include <mutex>
+
 #include "bridge_internal.cuh"
 
 namespace emc2 {
@@ -230,3 +233,116 @@ int launch_route_dispatch(emc2_bridge* h, int B, int N, const float* d_points, c
 }
 
 }  // namespace emc2
+
+// ------------------------------------------------------------------ handle-free variant
+// emc2_route_dispatch_static: the same three kernels, with the tile histograms and tile bases in
+// an array that is part of the library image instead of a cudaMalloc'ed slab.
+namespace emc2 {
+namespace {
+
+// [0, ENTRIES): tile counts; [ENTRIES, 2*ENTRIES): tile bases.  Device code could name this
+// array directly; host code may only use the address cudaGetSymbolAddress reports (the host-side
+// symbol is a stand-in, not a device pointer).
+static __device__ __align__(256) int g_static_route_scratch[2 * EMC2_STATIC_SCRATCH_ENTRIES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+int* g_static_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the array on `device`, which must be the current device.  Looked up once per
+// device and cached.
+cudaError_t static_scratch(int device, int** out) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void* p = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&p, g_static_route_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_ptr[device] = static_cast<int*>(p);
+    }
+    *out = g_static_ptr[device];
+    return cudaSuccess;
+}
+
+bool aligned16_static(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+}  // namespace emc2
+
+extern "C" int emc2_route_dispatch_static(const emc2_config_t* config, int32_t B, int32_t N,
+                                          const float* d_points, const uint8_t* d_vis_mask,
+                                          const float* d_gathered, uint8_t* d_expert, int32_t* d_offsets,
+                                          int32_t* d_perm, float* d_points_out, float* d_feat_out,
+                                          void* cuda_stream) {
+    using namespace emc2;
+    if (!config) return EMC2_ERR_INVALID_ARG;
+    const emc2_config_t& c = *config;
+    // Only the fields this stage reads are checked.
+    if (c.device < 0 || c.device >= kMaxDevices) return EMC2_ERR_BAD_CONFIG;
+    if (c.point_floats != 4 && c.point_floats != 5) return EMC2_ERR_BAD_CONFIG;
+    if (c.feat_c < 4 || (c.feat_c & 3)) return EMC2_ERR_BAD_CONFIG;
+    if (c.num_thresholds < 0 || c.num_thresholds > EMC2_MAX_THRESHOLDS) return EMC2_ERR_BAD_CONFIG;
+    for (int t = 0; t < c.num_thresholds; ++t) {
+        if (!(c.thresholds[t] >= 0.0f) || !std::isfinite(c.thresholds[t])) return EMC2_ERR_BAD_CONFIG;
+        if (t && !(c.thresholds[t] >= c.thresholds[t - 1])) return EMC2_ERR_BAD_CONFIG;
+    }
+    if (c.num_experts < 1 || c.num_experts > EMC2_MAX_EXPERTS) return EMC2_ERR_BAD_CONFIG;
+    for (int v = 0; v < 2; ++v)
+        for (int d = 0; d <= c.num_thresholds; ++d)
+            if (c.lut[v][d] >= c.num_experts) return EMC2_ERR_BAD_CONFIG;
+    if (B < 0 || N < 0 || B > EMC2_MAX_BATCH) return EMC2_ERR_INVALID_ARG;
+    const int E = c.num_experts;
+    const int tiles = (N + kTile - 1) / kTile;
+    if ((int64_t)B * tiles * E > (int64_t)EMC2_STATIC_SCRATCH_ENTRIES) return EMC2_ERR_TOO_LARGE;
+    if (B == 0) return EMC2_OK;
+    if (!d_offsets) return EMC2_ERR_INVALID_ARG;
+    if (N > 0 && (!d_points || !d_vis_mask || !d_gathered || !d_expert || !d_perm || !d_points_out ||
+                  !d_feat_out))
+        return EMC2_ERR_INVALID_ARG;
+    if (!aligned16_static(d_points) || !aligned16_static(d_gathered) || !aligned16_static(d_feat_out))
+        return EMC2_ERR_INVALID_ARG;
+    if (N > 0 && (d_points_out == d_points || d_feat_out == d_gathered)) return EMC2_ERR_INVALID_ARG;
+
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) return EMC2_ERR_CUDA;
+    if (prev != c.device && cudaSetDevice(c.device) != cudaSuccess) return EMC2_ERR_CUDA;
+    int rc = EMC2_OK;
+    int* scratch = nullptr;
+    if (static_scratch(c.device, &scratch) != cudaSuccess) rc = EMC2_ERR_CUDA;
+    if (rc == EMC2_OK) {
+        cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+        int* tile_counts = scratch;
+        int* tile_base = scratch + EMC2_STATIC_SCRATCH_ENTRIES;
+        const dim3 grid(tiles > 0 ? tiles : 1, B);
+        if (tiles > 0) {
+            RouteArgs ra;
+            ra.pts = d_points; ra.vis = d_vis_mask; ra.expert = d_expert; ra.tile_counts = tile_counts;
+            ra.N = N; ra.tiles = tiles; ra.E = E; ra.T = c.num_thresholds;
+            for (int k = 0; k < EMC2_MAX_THRESHOLDS; ++k)
+                ra.thr2[k] = k < c.num_thresholds ? c.thresholds[k] * c.thresholds[k] : 0.0f;
+            for (int k = 0; k < 16; ++k) ra.lut[k] = c.lut[k >> 3][k & 7];
+            if (c.point_floats == 4) route_hist_kernel<4><<<grid, kThreads, 0, st>>>(ra);
+            else route_hist_kernel<5><<<grid, kThreads, 0, st>>>(ra);
+        }
+        route_scan_kernel<<<B, kThreads, 0, st>>>(tile_counts, tile_base, d_offsets, tiles, E, N);
+        if (tiles > 0) {
+            ScatterArgs sa;
+            sa.pts = d_points; sa.feat = reinterpret_cast<const float4*>(d_gathered); sa.expert = d_expert;
+            sa.tile_base = tile_base; sa.perm = d_perm; sa.pts_out = d_points_out;
+            sa.feat_out = reinterpret_cast<float4*>(d_feat_out);
+            sa.N = N; sa.tiles = tiles; sa.E = E; sa.cf4 = c.feat_c / 4;
+            const int threads = sa.cf4 == 16 ? 256 : sa.cf4 == 20 ? 320 : kThreads;
+            if (c.point_floats == 4) {
+                if (sa.cf4 == 16) dispatch_scatter_kernel<4, 16><<<grid, threads, 0, st>>>(sa);
+                else if (sa.cf4 == 20) dispatch_scatter_kernel<4, 20><<<grid, threads, 0, st>>>(sa);
+                else dispatch_scatter_kernel<4, 0><<<grid, threads, 0, st>>>(sa);
+            } else {
+                if (sa.cf4 == 16) dispatch_scatter_kernel<5, 16><<<grid, threads, 0, st>>>(sa);
+                else if (sa.cf4 == 20) dispatch_scatter_kernel<5, 20><<<grid, threads, 0, st>>>(sa);
+                else dispatch_scatter_kernel<5, 0><<<grid, threads, 0, st>>>(sa);
+            }
+        }
+        if (cudaGetLastError() != cudaSuccess) rc = EMC2_ERR_CUDA;
+    }
+    if (prev != c.device) cudaSetDevice(prev);
+    return rc;
+}
