@@ -8,7 +8,7 @@
 namespace emc2 {
 
 static const char* const kKernelNames[K_KINDS] = {
-    "vox_mark", "vox_reduce", "vox_blockscan", "vox_emit", "vox_accum", "vox_overflow", "vox_finalize",
+    "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
     "project_gather", "route_hist", "route_scan", "dispatch_scatter"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
@@ -59,7 +59,8 @@ int validate(const emc2_config_t& c) {
     if (c.device < 0) return EMC2_ERR_BAD_CONFIG;
     if (c.max_batch < 1 || c.max_batch > EMC2_MAX_BATCH) return EMC2_ERR_BAD_CONFIG;
     if (c.max_points < 1) return EMC2_ERR_BAD_CONFIG;
-    if ((int64_t)c.max_batch * c.max_points > (int64_t)1 << 30) return EMC2_ERR_BAD_CONFIG;
+    // Per-voxel point counts are accumulated in fp32, which is exact up to 2^24.
+    if ((int64_t)c.max_batch * c.max_points > (int64_t)1 << 24) return EMC2_ERR_BAD_CONFIG;
     if (c.point_floats != 4 && c.point_floats != 5) return EMC2_ERR_BAD_CONFIG;
     for (int s = 0; s < 2; ++s) {
         const emc2_grid_t& g = c.grid[s];
@@ -135,9 +136,12 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     for (int t = 0; t < EMC2_MAX_THRESHOLDS; ++t)
         h->thr2[t] = t < c.num_thresholds ? c.thresholds[t] * c.thresholds[t] : 0.0f;
 
+    h->scan_blocks = voxel_scan_max_blocks();
+    if (h->scan_blocks < 2) { delete h; return EMC2_ERR_CUDA; }
+
     // Plan the slab: everything the stage calls need, allocated once.
     SlabPlan plan;
-    size_t o_store[2], o_summary[2], o_prefix[2], o_covf[2], o_sums[2], o_arr[2], o_cl[2], o_bs[2], o_bo[2], o_ovf[2][4], o_tot[2];
+    size_t o_store[2], o_flag[2], o_acc[2], o_ovf[2][5], o_tot[2];
     for (int s = 0; s < 2; ++s) {
         ScaleDev& d = h->scale[s];
         const emc2_grid_t& g = c.grid[s];
@@ -146,24 +150,18 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         d.cells = (uint32_t)((uint64_t)g.dims[0] * g.dims[1] * g.dims[2]);
         const uint64_t total_cells = (uint64_t)d.cells * c.max_batch;
         d.mode = total_cells <= (uint64_t)kMaxTableCells ? MODE_TABLE : MODE_BITMAP;
-        const uint64_t per_chunk = d.mode == MODE_BITMAP ? 256 : 8;
-        d.nchunks = (uint32_t)((total_cells + per_chunk - 1) / per_chunk);
-        d.nsumwords = (d.nchunks + 31) / 32;
-        d.scan_blocks = (int)((d.nchunks + kThreads - 1) / kThreads);
+        const uint64_t per_tile = d.mode == MODE_BITMAP ? kBitmapTileCells : kTableTileCells;
+        d.ntiles = (uint32_t)((total_cells + per_tile - 1) / per_tile);
         d.max_ovf = d.cap > 0 ? (uint32_t)(maxpts / ((size_t)d.cap + 1) + 1) : 0;
-        o_store[s] = plan.take((size_t)d.nsumwords * 32 * kChunkBytes);
-        o_summary[s] = plan.take((size_t)d.nsumwords * 4);
-        o_prefix[s] = plan.take((size_t)d.nsumwords * 32 * 4);
-        o_covf[s] = d.cap > 0 ? plan.take((size_t)d.nsumwords * 32 * 4) : 0;
-        o_sums[s] = plan.take(maxpts * c.point_floats * sizeof(double));
-        o_arr[s] = plan.take(maxpts * sizeof(int));
-        o_cl[s] = plan.take(maxpts * sizeof(uint32_t));
-        o_bs[s] = plan.take((size_t)d.scan_blocks * 3 * sizeof(int));
-        o_bo[s] = plan.take((size_t)d.scan_blocks * 3 * sizeof(int));
+        o_store[s] = plan.take((size_t)d.ntiles * kThreads * 32);
+        o_flag[s] = plan.take((size_t)d.ntiles * sizeof(uint32_t));
+        o_acc[s] = plan.take(maxpts * 2 * sizeof(float4));
         for (int k = 0; k < 3; ++k) o_ovf[s][k] = d.cap > 0 ? plan.take((size_t)d.max_ovf * sizeof(int)) : 0;
         o_ovf[s][3] = d.cap > 0 ? plan.take(maxpts * sizeof(int)) : 0;
+        o_ovf[s][4] = d.cap > 0 ? plan.take((size_t)d.max_ovf * kCursorStride * sizeof(int)) : 0;
         o_tot[s] = plan.take(4 * sizeof(int));
     }
+    const size_t o_part = plan.take((size_t)h->scan_blocks * 3 * sizeof(int));
     h->max_tiles = (c.max_points + kTile - 1) / kTile;
     const size_t tile_ints = (size_t)c.max_batch * h->max_tiles * c.num_experts;
     const size_t o_tc = plan.take(tile_ints * sizeof(int));
@@ -173,28 +171,23 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     h->slab_bytes = plan.off;
     cudaError_t e = cudaMalloc(&h->slab, h->slab_bytes);
     if (e != cudaSuccess) { h->slab = nullptr; delete h; return EMC2_ERR_CUDA; }
-    // The voxel stores, summaries, sums and arrival counters must be all-zero between calls;
-    // every call restores that.
+    // The voxel stores must be all-zero between calls; every call restores that.
     e = cudaMemset(h->slab, 0, h->slab_bytes);
     if (e != cudaSuccess) { cudaFree(h->slab); delete h; return EMC2_ERR_CUDA; }
     char* base = static_cast<char*>(h->slab);
     for (int s = 0; s < 2; ++s) {
         ScaleDev& d = h->scale[s];
         d.store = reinterpret_cast<uint32_t*>(base + o_store[s]);
-        d.summary = reinterpret_cast<uint32_t*>(base + o_summary[s]);
-        d.chunk_prefix = reinterpret_cast<uint32_t*>(base + o_prefix[s]);
-        d.chunk_ovf = d.cap > 0 ? reinterpret_cast<uint32_t*>(base + o_covf[s]) : nullptr;
-        d.sums = reinterpret_cast<double*>(base + o_sums[s]);
-        d.arrivals = reinterpret_cast<int*>(base + o_arr[s]);
-        d.cell_list = reinterpret_cast<uint32_t*>(base + o_cl[s]);
-        d.blk_sums = reinterpret_cast<int*>(base + o_bs[s]);
-        d.blk_offs = reinterpret_cast<int*>(base + o_bo[s]);
+        d.tile_flag = reinterpret_cast<uint32_t*>(base + o_flag[s]);
+        d.acc = reinterpret_cast<float4*>(base + o_acc[s]);
         d.ovf_off = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][0]) : nullptr;
-        d.ovf_cursor = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][1]) : nullptr;
-        d.ovf_vox = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][2]) : nullptr;
+        d.ovf_vox = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][1]) : nullptr;
+        d.ovf_cell = d.cap > 0 ? reinterpret_cast<uint32_t*>(base + o_ovf[s][2]) : nullptr;
         d.ovf_list = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][3]) : nullptr;
+        d.ovf_cursor = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][4]) : nullptr;
         d.totals = reinterpret_cast<int*>(base + o_tot[s]);
     }
+    h->d_scan_part = reinterpret_cast<int*>(base + o_part);
     h->d_tile_counts = reinterpret_cast<int*>(base + o_tc);
     h->d_tile_base = reinterpret_cast<int*>(base + o_tb);
     h->d_status = reinterpret_cast<int*>(base + o_status);

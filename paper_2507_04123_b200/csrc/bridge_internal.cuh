@@ -12,17 +12,16 @@ namespace emc2 {
 
 constexpr int kTile = 256;           // points per CTA tile in the per-point kernels
 constexpr int kThreads = 256;
-constexpr int kChunkBytes = 32;      // one L2 sector: 256 bitmap cells or 8 table cells
-constexpr int kMaxTableCells = 1 << 26;  // direct count table up to 64 Mi cells per batch
+constexpr int kBitmapTileCells = kThreads * 4 * 32;  // a bitmap tile: 256 sectors of four {bits, rank} pairs
+constexpr int kTableTileCells = kThreads * 2;         // a table tile: 256 sectors of two cell records
+constexpr int kMaxTableCells = 1 << 24;  // per-cell records up to 16 Mi cells per batch (256 MB)
+constexpr int kCursorStride = 8;         // ints between list cursors: one 32-byte sector each
 
 // Kernel kinds, for the launch counters and the optional event timing.
 enum KernelKind {
     K_VOX_MARK = 0,
-    K_VOX_REDUCE,
-    K_VOX_BLOCKSCAN,
-    K_VOX_EMIT,
+    K_VOX_SCAN,
     K_VOX_ACCUM,
-    K_VOX_OVERFLOW,
     K_VOX_FINALIZE,
     K_PROJECT_GATHER,
     K_ROUTE_HIST,
@@ -41,24 +40,18 @@ struct ScaleDev {
     int cap;                // 0 = none
     int mode;               // ScaleMode
     uint32_t cells;         // cells per frame
-    uint32_t nchunks;       // 32-byte chunks of `store` for the largest batch
-    uint32_t nsumwords;     // 32-bit words of `summary`
-    uint32_t max_ovf;       // most voxels that can exceed the cap
-    uint32_t* store;        // bitmap words, or int32 counts
-    uint32_t* summary;      // one bit per chunk: chunk has an occupied cell
-    uint32_t* chunk_prefix; // voxels before the chunk (valid for flagged chunks)
-    uint32_t* chunk_ovf;    // overflowing voxels before the chunk (capped scales)
-    double* sums;           // [max voxels, C] fp64 sums of all but the first point; zero between calls
-    int* arrivals;          // [max voxels] points accumulated so far; zero between calls
-    uint32_t* cell_list;    // [max voxels] cell id of each unique voxel
-    int* blk_sums;          // [scan blocks, 3]
-    int* blk_offs;          // [scan blocks, 3]
-    int* ovf_off;           // per overflowing voxel j: start of its points in ovf_list
-    int* ovf_cursor;        // per overflowing voxel j: points appended so far
-    int* ovf_vox;           // per overflowing voxel j: its row m in the unique list
-    int* ovf_list;          // global point indices of the points in overflowing voxels
-    int* totals;            // [0] voxels, [1] overflowing voxels, [2] overflowing points
-    int scan_blocks;
+    uint32_t ntiles;        // 8 KB tiles of `store` for the largest batch
+    uint32_t max_ovf;       // most cells that can exceed the cap
+    uint32_t* store;        // bitmap: {bits, rank} per 32 cells; table: {count, rank, over-cap rank, -} per cell;
+                            // bits / counts are zero between calls
+    uint32_t* tile_flag;    // [ntiles] tile holds an occupied cell (rewritten by every call)
+    float4* acc;            // [max voxels][2] per-voxel accumulators
+    int* ovf_off;           // per cell over the cap j: start of its points in ovf_list
+    int* ovf_cursor;        // per cell over the cap j: points appended so far, at [j * kCursorStride]
+    uint32_t* ovf_cell;     // per cell over the cap j: its cell id
+    int* ovf_vox;           // per cell over the cap j: its row m in the unique list
+    int* ovf_list;          // global point indices of the points in cells over the cap
+    int* totals;            // [0] voxels, [1] cells over the cap, [2] points in cells over the cap
 };
 
 struct ProfRec {
@@ -77,6 +70,8 @@ struct emc2_bridge {
     int* d_status = nullptr;       // sticky device status word
     int* d_tile_counts = nullptr;  // [B, tiles per frame, E]
     int* d_tile_base = nullptr;    // same shape, exclusive bases
+    int* d_scan_part = nullptr;    // [scan_blocks][3] per-CTA totals of the voxel rank scan
+    int scan_blocks = 0;           // CTAs of the cooperative rank scan (all co-resident)
     int max_tiles = 0;
     int last_cuda_error = 0;
     bool profiling = false;
@@ -100,6 +95,8 @@ struct LaunchScope {
 
 int check_cuda(emc2_bridge* h, cudaError_t e);
 
+// Largest cooperative grid of the voxel rank scan on the current device (0: unsupported).
+int voxel_scan_max_blocks();
 int launch_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* const d_coords[2],
                     int32_t* const d_counts[2], float* const d_mean[2], int32_t* const d_point_voxel[2],
                     const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st);

@@ -1,18 +1,37 @@
 // Stage 1 of the bridge: two-scale voxelization, dedup in canonical order, per-voxel counts
 // and means, BEV scatter (Sec. 3.1 preprocessing; BEV for the 2D expert of Sec. 3.3).
 //
-// Dedup is direct-addressed, with no sort: every cell of the batch owns one bit (large grids)
-// or one 32-bit counter (grids small enough for a count table).  The store is cut into
-// 32-byte chunks (one L2 sector: 256 bitmap cells or 8 counters); a summary bitmap holds one
-// bit per chunk.  Points mark their cell with one atomic; a prefix sum over the occupied
-// chunks (the parallel prefix-sum index search of Sec. 3.6) then gives every occupied cell its
-// rank in ascending (b, z, y, x) order, which is the canonical voxel order.  A second pass
-// over the points looks the rank up (one sector load plus popcounts) and accumulates: the
-// first point to reach a voxel stores its values straight into the output row, later points
-// add into fp64 scratch sums.  A per-voxel pass writes coordinates, counts, means and the BEV
-// image and puts every scratch word it used back to zero, so the cost of a call follows the
-// occupied cells, not the grid volume.
+// Dedup is direct-addressed, with no sort and no hash probing.  Large grids keep one bit per
+// cell: the store is an array of {32 cell bits, rank} pairs in cell order.  Grids small enough
+// keep one record {point count, rank, rank among cells over the cap, -} per cell.  "Rank" is
+// the number of occupied cells before this word / cell in ascending (b, z, y, x) order, which
+// is the canonical voxel order, so a point finds its voxel row with ONE 8- or 16-byte load plus
+// a popcount, and no sort is ever needed.
+//
+//   vox_mark      every point marks its two cells with one fire-and-forget reduction each;
+//                 the same launch zeroes the BEV image.
+//   vox_scan      one cooperative launch: counts per 8 KB tile of the store, grid barrier,
+//                 then the exclusive prefix sums (the parallel prefix-sum index search of
+//                 Sec. 3.6) are written into the rank fields; accumulators are cleared and the
+//                 bookkeeping of cells over the cap is laid out.
+//   vox_accum     every point looks its rank up, writes point_voxel and adds itself to its
+//                 voxels' accumulators with two fp32 vector reductions (offsets from the cell
+//                 corner, the other channels, the count).
+//                 Points of cells over the cap go to per-cell lists instead.
+//   vox_finalize  walks the occupied tiles of the store: one thread per word / cell writes
+//                 coordinates, count, mean and the BEV cell of its voxels and puts the store
+//                 back to zero; in the same launch one warp per cell over the cap keeps the
+//                 `cap` lowest point indices (keep-first-by-index) and sums them in fp64.
+//
+// Writes and reductions that land in one 32-byte sector are served one after another by the
+// L2 (about 10 ns each on B200), so nothing here funnels many points into a shared flag or
+// counter: the only contended words are the cells themselves.  The cost of a call follows the
+// occupied tiles, not the grid volume, except for one streaming read of the store.
+#include <cooperative_groups.h>
+
 #include "bridge_internal.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace emc2 {
 namespace {
@@ -20,9 +39,30 @@ namespace {
 constexpr int kStatusCapacity = 1;
 constexpr int kPtsPerThread = 4;                      // independent points per thread (memory-level parallelism)
 constexpr int kBigTile = kThreads * kPtsPerThread;    // points per CTA in the two per-point passes
+constexpr int kOvfBlocks = 296;                       // CTAs of vox_finalize that serve cells over the cap
 
-// ------------------------------------------------------------------ block-level helpers
-// Exclusive scan of three counters across the CTA; returns CTA totals in tot[].
+// Where a point's cell sits in the unique list.
+struct Slot {
+    int m;      // row in the unique list, -1 if the point is outside the grid
+    int j;      // rank among cells over the cap, -1 if the cell is not over it
+};
+
+__device__ __forceinline__ Slot slot_of(const ScaleDev& g, uint32_t cell) {
+    Slot s;
+    s.m = -1; s.j = -1;
+    if (cell == 0xFFFFFFFFu) return s;
+    if (g.mode == MODE_BITMAP) {
+        const uint2 pr = *reinterpret_cast<const uint2*>(g.store + 2 * (size_t)(cell >> 5));
+        s.m = (int)(pr.y + __popc(pr.x & ((1u << (cell & 31u)) - 1u)));
+    } else {
+        const uint4 q = *reinterpret_cast<const uint4*>(g.store + 4 * (size_t)cell);
+        s.m = (int)q.y;
+        if (g.cap > 0 && (int)q.x > g.cap) s.j = (int)q.z;
+    }
+    return s;
+}
+
+// Exclusive scan of three counters across the CTA; CTA totals in tot[].
 __device__ __forceinline__ void block_excl_scan3(int v[3], int tot[3], int (*sm)[3]) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
     int inc[3];
@@ -31,7 +71,7 @@ __device__ __forceinline__ void block_excl_scan3(int v[3], int tot[3], int (*sm)
         int x = v[k];
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
-            int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
+            const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
             if (lane >= d) x += y;
         }
         inc[k] = x;
@@ -44,7 +84,7 @@ __device__ __forceinline__ void block_excl_scan3(int v[3], int tot[3], int (*sm)
             int x = lane < nwarp ? sm[lane][k] : 0;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
-                int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
+                const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
                 if (lane >= d) x += y;
             }
             if (lane < nwarp) sm[lane][k] = x;   // inclusive over warps
@@ -53,81 +93,33 @@ __device__ __forceinline__ void block_excl_scan3(int v[3], int tot[3], int (*sm)
     __syncthreads();
 #pragma unroll
     for (int k = 0; k < 3; ++k) {
-        int wbase = warp ? sm[warp - 1][k] : 0;
+        const int wbase = warp ? sm[warp - 1][k] : 0;
         tot[k] = sm[nwarp - 1][k];
         v[k] = wbase + inc[k] - v[k];
     }
     __syncthreads();
 }
 
-struct Chunk {
-    uint32_t w[8];
-};
-
-__device__ __forceinline__ Chunk load_chunk(const uint32_t* store, uint32_t chunk) {
-    const uint4* p = reinterpret_cast<const uint4*>(store + (size_t)chunk * 8);
-    uint4 a = p[0], b = p[1];
-    Chunk c;
-    c.w[0] = a.x; c.w[1] = a.y; c.w[2] = a.z; c.w[3] = a.w;
-    c.w[4] = b.x; c.w[5] = b.y; c.w[6] = b.z; c.w[7] = b.w;
-    return c;
-}
-
-// Occupied cells, overflowing cells and points in overflowing cells of one chunk.
-__device__ __forceinline__ void chunk_stats(const ScaleDev& g, const Chunk& c, int s[3]) {
-    if (g.mode == MODE_BITMAP) {
+// Sum of three counters across the CTA, result valid in every thread.
+__device__ __forceinline__ void block_sum3(int v[3], int (*sm)[3]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) s[0] += __popc(c.w[i]);
-    } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            int n = (int)c.w[i];
-            s[0] += n > 0;
-            if (g.cap > 0 && n > g.cap) { s[1] += 1; s[2] += n; }
-        }
+    for (int k = 0; k < 3; ++k) {
+        const int x = warp_sum(v[k]);
+        if (lane == 0) sm[warp][k] = x;
     }
-}
-
-// Where a point's cell sits in the unique list.
-struct Slot {
-    int m;      // row in the unique list, -1 if the point is outside the grid
-    int n;      // points in the cell (count table only)
-    int j;      // rank among cells that exceed the cap, -1 if the cell does not
-};
-
-__device__ __forceinline__ Slot slot_of(const ScaleDev& g, uint32_t cell) {
-    Slot s;
-    s.m = -1; s.n = 0; s.j = -1;
-    if (cell == 0xFFFFFFFFu) return s;
-    if (g.mode == MODE_BITMAP) {
-        const uint32_t chunk = cell >> 8, w = (cell >> 5) & 7u, bit = cell & 31u;
-        const Chunk c = load_chunk(g.store, chunk);
-        uint32_t r = g.chunk_prefix[chunk];
+    __syncthreads();
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            uint32_t mask = i < (int)w ? 0xFFFFFFFFu : (i == (int)w ? ((1u << bit) - 1u) : 0u);
-            r += __popc(c.w[i] & mask);
-        }
-        s.m = (int)r;
-    } else {
-        const uint32_t chunk = cell >> 3, w = cell & 7u;
-        const Chunk c = load_chunk(g.store, chunk);
-        uint32_t r = g.chunk_prefix[chunk];
-        int before_ovf = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            r += (i < (int)w && c.w[i] != 0u) ? 1u : 0u;
-            before_ovf += (i < (int)w && g.cap > 0 && (int)c.w[i] > g.cap) ? 1 : 0;
-        }
-        int n = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) n = i == (int)w ? (int)c.w[i] : n;   // no dynamic register indexing
-        s.m = (int)r;
-        s.n = n;
-        if (g.cap > 0 && n > g.cap) s.j = (int)g.chunk_ovf[chunk] + before_ovf;
+    for (int k = 0; k < 3; ++k) {
+        int x = 0;
+        for (int w = 0; w < nwarp; ++w) x += sm[w][k];
+        v[k] = x;
     }
-    return s;
+    __syncthreads();
 }
+
+// Lower corner of cell i along one axis; both per-point and per-voxel code use this value.
+__device__ __forceinline__ float cell_corner(float mn, float vs, int i) { return __fmaf_rn((float)i, vs, mn); }
 
 // ------------------------------------------------------------------ pass 1: mark cells
 template <int C>
@@ -146,42 +138,22 @@ vox_mark_kernel(const float* __restrict__ pts, long long total, int N, ScaleDev 
     if (npts <= 0) return;
     load_tile_f32(pts + g0 * C, npts * C, sp);
     __syncthreads();
-    uint32_t cell[2][kPtsPerThread];
+    const int b0 = (int)(g0 / N);
+    const int i0 = (int)(g0 - (long long)b0 * N);        // index of the tile's first point in frame b0
 #pragma unroll
     for (int i = 0; i < kPtsPerThread; ++i) {
         const int t = threadIdx.x + i * kThreads;
-        cell[0][i] = cell[1][i] = 0xFFFFFFFFu;
-        if (t < npts) {
-            const float x = sp[t * C], y = sp[t * C + 1], z = sp[t * C + 2];
-            const int b = (int)((g0 + t) / N);
-            cell[0][i] = cell_of(s0, x, y, z, b);
-            cell[1][i] = cell_of(s1, x, y, z, b);
-        }
-    }
-    // All marking atomics are issued before any result is consumed.
-    uint32_t old[2][kPtsPerThread];
+        if (t >= npts) continue;
+        const float x = sp[t * C], y = sp[t * C + 1], z = sp[t * C + 2];
+        const int b = b0 + (i0 + t) / N;
 #pragma unroll
-    for (int sc = 0; sc < 2; ++sc) {
-        const ScaleDev& g = sc ? s1 : s0;
-#pragma unroll
-        for (int i = 0; i < kPtsPerThread; ++i) {
-            const uint32_t c = cell[sc][i];
-            old[sc][i] = 1u;
-            if (c != 0xFFFFFFFFu)
-                old[sc][i] = g.mode == MODE_BITMAP ? atomicOr(&g.store[c >> 5], 1u << (c & 31u))
-                                                   : atomicAdd(&g.store[c], 1u);
-        }
-    }
-#pragma unroll
-    for (int sc = 0; sc < 2; ++sc) {
-        const ScaleDev& g = sc ? s1 : s0;
-        const int shift = g.mode == MODE_BITMAP ? 8 : 3;
-#pragma unroll
-        for (int i = 0; i < kPtsPerThread; ++i) {
-            if (old[sc][i] == 0u) {              // first touch of a word / cell: flag its chunk
-                const uint32_t chunk = cell[sc][i] >> shift;
-                atomicOr(&g.summary[chunk >> 5], 1u << (chunk & 31u));
-            }
+        for (int sc = 0; sc < 2; ++sc) {
+            const ScaleDev& g = sc ? s1 : s0;
+            const uint32_t cell = cell_of(g, x, y, z, b);
+            if (cell == 0xFFFFFFFFu) continue;
+            // Results unused: these compile to reductions, which the thread does not wait for.
+            if (g.mode == MODE_BITMAP) atomicOr(&g.store[2 * (size_t)(cell >> 5)], 1u << (cell & 31u));
+            else atomicAdd(&g.store[4 * (size_t)cell], 1u);
         }
     }
 }
@@ -189,118 +161,132 @@ vox_mark_kernel(const float* __restrict__ pts, long long total, int N, ScaleDev 
 // ------------------------------------------------------------------ pass 2: ranks
 struct ScanArgs {
     ScaleDev s[2];
-    uint32_t nchunks_used[2];   // chunks covering this call's B frames
+    uint32_t ntiles_used[2];    // tiles covering this call's B frames
     int capacity[2];
     int32_t* num_voxels;
     int* status;
+    int* part;                  // [gridDim.x][3] per-CTA totals
+    int g0;                     // CTAs [0, g0) serve scale 0, the rest scale 1
 };
 
-__device__ __forceinline__ bool chunk_flagged(const ScaleDev& g, uint32_t chunk, uint32_t nchunks) {
-    return chunk < nchunks && ((g.summary[chunk >> 5] >> (chunk & 31u)) & 1u);
+// One thread owns one 32-byte sector of the store: four {bits, rank} pairs or two cell records.
+struct Sector {
+    uint4 a, b;
+};
+
+__device__ __forceinline__ Sector load_sector(const uint32_t* store, uint32_t tile, int t) {
+    const uint4* p = reinterpret_cast<const uint4*>(store) + ((size_t)tile * kThreads + t) * 2;
+    Sector s;
+    s.a = p[0];
+    s.b = p[1];
+    return s;
 }
 
-// One thread per chunk; per-CTA totals of (voxels, overflowing voxels, overflowing points).
-__global__ void __launch_bounds__(kThreads) vox_reduce_kernel(ScanArgs a) {
+// Occupied cells, cells over the cap and points in cells over the cap of one sector.
+__device__ __forceinline__ void sector_stats(const ScaleDev& g, const Sector& s, int v[3]) {
+    if (g.mode == MODE_BITMAP) {
+        v[0] += __popc(s.a.x) + __popc(s.a.z) + __popc(s.b.x) + __popc(s.b.z);
+    } else {
+        const int n0 = (int)s.a.x, n1 = (int)s.b.x;
+        v[0] += (n0 > 0) + (n1 > 0);
+        if (g.cap > 0) {
+            if (n0 > g.cap) { v[1] += 1; v[2] += n0; }
+            if (n1 > g.cap) { v[1] += 1; v[2] += n1; }
+        }
+    }
+}
+
+// Cooperative launch.  Every CTA owns a contiguous range of tiles of one scale.  Phase 1 counts
+// and notes which tiles hold anything; after the grid barrier every CTA adds up the totals of
+// the CTAs before it; phase 2 walks the occupied tiles again and writes the ranks.
+__global__ void __launch_bounds__(kThreads) vox_scan_kernel(ScanArgs a) {
     __shared__ int sm[kThreads / 32][3];
-    const int sc = blockIdx.y;
+    cg::grid_group grid = cg::this_grid();
+    const int sc = (int)blockIdx.x >= a.g0 ? 1 : 0;
+    const int first = sc ? a.g0 : 0;
+    const int cta = (int)blockIdx.x - first;
+    const int ncta = sc ? (int)gridDim.x - a.g0 : a.g0;
     const ScaleDev& g = a.s[sc];
-    const uint32_t nblk = (a.nchunks_used[sc] + kThreads - 1) / kThreads;
-    if (blockIdx.x >= nblk) return;
-    const uint32_t chunk = blockIdx.x * kThreads + threadIdx.x;
-    int s[3] = {0, 0, 0};
-    if (chunk_flagged(g, chunk, a.nchunks_used[sc])) chunk_stats(g, load_chunk(g.store, chunk), s);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int k = 0; k < 3; ++k) {
-        int v = warp_sum(s[k]);
-        if (lane == 0) sm[warp][k] = v;
-    }
-    __syncthreads();
-    if (threadIdx.x < 3) {
-        int v = 0;
-        for (int w = 0; w < kThreads / 32; ++w) v += sm[w][threadIdx.x];
-        g.blk_sums[blockIdx.x * 3 + threadIdx.x] = v;
-    }
-}
+    const uint32_t ntiles = a.ntiles_used[sc];
+    const uint32_t per = (ntiles + (uint32_t)ncta - 1u) / (uint32_t)ncta;
+    const uint32_t lo = min(ntiles, (uint32_t)cta * per), hi = min(ntiles, lo + per);
+    const int t = threadIdx.x;
 
-// One CTA per scale: exclusive scan of the per-CTA sums (each thread owns a run of
-// consecutive entries, so one CTA-wide scan covers 1024 * run entries); totals, capacity check.
-__global__ void __launch_bounds__(1024) vox_blockscan_kernel(ScanArgs a) {
-    __shared__ int sm[32][3];
-    const int sc = blockIdx.x;
-    const ScaleDev& g = a.s[sc];
-    const int nblk = (int)((a.nchunks_used[sc] + kThreads - 1) / kThreads);
-    const int per = (nblk + (int)blockDim.x - 1) / (int)blockDim.x;
-    const int lo = min(nblk, (int)threadIdx.x * per), hi = min(nblk, lo + per);
-    int v[3] = {0, 0, 0}, tot[3];
-    for (int i = lo; i < hi; ++i) {
-        v[0] += g.blk_sums[i * 3]; v[1] += g.blk_sums[i * 3 + 1]; v[2] += g.blk_sums[i * 3 + 2];
+    int s[3] = {0, 0, 0};
+    for (uint32_t tile = lo; tile < hi; ++tile) {
+        const int before = s[0];
+        sector_stats(g, load_sector(g.store, tile, t), s);
+        const int any = __syncthreads_or(s[0] != before);
+        if (t == 0) g.tile_flag[tile] = (uint32_t)any;
     }
-    block_excl_scan3(v, tot, sm);
-    for (int i = lo; i < hi; ++i) {
-        g.blk_offs[i * 3] = v[0]; g.blk_offs[i * 3 + 1] = v[1]; g.blk_offs[i * 3 + 2] = v[2];
-        v[0] += g.blk_sums[i * 3]; v[1] += g.blk_sums[i * 3 + 1]; v[2] += g.blk_sums[i * 3 + 2];
+    block_sum3(s, sm);
+    if (t < 3) a.part[blockIdx.x * 3 + t] = s[t];
+    grid.sync();
+
+    // Totals of the CTAs before this one (same scale) and of the whole scale.
+    int base[3] = {0, 0, 0}, tot[3] = {0, 0, 0};
+    for (int c = t; c < ncta; c += kThreads) {
+        const int* p = a.part + (size_t)(first + c) * 3;
+        const int v0 = p[0], v1 = p[1], v2 = p[2];
+        tot[0] += v0; tot[1] += v1; tot[2] += v2;
+        if (c < cta) { base[0] += v0; base[1] += v1; base[2] += v2; }
     }
-    if (threadIdx.x == 0) {
+    block_sum3(base, sm);
+    block_sum3(tot, sm);
+    if (cta == 0 && t == 0) {
         g.totals[0] = tot[0]; g.totals[1] = tot[1]; g.totals[2] = tot[2];
         a.num_voxels[sc] = tot[0];
         if (tot[0] > a.capacity[sc]) atomicOr(a.status, kStatusCapacity);
     }
-}
-
-// One thread per chunk: rank of the chunk's first voxel, the cell id of every voxel (so that
-// later passes can run one thread per voxel), and the bookkeeping of cells over the cap.
-__global__ void __launch_bounds__(kThreads) vox_emit_kernel(ScanArgs a) {
-    __shared__ int sm[kThreads / 32][3];
-    const int sc = blockIdx.y;
-    const ScaleDev& g = a.s[sc];
-    const uint32_t nblk = (a.nchunks_used[sc] + kThreads - 1) / kThreads;
-    if (blockIdx.x >= nblk) return;
-    const uint32_t chunk = blockIdx.x * kThreads + threadIdx.x;
-    const bool flagged = chunk_flagged(g, chunk, a.nchunks_used[sc]);
-    Chunk c;
-    int run[3] = {0, 0, 0}, tot[3];
-    if (flagged) {
-        c = load_chunk(g.store, chunk);
-        chunk_stats(g, c, run);
+    // Clear the accumulators of the voxels found (two 16-byte halves per voxel).
+    {
+        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        const size_t n = 2 * (size_t)tot[0];
+        for (size_t i = (size_t)cta * kThreads + t; i < n; i += (size_t)ncta * kThreads) g.acc[i] = z;
     }
-    block_excl_scan3(run, tot, sm);       // run[] = exclusive offsets inside the CTA
-    if (!flagged) return;
-    int m = g.blk_offs[blockIdx.x * 3] + run[0];
-    g.chunk_prefix[chunk] = (uint32_t)m;
-    if (g.mode == MODE_BITMAP) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            uint32_t word = c.w[i];
-            while (word) {
-                const int bit = __ffs(word) - 1;
-                word &= word - 1;
-                g.cell_list[m++] = chunk * 256u + i * 32u + bit;
+
+    int carry[3] = {base[0], base[1], base[2]};
+    for (uint32_t tile = lo; tile < hi; ++tile) {
+        if (!g.tile_flag[tile]) continue;         // written by this CTA in phase 1; same for all threads
+        Sector x = load_sector(g.store, tile, t);
+        int run[3] = {0, 0, 0}, ttot[3];
+        sector_stats(g, x, run);
+        const bool mine = run[0] > 0;
+        block_excl_scan3(run, ttot, sm);          // run[] = exclusive offsets inside the tile
+        if (mine) {
+            int m = carry[0] + run[0];
+            if (g.mode == MODE_BITMAP) {
+                x.a.y = (uint32_t)m; m += __popc(x.a.x);
+                x.a.w = (uint32_t)m; m += __popc(x.a.z);
+                x.b.y = (uint32_t)m; m += __popc(x.b.x);
+                x.b.w = (uint32_t)m;
+            } else {
+                int j = carry[1] + run[1], off = carry[2] + run[2];
+                const uint32_t cell0 = (tile * (uint32_t)kThreads + t) * 2u;
+                x.a.y = (uint32_t)m; x.a.z = (uint32_t)j;
+                const int n0 = (int)x.a.x, n1 = (int)x.b.x;
+                if (g.cap > 0 && n0 > g.cap) {
+                    g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+                    j += 1; off += n0;
+                }
+                m += n0 > 0;
+                x.b.y = (uint32_t)m; x.b.z = (uint32_t)j;
+                if (g.cap > 0 && n1 > g.cap) {
+                    g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0 + 1u; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+                }
             }
+            uint4* p = reinterpret_cast<uint4*>(g.store) + ((size_t)tile * kThreads + t) * 2;
+            p[0] = x.a;
+            p[1] = x.b;
         }
-    } else {
-        int j = g.blk_offs[blockIdx.x * 3 + 1] + run[1];
-        int off = g.blk_offs[blockIdx.x * 3 + 2] + run[2];
-        if (g.cap > 0) g.chunk_ovf[chunk] = (uint32_t)j;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int n = (int)c.w[i];
-            if (n == 0) continue;
-            if (g.cap > 0 && n > g.cap) {
-                g.ovf_vox[j] = m;
-                g.ovf_off[j] = off;
-                g.ovf_cursor[j] = 0;
-                j += 1;
-                off += n;
-            }
-            g.cell_list[m++] = chunk * 8u + i;
-        }
+        carry[0] += ttot[0]; carry[1] += ttot[1]; carry[2] += ttot[2];
     }
 }
 
 // ------------------------------------------------------------------ pass 3: accumulate
 struct AccumArgs {
     ScaleDev s[2];
+    uint32_t ntiles_used[2];
     int capacity[2];
     int32_t* coords[2];
     int32_t* counts[2];
@@ -309,11 +295,10 @@ struct AccumArgs {
     float* bev;
 };
 
-// The first point to arrive in a voxel stores its values in the output row; the others add
-// into the fp64 scratch row.  For a count table "first" is decided without an arrival
-// counter when the cell holds one point; otherwise an atomic counter elects it.  The kernel
-// runs in three phases so that a thread's memory operations overlap: (A) all rank lookups,
-// (B) all arrival / list-cursor atomics, (C) all stores and fp64 reductions.
+// Per-voxel accumulator, 32 bytes of fp32: {sum dx, sum dy, sum dz, sum ch3}, {sum ch4, count, -, -},
+// where d* are offsets from the cell's lower corner, so that those sums stay small.  Two vector
+// reductions per point and scale.  A sum of n terms carries a relative error of at most n * 2^-24
+// (far less in practice, since the roundings do not line up).
 template <int C>
 __global__ void __launch_bounds__(kThreads)
 vox_accum_kernel(const float* __restrict__ pts, long long total, int N, AccumArgs a) {
@@ -322,179 +307,229 @@ vox_accum_kernel(const float* __restrict__ pts, long long total, int N, AccumArg
     const int npts = (int)min((long long)kBigTile, total - g0);
     load_tile_f32(pts + g0 * C, npts * C, sp);
     __syncthreads();
+    const int b0 = (int)(g0 / N);
+    const int i0 = (int)(g0 - (long long)b0 * N);
+    // All rank lookups first, so that a thread has eight loads in flight.
     Slot slot[2][kPtsPerThread];
+    int cx[2][kPtsPerThread], cy[2][kPtsPerThread], cz[2][kPtsPerThread];
 #pragma unroll
     for (int i = 0; i < kPtsPerThread; ++i) {
         const int t = threadIdx.x + i * kThreads;
-        uint32_t c0 = 0xFFFFFFFFu, c1 = 0xFFFFFFFFu;
-        if (t < npts) {
-            const float x = sp[t * C], y = sp[t * C + 1], z = sp[t * C + 2];
-            const int b = (int)((g0 + t) / N);
-            c0 = cell_of(a.s[0], x, y, z, b);
-            c1 = cell_of(a.s[1], x, y, z, b);
-        }
-        slot[0][i] = slot_of(a.s[0], c0);
-        slot[1][i] = slot_of(a.s[1], c1);
-    }
-    // Phase B.  ticket >= 0: position in arrival order (0 = first); -1: nothing to do.
-    // For a cell over the cap the ticket is the slot in its overflow list.
-    int ticket[2][kPtsPerThread];
 #pragma unroll
-    for (int sc = 0; sc < 2; ++sc) {
-        const ScaleDev& g = a.s[sc];
-#pragma unroll
-        for (int i = 0; i < kPtsPerThread; ++i) {
-            const Slot s = slot[sc][i];
-            int tk = -1;
-            if (s.m >= 0) {
-                if (s.j >= 0) tk = atomicAdd(&g.ovf_cursor[s.j], 1);
-                else if (s.m < a.capacity[sc])
-                    tk = (g.mode == MODE_BITMAP || s.n > 1) ? atomicAdd(&g.arrivals[s.m], 1) : 0;
+        for (int sc = 0; sc < 2; ++sc) {
+            const ScaleDev& g = a.s[sc];
+            uint32_t cell = 0xFFFFFFFFu;
+            cx[sc][i] = cy[sc][i] = cz[sc][i] = 0;
+            if (t < npts) {
+                const float x = sp[t * C], y = sp[t * C + 1], z = sp[t * C + 2];
+                const int ix = axis_cell(x, g.mn[0], g.vs[0], g.dims[0]);
+                const int iy = axis_cell(y, g.mn[1], g.vs[1], g.dims[1]);
+                const int iz = axis_cell(z, g.mn[2], g.vs[2], g.dims[2]);
+                if ((ix | iy | iz) >= 0) {
+                    const int b = b0 + (i0 + t) / N;
+                    cell = (((uint32_t)b * g.dims[2] + iz) * g.dims[1] + iy) * g.dims[0] + ix;
+                    cx[sc][i] = ix; cy[sc][i] = iy; cz[sc][i] = iz;
+                }
             }
-            ticket[sc][i] = tk;
+            slot[sc][i] = slot_of(g, cell);
         }
     }
-    // Phase C.
 #pragma unroll
     for (int sc = 0; sc < 2; ++sc) {
         const ScaleDev& g = a.s[sc];
-        float* mean = a.mean[sc];
         int32_t* pv = a.point_voxel[sc];
 #pragma unroll
         for (int i = 0; i < kPtsPerThread; ++i) {
             const int t = threadIdx.x + i * kThreads;
             if (t >= npts) continue;
             const Slot s = slot[sc][i];
-            const int tk = ticket[sc][i];
             if (s.j >= 0) {
-                // Which of this voxel's points survive the cap is decided by vox_overflow_kernel,
-                // which also writes their point_voxel entries.
+                // Which of this cell's points survive the cap is decided per cell in
+                // vox_finalize_kernel, which also writes their point_voxel entries.
+                const int tk = atomicAdd(&g.ovf_cursor[(size_t)s.j * kCursorStride], 1);
                 g.ovf_list[g.ovf_off[s.j] + tk] = (int)(g0 + t);
                 continue;
             }
-            if (tk == 0) {
-#pragma unroll
-                for (int k = 0; k < C; ++k) mean[(size_t)s.m * C + k] = sp[t * C + k];
-            } else if (tk > 0) {
-#pragma unroll
-                for (int k = 0; k < C; ++k) atomicAdd(&g.sums[(size_t)s.m * C + k], (double)sp[t * C + k]);
-            }
             if (pv) pv[g0 + t] = s.m;
-        }
-    }
-}
-
-// One warp per overflowing voxel: keep the `cap` lowest point indices (keep-first-by-index),
-// sum them, and write point_voxel for all of the voxel's points.
-template <int C>
-__global__ void __launch_bounds__(kThreads)
-vox_overflow_kernel(const float* __restrict__ pts, long long total, AccumArgs a, int sc) {
-    const ScaleDev& g = a.s[sc];
-    const int lane = threadIdx.x & 31;
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int nwarps = (gridDim.x * blockDim.x) >> 5;
-    const int novf = g.totals[1];
-    int32_t* pv = a.point_voxel[sc];
-    for (int j = warp; j < novf; j += nwarps) {
-        const int m = g.ovf_vox[j];
-        const int n = g.ovf_cursor[j];
-        const int* list = g.ovf_list + g.ovf_off[j];
-        // Smallest t with #{v <= t} >= cap, by bisection on the index value.
-        long long lo = -1, hi = total - 1;
-        while (hi - lo > 1) {
-            const long long mid = lo + (hi - lo) / 2;
-            int c = 0;
-            for (int i = lane; i < n; i += 32) c += list[i] <= mid;
-            c = warp_sum(c);
-            if (c >= g.cap) hi = mid; else lo = mid;
-        }
-        double acc[C];
-#pragma unroll
-        for (int k = 0; k < C; ++k) acc[k] = 0.0;
-        for (int i = lane; i < n; i += 32) {
-            const int v = list[i];
-            const bool keep = v <= hi;
-            if (pv) pv[v] = keep ? m : -1;
-            if (keep) {
-#pragma unroll
-                for (int k = 0; k < C; ++k) acc[k] += (double)pts[(size_t)v * C + k];
-            }
-        }
-#pragma unroll
-        for (int k = 0; k < C; ++k) {
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) acc[k] += __shfl_xor_sync(0xFFFFFFFFu, acc[k], d);
-        }
-        if (lane == 0 && m < a.capacity[sc]) {
-            // Full sum in scratch; vox_finalize_kernel sees an overflowing cell and ignores
-            // the (unwritten) output row.
-#pragma unroll
-            for (int k = 0; k < C; ++k) g.sums[(size_t)m * C + k] = acc[k];
+            if (s.m < 0 || s.m >= a.capacity[sc]) continue;
+            const float dx = __fsub_rn(sp[t * C], cell_corner(g.mn[0], g.vs[0], cx[sc][i]));
+            const float dy = __fsub_rn(sp[t * C + 1], cell_corner(g.mn[1], g.vs[1], cy[sc][i]));
+            const float dz = __fsub_rn(sp[t * C + 2], cell_corner(g.mn[2], g.vs[2], cz[sc][i]));
+            float4* row = g.acc + 2 * (size_t)s.m;
+            atomicAdd(row, make_float4(dx, dy, dz, sp[t * C + 3]));
+            atomicAdd(reinterpret_cast<float2*>(row + 1), make_float2(C > 4 ? sp[t * C + 4] : 0.0f, 1.0f));
         }
     }
 }
 
 // ------------------------------------------------------------------ pass 4: rows, BEV, cleanup
-// One thread per voxel of either scale: coordinates from the cell id, count, mean (first
-// arrival + fp64 sums), BEV cell; then the voxel's scratch words go back to zero.  Loads are
-// grouped ahead of all stores so that they overlap.
+// Writes the output rows of voxel m, whose cell is `cell`, from its accumulator.
 template <int C>
-__global__ void __launch_bounds__(kThreads) vox_finalize_kernel(AccumArgs a) {
-    const int sc = blockIdx.y;
-    const ScaleDev& g = a.s[sc];
-    const int m = blockIdx.x * blockDim.x + threadIdx.x;
-    if (m >= g.totals[0]) return;
-    const bool bitmap = g.mode == MODE_BITMAP;
-    const bool in_cap = m < a.capacity[sc];
-    float* row = a.mean[sc] + (size_t)m * C;
-    double* srow = g.sums + (size_t)m * C;
-    // Level 1: everything addressed by m.
-    const uint32_t cell = g.cell_list[m];
-    const int arr = g.arrivals[m];
-    float first[C];
-#pragma unroll
-    for (int k = 0; k < C; ++k) first[k] = in_cap ? row[k] : 0.0f;
-    // Level 2: the cell's point count.
-    int n = bitmap ? arr : (int)g.store[cell];
-    const bool over = !bitmap && g.cap > 0 && n > g.cap;
-    if (over) n = g.cap;
-    // Level 3: fp64 sums, only where more than one point contributed.
-    const bool use_sums = in_cap && (n > 1 || over);
-    double s[C];
-#pragma unroll
-    for (int k = 0; k < C; ++k) s[k] = use_sums ? srow[k] : 0.0;
-
+__device__ __forceinline__ void write_voxel(const AccumArgs& a, int sc, const ScaleDev& g, int m, uint32_t cell,
+                                            bool over) {
+    if (m >= a.capacity[sc]) return;
+    const float4 a0 = g.acc[2 * (size_t)m];
+    const float4 a1 = g.acc[2 * (size_t)m + 1];
     uint32_t r = cell;
     const uint32_t x = r % g.dims[0]; r /= g.dims[0];
     const uint32_t y = r % g.dims[1]; r /= g.dims[1];
     const uint32_t z = r % g.dims[2]; r /= g.dims[2];
-    float mu[C];
-    const double cnt = (double)n;
-#pragma unroll
-    for (int k = 0; k < C; ++k)
-        mu[k] = use_sums ? (float)((over ? s[k] : s[k] + (double)first[k]) / cnt) : first[k];
-
-    // Stores: cleanup first (also for rows past the caller's capacity), then the outputs.
-    if (bitmap) {
-        g.store[cell >> 5] = 0u;                       // neighbours in the word write 0 as well
-        g.summary[cell >> 13] = 0u;
-    } else {
-        g.store[cell] = 0u;
-        g.summary[cell >> 8] = 0u;
-    }
-    if (arr) g.arrivals[m] = 0;
-    if (!in_cap) return;
-    if (use_sums) {
-#pragma unroll
-        for (int k = 0; k < C; ++k) { srow[k] = 0.0; row[k] = mu[k]; }
-    }
     reinterpret_cast<int4*>(a.coords[sc])[m] = make_int4((int)r, (int)z, (int)y, (int)x);
+    const int n = over ? g.cap : (int)a1.y;
     a.counts[sc][m] = n;
+    if (over) return;                             // mean and BEV cell come from the cell's warp
+    const double inv = 1.0 / (double)n;
+    float mu[C];
+    mu[0] = (float)((double)cell_corner(g.mn[0], g.vs[0], (int)x) + (double)a0.x * inv);
+    mu[1] = (float)((double)cell_corner(g.mn[1], g.vs[1], (int)y) + (double)a0.y * inv);
+    mu[2] = (float)((double)cell_corner(g.mn[2], g.vs[2], (int)z) + (double)a0.z * inv);
+    mu[3] = (float)((double)a0.w * inv);
+    if (C > 4) mu[4] = (float)((double)a1.x * inv);
+    float* row = a.mean[sc] + (size_t)m * C;
+#pragma unroll
+    for (int k = 0; k < C; ++k) row[k] = mu[k];
     if (sc == 1 && a.bev) {
         const size_t plane = (size_t)g.dims[1] * g.dims[0];
         float* dst = a.bev + (size_t)r * C * plane + (size_t)y * g.dims[0] + x;
 #pragma unroll
         for (int k = 0; k < C; ++k) dst[(size_t)k * plane] = mu[k];
+    }
+}
+
+// CTAs [0, ovf_blocks) serve cells over the cap, one warp per cell: the `cap` lowest point
+// indices are kept (keep-first-by-index), summed in fp64 and written as the voxel's mean; all of
+// the cell's points get their point_voxel entry.  The other CTAs stride over the occupied tiles
+// of both stores, one thread per word / cell: coordinates from the cell id, count, mean, BEV
+// cell; then the word / cell goes back to zero.
+template <int C>
+__global__ void __launch_bounds__(kThreads)
+vox_finalize_kernel(const float* __restrict__ pts, long long total, AccumArgs a, int ovf_blocks) {
+    if ((int)blockIdx.x < ovf_blocks) {
+        const int lane = threadIdx.x & 31;
+        const int warp = (blockIdx.x * kThreads + threadIdx.x) >> 5;
+        const int nwarps = (ovf_blocks * kThreads) >> 5;
+        for (int sc = 0; sc < 2; ++sc) {
+            const ScaleDev& g = a.s[sc];
+            if (g.cap <= 0) continue;
+            const int novf = g.totals[1];
+            int32_t* pv = a.point_voxel[sc];
+            for (int j = warp; j < novf; j += nwarps) {
+                const int m = g.ovf_vox[j];
+                const int n = g.ovf_cursor[(size_t)j * kCursorStride];
+                const int* list = g.ovf_list + g.ovf_off[j];
+                // Smallest index value v with #{list <= v} >= cap, by bisection on the value.
+                long long lo = -1, hi = total - 1;
+                while (hi - lo > 1) {
+                    const long long mid = lo + (hi - lo) / 2;
+                    int c = 0;
+                    for (int i = lane; i < n; i += 32) c += list[i] <= mid;
+                    c = warp_sum(c);
+                    if (c >= g.cap) hi = mid; else lo = mid;
+                }
+                double acc[C];
+#pragma unroll
+                for (int k = 0; k < C; ++k) acc[k] = 0.0;
+                for (int i = lane; i < n; i += 32) {
+                    const int v = list[i];
+                    const bool keep = v <= hi;
+                    if (pv) pv[v] = keep ? m : -1;
+                    if (keep) {
+#pragma unroll
+                        for (int k = 0; k < C; ++k) acc[k] += (double)pts[(size_t)v * C + k];
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < C; ++k) {
+#pragma unroll
+                    for (int d = 16; d > 0; d >>= 1) acc[k] += __shfl_xor_sync(0xFFFFFFFFu, acc[k], d);
+                }
+                if (lane < C && m < a.capacity[sc]) {
+                    double v = 0.0;
+#pragma unroll
+                    for (int k = 0; k < C; ++k) v = lane == k ? acc[k] : v;
+                    const float mu = (float)(v / (double)g.cap);
+                    a.mean[sc][(size_t)m * C + lane] = mu;
+                    if (sc == 1 && a.bev) {
+                        uint32_t r = g.ovf_cell[j];
+                        const uint32_t x = r % g.dims[0]; r /= g.dims[0];
+                        const uint32_t y = r % g.dims[1]; r /= g.dims[1];
+                        const size_t plane = (size_t)g.dims[1] * g.dims[0];
+                        a.bev[((size_t)r * C + lane) * plane + (size_t)y * g.dims[0] + x] = mu;
+                    }
+                }
+            }
+        }
+        return;
+    }
+    // Voxel rows.  Occupied cells are first compacted into a shared list (their rows are
+    // consecutive: the first one's rank plus the list position), then the list is worked off one
+    // voxel per thread, so that accumulator reads and row writes are dense whatever the
+    // occupancy pattern.
+    __shared__ uint32_t s_cell[kThreads * 32];    // cell ids of one round; table mode: bit 31 = over the cap
+    __shared__ int s_warp[kThreads / 32];
+    __shared__ int s_first;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t t0 = a.ntiles_used[0], t1 = a.ntiles_used[1];
+    const uint32_t nblk = gridDim.x - ovf_blocks;
+    for (uint32_t v = blockIdx.x - ovf_blocks; v < t0 + t1; v += nblk) {
+        const int sc = v >= t0 ? 1 : 0;
+        const uint32_t tile = sc ? v - t0 : v;
+        const ScaleDev& g = a.s[sc];
+        if (!g.tile_flag[tile]) continue;
+        const bool bitmap = g.mode == MODE_BITMAP;
+        const int rounds = bitmap ? 4 : 2;        // 1024 words or 512 cells per tile, 256 per round
+        for (int rnd = 0; rnd < rounds; ++rnd) {
+            uint32_t bits = 0u, id0 = 0u;
+            int rank = 0, k = 0;
+            if (bitmap) {
+                const uint32_t word = tile * (uint32_t)(4 * kThreads) + rnd * kThreads + threadIdx.x;
+                uint2* pp = reinterpret_cast<uint2*>(g.store) + word;
+                const uint2 pr = *pp;
+                if (pr.x) *pp = make_uint2(0u, 0u);
+                bits = pr.x; rank = (int)pr.y; id0 = word * 32u; k = __popc(bits);
+            } else {
+                const uint32_t cell = tile * (uint32_t)(2 * kThreads) + rnd * kThreads + threadIdx.x;
+                uint4* pq = reinterpret_cast<uint4*>(g.store) + cell;
+                const uint4 q = *pq;
+                if (q.x) *pq = make_uint4(0u, 0u, 0u, 0u);
+                bits = q.x ? 1u : 0u; rank = (int)q.y; k = (int)bits;
+                id0 = cell | ((g.cap > 0 && (int)q.x > g.cap) ? 0x80000000u : 0u);
+            }
+            // Exclusive position of this thread's cells in the round's list.
+            int inc = k;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= d) inc += y;
+            }
+            if (lane == 31) s_warp[warp] = inc;
+            __syncthreads();
+            int off = inc - k, total_k = 0;
+#pragma unroll
+            for (int w = 0; w < kThreads / 32; ++w) {
+                const int c = s_warp[w];
+                if (w < warp) off += c;
+                total_k += c;
+            }
+            if (k > 0 && off == 0) s_first = rank;   // exactly one thread owns the round's first voxel
+            if (bitmap) {
+                while (bits) {
+                    const int bit = __ffs(bits) - 1;
+                    bits &= bits - 1;
+                    s_cell[off++] = id0 + bit;
+                }
+            } else if (k) {
+                s_cell[off] = id0;
+            }
+            __syncthreads();
+            const int m0 = s_first;
+            for (int i = threadIdx.x; i < total_k; i += kThreads) {
+                const uint32_t c = s_cell[i];
+                if (bitmap) write_voxel<C>(a, sc, g, m0 + i, c, false);
+                else write_voxel<C>(a, sc, g, m0 + i, c & 0x7FFFFFFFu, (c >> 31) != 0u);
+            }
+            __syncthreads();
+        }
     }
 }
 
@@ -506,23 +541,28 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     const int ptiles = (int)((total + kBigTile - 1) / kBigTile);
     ScanArgs sa;
     AccumArgs aa;
-    int scan_blocks = 1;
+    bool any_cap = false;
     for (int s = 0; s < 2; ++s) {
         sa.s[s] = h->scale[s];
         aa.s[s] = h->scale[s];
         const uint64_t cells = (uint64_t)B * h->scale[s].cells;
-        const uint64_t per_chunk = h->scale[s].mode == MODE_BITMAP ? 256 : 8;
-        sa.nchunks_used[s] = (uint32_t)((cells + per_chunk - 1) / per_chunk);
-        scan_blocks = max(scan_blocks, (int)((sa.nchunks_used[s] + kThreads - 1) / kThreads));
+        const uint64_t per_tile = h->scale[s].mode == MODE_BITMAP ? kBitmapTileCells : kTableTileCells;
+        sa.ntiles_used[s] = aa.ntiles_used[s] = (uint32_t)((cells + per_tile - 1) / per_tile);
         sa.capacity[s] = aa.capacity[s] = capacity[s];
         aa.coords[s] = d_coords[s];
         aa.counts[s] = d_counts[s];
         aa.mean[s] = d_mean[s];
         aa.point_voxel[s] = d_point_voxel ? d_point_voxel[s] : nullptr;
+        any_cap = any_cap || h->scale[s].cap > 0;
     }
     sa.num_voxels = d_num_voxels;
     sa.status = h->d_status;
+    sa.part = h->d_scan_part;
     aa.bev = d_bev;
+    // Split the cooperative grid between the scales in proportion to their tile counts.
+    const int G = h->scan_blocks;
+    const double share = (double)sa.ntiles_used[0] / (double)((uint64_t)sa.ntiles_used[0] + sa.ntiles_used[1] + 1);
+    sa.g0 = min(G - 1, max(1, (int)(share * G)));
 
     const size_t bev_n = d_bev ? (size_t)B * C * h->scale[1].dims[1] * h->scale[1].dims[0] : 0;
     const bool bev_vec = (bev_n & 3) == 0;
@@ -538,39 +578,39 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
         }
     }
     {
-        LaunchScope ls(h, K_VOX_REDUCE, st);
-        vox_reduce_kernel<<<dim3(scan_blocks, 2), kThreads, 0, st>>>(sa);
-    }
-    {
-        LaunchScope ls(h, K_VOX_BLOCKSCAN, st);
-        vox_blockscan_kernel<<<2, 1024, 0, st>>>(sa);
-    }
-    {
-        LaunchScope ls(h, K_VOX_EMIT, st);
-        vox_emit_kernel<<<dim3(scan_blocks, 2), kThreads, 0, st>>>(sa);
+        LaunchScope ls(h, K_VOX_SCAN, st);
+        void* args[] = {&sa};
+        cudaError_t e = cudaLaunchCooperativeKernel((const void*)vox_scan_kernel, dim3(G), dim3(kThreads), args, 0, st);
+        if (e != cudaSuccess) return check_cuda(h, e);
     }
     if (total > 0) {
         {
             LaunchScope ls(h, K_VOX_ACCUM, st);
             vox_accum_kernel<C><<<ptiles, kThreads, 0, st>>>(d_points, total, N, aa);
         }
-        for (int s = 0; s < 2; ++s) {
-            if (h->scale[s].cap > 0) {
-                LaunchScope ls(h, K_VOX_OVERFLOW, st);
-                vox_overflow_kernel<C><<<148 * 2, kThreads, 0, st>>>(d_points, total, aa, s);
-            }
-        }
         {
-            // The number of voxels is only known on the device; it cannot exceed the points.
-            const int blocks = (int)((total + kThreads - 1) / kThreads);
+            // Which tiles hold voxels is only known on the device: a fixed grid strides over them.
+            const int ovf_blocks = any_cap ? kOvfBlocks : 0;
+            const uint32_t tiles = sa.ntiles_used[0] + sa.ntiles_used[1];
+            const int vox_blocks = (int)min((uint32_t)(148 * 8), max(tiles, 1u));
             LaunchScope ls(h, K_VOX_FINALIZE, st);
-            vox_finalize_kernel<C><<<dim3(blocks, 2), kThreads, 0, st>>>(aa);
+            vox_finalize_kernel<C><<<ovf_blocks + vox_blocks, kThreads, 0, st>>>(d_points, total, aa, ovf_blocks);
         }
     }
     return check_cuda(h, cudaGetLastError());
 }
 
 }  // namespace
+
+int voxel_scan_max_blocks() {
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, vox_scan_kernel, kThreads, 0) != cudaSuccess) return 0;
+    int coop = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return 0;
+    return sms * min(per_sm, 4);
+}
 
 int launch_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* const d_coords[2],
                     int32_t* const d_counts[2], float* const d_mean[2], int32_t* const d_point_voxel[2],
