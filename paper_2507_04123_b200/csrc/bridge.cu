@@ -141,27 +141,32 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
 
     // Plan the slab: everything the stage calls need, allocated once.
     SlabPlan plan;
-    size_t o_store[2], o_flag[2], o_acc[2], o_ovf[2][5], o_tot[2];
+    size_t o_store[2], o_flag[2], o_acc[2], o_cl[2], o_ovf[2][5], o_tot[2];
     for (int s = 0; s < 2; ++s) {
         ScaleDev& d = h->scale[s];
         const emc2_grid_t& g = c.grid[s];
-        for (int k = 0; k < 3; ++k) { d.mn[k] = g.min[k]; d.vs[k] = g.voxel[k]; d.dims[k] = g.dims[k]; }
+        for (int k = 0; k < 3; ++k) {
+            d.mn[k] = g.min[k]; d.vs[k] = g.voxel[k]; d.dims[k] = g.dims[k];
+            d.div[k] = make_fast_div((uint32_t)g.dims[k]);
+        }
         d.cap = g.max_points;
         d.cells = (uint32_t)((uint64_t)g.dims[0] * g.dims[1] * g.dims[2]);
         const uint64_t total_cells = (uint64_t)d.cells * c.max_batch;
         d.mode = total_cells <= (uint64_t)kMaxTableCells ? MODE_TABLE : MODE_BITMAP;
-        const uint64_t per_tile = d.mode == MODE_BITMAP ? kBitmapTileCells : kTableTileCells;
-        d.ntiles = (uint32_t)((total_cells + per_tile - 1) / per_tile);
+        const uint64_t per_group = d.mode == MODE_BITMAP ? kBitmapGroupCells : kTableGroupCells;
+        d.ngroups = (uint32_t)((total_cells + per_group - 1) / per_group);
         d.max_ovf = d.cap > 0 ? (uint32_t)(maxpts / ((size_t)d.cap + 1) + 1) : 0;
-        o_store[s] = plan.take((size_t)d.ntiles * kThreads * 32);
-        o_flag[s] = plan.take((size_t)d.ntiles * sizeof(uint32_t));
+        o_store[s] = plan.take((size_t)d.ngroups * 1024);
+        o_flag[s] = plan.take((size_t)d.ngroups * sizeof(int4));
         o_acc[s] = plan.take(maxpts * 2 * sizeof(float4));
+        o_cl[s] = plan.take(maxpts * sizeof(uint32_t));
         for (int k = 0; k < 3; ++k) o_ovf[s][k] = d.cap > 0 ? plan.take((size_t)d.max_ovf * sizeof(int)) : 0;
         o_ovf[s][3] = d.cap > 0 ? plan.take(maxpts * sizeof(int)) : 0;
         o_ovf[s][4] = d.cap > 0 ? plan.take((size_t)d.max_ovf * kCursorStride * sizeof(int)) : 0;
         o_tot[s] = plan.take(4 * sizeof(int));
     }
     const size_t o_part = plan.take((size_t)h->scan_blocks * 3 * sizeof(int));
+    const size_t o_wofs = plan.take((size_t)h->scan_blocks * (kThreads / 32) * 3 * sizeof(int));
     h->max_tiles = (c.max_points + kTile - 1) / kTile;
     const size_t tile_ints = (size_t)c.max_batch * h->max_tiles * c.num_experts;
     const size_t o_tc = plan.take(tile_ints * sizeof(int));
@@ -178,8 +183,9 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     for (int s = 0; s < 2; ++s) {
         ScaleDev& d = h->scale[s];
         d.store = reinterpret_cast<uint32_t*>(base + o_store[s]);
-        d.tile_flag = reinterpret_cast<uint32_t*>(base + o_flag[s]);
+        d.group_info = reinterpret_cast<int4*>(base + o_flag[s]);
         d.acc = reinterpret_cast<float4*>(base + o_acc[s]);
+        d.cell_list = reinterpret_cast<uint32_t*>(base + o_cl[s]);
         d.ovf_off = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][0]) : nullptr;
         d.ovf_vox = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][1]) : nullptr;
         d.ovf_cell = d.cap > 0 ? reinterpret_cast<uint32_t*>(base + o_ovf[s][2]) : nullptr;
@@ -188,6 +194,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         d.totals = reinterpret_cast<int*>(base + o_tot[s]);
     }
     h->d_scan_part = reinterpret_cast<int*>(base + o_part);
+    h->d_scan_warp_ofs = reinterpret_cast<int*>(base + o_wofs);
     h->d_tile_counts = reinterpret_cast<int*>(base + o_tc);
     h->d_tile_base = reinterpret_cast<int*>(base + o_tb);
     h->d_status = reinterpret_cast<int*>(base + o_status);

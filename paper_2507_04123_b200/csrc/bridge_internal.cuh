@@ -12,9 +12,10 @@ namespace emc2 {
 
 constexpr int kTile = 256;           // points per CTA tile in the per-point kernels
 constexpr int kThreads = 256;
-constexpr int kBitmapTileCells = kThreads * 4 * 32;  // a bitmap tile: 256 sectors of four {bits, rank} pairs
-constexpr int kTableTileCells = kThreads * 2;         // a table tile: 256 sectors of two cell records
+constexpr int kBitmapGroupCells = 32 * 4 * 32;  // a 1 KB bitmap group: 32 sectors of four {bits, rank} pairs
+constexpr int kTableGroupCells = 32 * 2;         // a 1 KB table group: 32 sectors of two cell records
 constexpr int kMaxTableCells = 1 << 24;  // per-cell records up to 16 Mi cells per batch (256 MB)
+constexpr int kMaxScanBlocks = 1024;     // CTAs of the cooperative rank scan, at most
 constexpr int kCursorStride = 8;         // ints between list cursors: one 32-byte sector each
 
 // Kernel kinds, for the launch counters and the optional event timing.
@@ -32,20 +33,48 @@ enum KernelKind {
 
 enum ScaleMode { MODE_BITMAP = 0, MODE_TABLE = 1 };
 
+// Division of any 32-bit unsigned number by a fixed divisor with a multiply and two shifts
+// (Granlund and Montgomery, "Division by invariant integers using multiplication", 1994).
+struct FastDiv {
+    uint32_t d, m, s1, s2;
+#ifdef __CUDACC__
+    __device__ __forceinline__ void divmod(uint32_t n, uint32_t& q, uint32_t& r) const {
+        const uint32_t t = __umulhi(m, n);
+        const uint32_t qq = (t + ((n - t) >> s1)) >> s2;
+        r = n - qq * d;
+        q = qq;
+    }
+#endif
+};
+
+inline FastDiv make_fast_div(uint32_t d) {
+    FastDiv f;
+    uint32_t L = 0;
+    while (L < 32 && ((uint64_t)1 << L) < d) ++L;
+    f.d = d;
+    f.m = (uint32_t)((((uint64_t)1 << 32) * (((uint64_t)1 << L) - d)) / d + 1);
+    f.s1 = L < 1 ? L : 1;
+    f.s2 = L > 0 ? L - 1 : 0;
+    return f;
+}
+
 // Per-scale grid description and scratch pointers, passed to kernels by value.
 struct ScaleDev {
     float mn[3];
     float vs[3];
     int dims[3];            // Gx, Gy, Gz
+    FastDiv div[3];         // division by Gx, Gy, Gz
     int cap;                // 0 = none
     int mode;               // ScaleMode
     uint32_t cells;         // cells per frame
-    uint32_t ntiles;        // 8 KB tiles of `store` for the largest batch
+    uint32_t ngroups;       // 1 KB groups of `store` for the largest batch
     uint32_t max_ovf;       // most cells that can exceed the cap
     uint32_t* store;        // bitmap: {bits, rank} per 32 cells; table: {count, rank, over-cap rank, -} per cell;
                             // bits / counts are zero between calls
-    uint32_t* tile_flag;    // [ntiles] tile holds an occupied cell (rewritten by every call)
+    int4* group_info;       // [ngroups] {voxels, cells over the cap, their points} before the group in its
+                            // warp's range of the rank scan, and the group's voxels (rewritten by every call)
     float4* acc;            // [max voxels][2] per-voxel accumulators
+    uint32_t* cell_list;    // [max voxels] cell id of each unique voxel (table stores: bit 31 = over the cap)
     int* ovf_off;           // per cell over the cap j: start of its points in ovf_list
     int* ovf_cursor;        // per cell over the cap j: points appended so far, at [j * kCursorStride]
     uint32_t* ovf_cell;     // per cell over the cap j: its cell id
@@ -71,6 +100,7 @@ struct emc2_bridge {
     int* d_tile_counts = nullptr;  // [B, tiles per frame, E]
     int* d_tile_base = nullptr;    // same shape, exclusive bases
     int* d_scan_part = nullptr;    // [scan_blocks][3] per-CTA totals of the voxel rank scan
+    int* d_scan_warp_ofs = nullptr;  // [scan_blocks * 8][3] per-warp offsets inside their CTA
     int scan_blocks = 0;           // CTAs of the cooperative rank scan (all co-resident)
     int max_tiles = 0;
     int last_cuda_error = 0;

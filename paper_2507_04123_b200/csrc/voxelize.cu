@@ -10,23 +10,24 @@
 //
 //   vox_mark      every point marks its two cells with one fire-and-forget reduction each;
 //                 the same launch zeroes the BEV image.
-//   vox_scan      one cooperative launch: counts per 8 KB tile of the store, grid barrier,
+//   vox_scan      one cooperative launch: counts per 1 KB group of the store, grid barrier,
 //                 then the exclusive prefix sums (the parallel prefix-sum index search of
-//                 Sec. 3.6) are written into the rank fields; accumulators are cleared and the
-//                 bookkeeping of cells over the cap is laid out.
+//                 Sec. 3.6) are written into the rank fields and the occupied cell ids listed
+//                 in that order; accumulators are cleared and the bookkeeping of cells over the
+//                 cap is laid out.
 //   vox_accum     every point looks its rank up, writes point_voxel and adds itself to its
 //                 voxels' accumulators with two fp32 vector reductions (offsets from the cell
 //                 corner, the other channels, the count).
 //                 Points of cells over the cap go to per-cell lists instead.
-//   vox_finalize  walks the occupied tiles of the store: one thread per word / cell writes
-//                 coordinates, count, mean and the BEV cell of its voxels and puts the store
-//                 back to zero; in the same launch one warp per cell over the cap keeps the
+//   vox_finalize  a warp per 32 consecutive voxels: coordinates from the listed cell id, count,
+//                 mean and BEV cell, with contiguous row traffic, and the store back to zero; in the same launch
+//                 one warp per cell over the cap keeps the
 //                 `cap` lowest point indices (keep-first-by-index) and sums them in fp64.
 //
 // Writes and reductions that land in one 32-byte sector are served one after another by the
 // L2 (about 10 ns each on B200), so nothing here funnels many points into a shared flag or
 // counter: the only contended words are the cells themselves.  The cost of a call follows the
-// occupied tiles, not the grid volume, except for one streaming read of the store.
+// occupied groups, not the grid volume, except for one streaming read of the store.
 #include <cooperative_groups.h>
 
 #include "bridge_internal.cuh"
@@ -62,10 +63,9 @@ __device__ __forceinline__ Slot slot_of(const ScaleDev& g, uint32_t cell) {
     return s;
 }
 
-// Exclusive scan of three counters across the CTA; CTA totals in tot[].
-__device__ __forceinline__ void block_excl_scan3(int v[3], int tot[3], int (*sm)[3]) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-    int inc[3];
+// Exclusive scan of three counters across the warp; warp totals in tot[].
+__device__ __forceinline__ void warp_excl_scan3(int v[3], int tot[3]) {
+    const int lane = threadIdx.x & 31;
 #pragma unroll
     for (int k = 0; k < 3; ++k) {
         int x = v[k];
@@ -74,48 +74,9 @@ __device__ __forceinline__ void block_excl_scan3(int v[3], int tot[3], int (*sm)
             const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
             if (lane >= d) x += y;
         }
-        inc[k] = x;
-        if (lane == 31) sm[warp][k] = x;
+        tot[k] = __shfl_sync(0xFFFFFFFFu, x, 31);
+        v[k] = x - v[k];
     }
-    __syncthreads();
-    if (warp == 0) {
-#pragma unroll
-        for (int k = 0; k < 3; ++k) {
-            int x = lane < nwarp ? sm[lane][k] : 0;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
-                if (lane >= d) x += y;
-            }
-            if (lane < nwarp) sm[lane][k] = x;   // inclusive over warps
-        }
-    }
-    __syncthreads();
-#pragma unroll
-    for (int k = 0; k < 3; ++k) {
-        const int wbase = warp ? sm[warp - 1][k] : 0;
-        tot[k] = sm[nwarp - 1][k];
-        v[k] = wbase + inc[k] - v[k];
-    }
-    __syncthreads();
-}
-
-// Sum of three counters across the CTA, result valid in every thread.
-__device__ __forceinline__ void block_sum3(int v[3], int (*sm)[3]) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-#pragma unroll
-    for (int k = 0; k < 3; ++k) {
-        const int x = warp_sum(v[k]);
-        if (lane == 0) sm[warp][k] = x;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int k = 0; k < 3; ++k) {
-        int x = 0;
-        for (int w = 0; w < nwarp; ++w) x += sm[w][k];
-        v[k] = x;
-    }
-    __syncthreads();
 }
 
 // Lower corner of cell i along one axis; both per-point and per-voxel code use this value.
@@ -161,21 +122,23 @@ vox_mark_kernel(const float* __restrict__ pts, long long total, int N, ScaleDev 
 // ------------------------------------------------------------------ pass 2: ranks
 struct ScanArgs {
     ScaleDev s[2];
-    uint32_t ntiles_used[2];    // tiles covering this call's B frames
+    uint32_t ngroups_used[2];   // 1 KB groups covering this call's B frames
     int capacity[2];
     int32_t* num_voxels;
     int* status;
     int* part;                  // [gridDim.x][3] per-CTA totals
+    int* warp_ofs;              // [gridDim.x * warps][3] totals of the warps before a warp in its CTA
     int g0;                     // CTAs [0, g0) serve scale 0, the rest scale 1
 };
 
-// One thread owns one 32-byte sector of the store: four {bits, rank} pairs or two cell records.
+// One lane owns one 32-byte sector of the store: four {bits, rank} pairs or two cell records;
+// a warp owns a 1 KB group.
 struct Sector {
     uint4 a, b;
 };
 
-__device__ __forceinline__ Sector load_sector(const uint32_t* store, uint32_t tile, int t) {
-    const uint4* p = reinterpret_cast<const uint4*>(store) + ((size_t)tile * kThreads + t) * 2;
+__device__ __forceinline__ Sector load_sector(const uint32_t* store, uint32_t group, int lane) {
+    const uint4* p = reinterpret_cast<const uint4*>(store) + ((size_t)group * 32 + lane) * 2;
     Sector s;
     s.a = p[0];
     s.b = p[1];
@@ -196,97 +159,149 @@ __device__ __forceinline__ void sector_stats(const ScaleDev& g, const Sector& s,
     }
 }
 
-// Cooperative launch.  Every CTA owns a contiguous range of tiles of one scale.  Phase 1 counts
-// and notes which tiles hold anything; after the grid barrier every CTA adds up the totals of
-// the CTAs before it; phase 2 walks the occupied tiles again and writes the ranks.
+// Cooperative launch.  Phase 1: every warp owns a contiguous range of groups of one scale, CTA
+// after CTA, counts them and records, per group, its count and the running total inside the
+// warp's range.  After the grid barrier every CTA scans the CTA totals, which makes the rank of
+// any group's first cell computable from three small records.  Phase 2 then hands the groups out
+// round-robin, so that densely occupied regions are spread over all warps, writes the ranks into
+// the store and lists the occupied cell ids in rank order.  The loops have no CTA barrier.
 __global__ void __launch_bounds__(kThreads) vox_scan_kernel(ScanArgs a) {
-    __shared__ int sm[kThreads / 32][3];
+    constexpr int kWarps = kThreads / 32;
+    __shared__ int sm[kWarps][3];
+    __shared__ int wtot[kWarps][3];
+    __shared__ int cta_base[kMaxScanBlocks][3];   // exclusive totals of the CTAs of this scale
     cg::grid_group grid = cg::this_grid();
     const int sc = (int)blockIdx.x >= a.g0 ? 1 : 0;
     const int first = sc ? a.g0 : 0;
     const int cta = (int)blockIdx.x - first;
     const int ncta = sc ? (int)gridDim.x - a.g0 : a.g0;
     const ScaleDev& g = a.s[sc];
-    const uint32_t ntiles = a.ntiles_used[sc];
-    const uint32_t per = (ntiles + (uint32_t)ncta - 1u) / (uint32_t)ncta;
-    const uint32_t lo = min(ntiles, (uint32_t)cta * per), hi = min(ntiles, lo + per);
-    const int t = threadIdx.x;
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const uint32_t ng = a.ngroups_used[sc];
+    const uint32_t per = max(1u, (ng + (uint32_t)(ncta * kWarps) - 1u) / (uint32_t)(ncta * kWarps));
+    const uint32_t lo = min(ng, (uint32_t)(cta * kWarps + warp) * per), hi = min(ng, lo + per);
 
-    int s[3] = {0, 0, 0};
-    for (uint32_t tile = lo; tile < hi; ++tile) {
-        const int before = s[0];
-        sector_stats(g, load_sector(g.store, tile, t), s);
-        const int any = __syncthreads_or(s[0] != before);
-        if (t == 0) g.tile_flag[tile] = (uint32_t)any;
+    int carry[3] = {0, 0, 0};
+    for (uint32_t grp = lo; grp < hi; grp += 4) {
+        Sector x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (grp + u < hi) x[u] = load_sector(g.store, grp + u, lane);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (grp + u >= hi) break;
+            int s[3] = {0, 0, 0};
+            sector_stats(g, x[u], s);
+#pragma unroll
+            for (int k = 0; k < 3; ++k) s[k] = warp_sum(s[k]);
+            if (lane == 0) g.group_info[grp + u] = make_int4(carry[0], carry[1], carry[2], s[0]);
+#pragma unroll
+            for (int k = 0; k < 3; ++k) carry[k] += s[k];
+        }
     }
-    block_sum3(s, sm);
-    if (t < 3) a.part[blockIdx.x * 3 + t] = s[t];
+    if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < 3; ++k) wtot[warp][k] = carry[k];
+    }
+    __syncthreads();
+    if (t < 3) {
+        int v = 0;
+        for (int w = 0; w < kWarps; ++w) {
+            a.warp_ofs[((size_t)blockIdx.x * kWarps + w) * 3 + t] = v;   // warp's offset inside its CTA
+            v += wtot[w][t];
+        }
+        a.part[blockIdx.x * 3 + t] = v;
+    }
     grid.sync();
 
-    // Totals of the CTAs before this one (same scale) and of the whole scale.
-    int base[3] = {0, 0, 0}, tot[3] = {0, 0, 0};
-    for (int c = t; c < ncta; c += kThreads) {
-        const int* p = a.part + (size_t)(first + c) * 3;
-        const int v0 = p[0], v1 = p[1], v2 = p[2];
-        tot[0] += v0; tot[1] += v1; tot[2] += v2;
-        if (c < cta) { base[0] += v0; base[1] += v1; base[2] += v2; }
+    // Exclusive scan of the CTA totals of this scale, by warp 0: each lane sums a run of CTAs.
+    if (warp == 0) {
+        const int run = (ncta + 31) / 32;
+        const int c_lo = min(ncta, lane * run), c_hi = min(ncta, c_lo + run);
+        int v[3] = {0, 0, 0}, tt[3];
+        for (int c = c_lo; c < c_hi; ++c) {
+            const int* p = a.part + (size_t)(first + c) * 3;
+            v[0] += p[0]; v[1] += p[1]; v[2] += p[2];
+        }
+        warp_excl_scan3(v, tt);
+        for (int c = c_lo; c < c_hi; ++c) {
+            const int* p = a.part + (size_t)(first + c) * 3;
+            cta_base[c][0] = v[0]; cta_base[c][1] = v[1]; cta_base[c][2] = v[2];
+            v[0] += p[0]; v[1] += p[1]; v[2] += p[2];
+        }
+        if (lane == 0) { sm[0][0] = tt[0]; sm[0][1] = tt[1]; sm[0][2] = tt[2]; }
     }
-    block_sum3(base, sm);
-    block_sum3(tot, sm);
+    __syncthreads();
+    const int tot0 = sm[0][0];
     if (cta == 0 && t == 0) {
-        g.totals[0] = tot[0]; g.totals[1] = tot[1]; g.totals[2] = tot[2];
-        a.num_voxels[sc] = tot[0];
-        if (tot[0] > a.capacity[sc]) atomicOr(a.status, kStatusCapacity);
+        g.totals[0] = sm[0][0]; g.totals[1] = sm[0][1]; g.totals[2] = sm[0][2];
+        a.num_voxels[sc] = tot0;
+        if (tot0 > a.capacity[sc]) atomicOr(a.status, kStatusCapacity);
     }
     // Clear the accumulators of the voxels found (two 16-byte halves per voxel).
     {
         const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-        const size_t n = 2 * (size_t)tot[0];
+        const size_t n = 2 * (size_t)tot0;
         for (size_t i = (size_t)cta * kThreads + t; i < n; i += (size_t)ncta * kThreads) g.acc[i] = z;
     }
 
-    int carry[3] = {base[0], base[1], base[2]};
-    for (uint32_t tile = lo; tile < hi; ++tile) {
-        if (!g.tile_flag[tile]) continue;         // written by this CTA in phase 1; same for all threads
-        Sector x = load_sector(g.store, tile, t);
-        int run[3] = {0, 0, 0}, ttot[3];
+    const uint32_t nw = (uint32_t)(ncta * kWarps);
+    for (uint32_t grp = (uint32_t)(cta * kWarps + warp); grp < ng; grp += nw) {
+        const int4 info = g.group_info[grp];      // same for all lanes
+        if (info.w == 0) continue;
+        const uint32_t owner = grp / per;         // warp that counted this group, within the scale
+        const int* wo = a.warp_ofs + ((size_t)first * kWarps + owner) * 3;
+        const int* cb = cta_base[owner / kWarps];
+        const int base0 = cb[0] + wo[0] + info.x;
+        Sector x = load_sector(g.store, grp, lane);
+        int run[3] = {0, 0, 0}, gtot[3];
         sector_stats(g, x, run);
         const bool mine = run[0] > 0;
-        block_excl_scan3(run, ttot, sm);          // run[] = exclusive offsets inside the tile
-        if (mine) {
-            int m = carry[0] + run[0];
-            if (g.mode == MODE_BITMAP) {
-                x.a.y = (uint32_t)m; m += __popc(x.a.x);
-                x.a.w = (uint32_t)m; m += __popc(x.a.z);
-                x.b.y = (uint32_t)m; m += __popc(x.b.x);
-                x.b.w = (uint32_t)m;
-            } else {
-                int j = carry[1] + run[1], off = carry[2] + run[2];
-                const uint32_t cell0 = (tile * (uint32_t)kThreads + t) * 2u;
-                x.a.y = (uint32_t)m; x.a.z = (uint32_t)j;
-                const int n0 = (int)x.a.x, n1 = (int)x.b.x;
-                if (g.cap > 0 && n0 > g.cap) {
-                    g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
-                    j += 1; off += n0;
-                }
-                m += n0 > 0;
-                x.b.y = (uint32_t)m; x.b.z = (uint32_t)j;
-                if (g.cap > 0 && n1 > g.cap) {
-                    g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0 + 1u; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+        warp_excl_scan3(run, gtot);               // run[] = exclusive offsets inside the group
+        if (!mine) continue;
+        int m = base0 + run[0];
+        if (g.mode == MODE_BITMAP) {
+            const uint32_t word0 = (grp * 32u + lane) * 4u;
+            const uint32_t bw[4] = {x.a.x, x.a.z, x.b.x, x.b.z};
+            uint32_t rk[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                rk[i] = (uint32_t)m;
+                uint32_t bits = bw[i];
+                while (bits) {                    // plain stores: nothing here waits on memory
+                    const int bit = __ffs(bits) - 1;
+                    bits &= bits - 1;
+                    g.cell_list[m++] = (word0 + i) * 32u + bit;
                 }
             }
-            uint4* p = reinterpret_cast<uint4*>(g.store) + ((size_t)tile * kThreads + t) * 2;
-            p[0] = x.a;
-            p[1] = x.b;
+            x.a.y = rk[0]; x.a.w = rk[1]; x.b.y = rk[2]; x.b.w = rk[3];
+        } else {
+            int j = cb[1] + wo[1] + info.y + run[1], off = cb[2] + wo[2] + info.z + run[2];
+            const uint32_t cell0 = (grp * 32u + lane) * 2u;
+            x.a.y = (uint32_t)m; x.a.z = (uint32_t)j;
+            const int n0 = (int)x.a.x, n1 = (int)x.b.x;
+            const bool o0 = g.cap > 0 && n0 > g.cap, o1 = g.cap > 0 && n1 > g.cap;
+            if (o0) {
+                g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+                j += 1; off += n0;
+            }
+            if (n0 > 0) g.cell_list[m++] = cell0 | (o0 ? 0x80000000u : 0u);
+            x.b.y = (uint32_t)m; x.b.z = (uint32_t)j;
+            if (o1) {
+                g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0 + 1u; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+            }
+            if (n1 > 0) g.cell_list[m] = (cell0 + 1u) | (o1 ? 0x80000000u : 0u);
         }
-        carry[0] += ttot[0]; carry[1] += ttot[1]; carry[2] += ttot[2];
+        uint4* p = reinterpret_cast<uint4*>(g.store) + ((size_t)grp * 32 + lane) * 2;
+        p[0] = x.a;
+        p[1] = x.b;
     }
 }
 
 // ------------------------------------------------------------------ pass 3: accumulate
 struct AccumArgs {
     ScaleDev s[2];
-    uint32_t ntiles_used[2];
+    uint32_t ngroups_used[2];
     int capacity[2];
     int32_t* coords[2];
     int32_t* counts[2];
@@ -363,32 +378,58 @@ vox_accum_kernel(const float* __restrict__ pts, long long total, int N, AccumArg
 }
 
 // ------------------------------------------------------------------ pass 4: rows, BEV, cleanup
-// Writes the output rows of voxel m, whose cell is `cell`, from its accumulator.
+// Writes the output rows of n <= 32 voxels with consecutive rows mb, mb+1, ..., one per lane;
+// lane i holds the cell-list entry of row mb + i; `stage` is 1 KB of the warp's own shared memory.  Accumulators are read and mean rows written as
+// contiguous blocks through shared memory, so the warp issues full-sector requests only.
 template <int C>
-__device__ __forceinline__ void write_voxel(const AccumArgs& a, int sc, const ScaleDev& g, int m, uint32_t cell,
-                                            bool over) {
-    if (m >= a.capacity[sc]) return;
-    const float4 a0 = g.acc[2 * (size_t)m];
-    const float4 a1 = g.acc[2 * (size_t)m + 1];
-    uint32_t r = cell;
-    const uint32_t x = r % g.dims[0]; r /= g.dims[0];
-    const uint32_t y = r % g.dims[1]; r /= g.dims[1];
-    const uint32_t z = r % g.dims[2]; r /= g.dims[2];
-    reinterpret_cast<int4*>(a.coords[sc])[m] = make_int4((int)r, (int)z, (int)y, (int)x);
-    const int n = over ? g.cap : (int)a1.y;
-    a.counts[sc][m] = n;
-    if (over) return;                             // mean and BEV cell come from the cell's warp
-    const double inv = 1.0 / (double)n;
+__device__ __forceinline__ void write_batch(const AccumArgs& a, int sc, int mb, int n, uint32_t entry,
+                                            float4* stage) {
+    const ScaleDev& g = a.s[sc];
+    const int lane = threadIdx.x & 31;
+    n = min(n, a.capacity[sc] - mb);              // rows past the caller's capacity are not written
+    if (n <= 0) return;
+    const float4* src = g.acc + 2 * (size_t)mb;
+    if (lane < 2 * n) stage[lane] = src[lane];
+    if (lane + 32 < 2 * n) stage[lane + 32] = src[lane + 32];
+    __syncwarp();
+    const float4 a0 = stage[2 * lane], a1 = stage[2 * lane + 1];
+    __syncwarp();
+    const bool active = lane < n;
+    const bool table = g.mode == MODE_TABLE;
+    const uint32_t cell = table ? (entry & 0x7FFFFFFFu) : entry;
+    const bool over = active && table && (entry >> 31) != 0u;
+    uint32_t r = cell, x, y, z;
+    g.div[0].divmod(r, r, x);
+    g.div[1].divmod(r, r, y);
+    g.div[2].divmod(r, r, z);
+    const int cnt = over ? g.cap : (int)a1.y;
+    // Offsets are below one cell size, so fp32 keeps the mean to a few 1e-7 of that size.
+    const float inv = __frcp_rn((float)cnt);
     float mu[C];
-    mu[0] = (float)((double)cell_corner(g.mn[0], g.vs[0], (int)x) + (double)a0.x * inv);
-    mu[1] = (float)((double)cell_corner(g.mn[1], g.vs[1], (int)y) + (double)a0.y * inv);
-    mu[2] = (float)((double)cell_corner(g.mn[2], g.vs[2], (int)z) + (double)a0.z * inv);
-    mu[3] = (float)((double)a0.w * inv);
-    if (C > 4) mu[4] = (float)((double)a1.x * inv);
-    float* row = a.mean[sc] + (size_t)m * C;
+    mu[0] = __fadd_rn(cell_corner(g.mn[0], g.vs[0], (int)x), a0.x * inv);
+    mu[1] = __fadd_rn(cell_corner(g.mn[1], g.vs[1], (int)y), a0.y * inv);
+    mu[2] = __fadd_rn(cell_corner(g.mn[2], g.vs[2], (int)z), a0.z * inv);
+    mu[3] = __fdiv_rn(a0.w, (float)cnt);
+    if (C > 4) mu[4] = __fdiv_rn(a1.x, (float)cnt);
+    if (active) {
+        reinterpret_cast<int4*>(a.coords[sc])[mb + lane] = make_int4((int)r, (int)z, (int)y, (int)x);
+        a.counts[sc][mb + lane] = cnt;
+    }
+    // Mean rows: the n * C floats of rows mb .. mb+n-1 are contiguous.  The row of a cell over the
+    // cap is written by that cell's own warp, so a batch holding one writes its rows one by one.
+    float* rows = a.mean[sc] + (size_t)mb * C;
+    if (!__any_sync(0xFFFFFFFFu, over)) {
+        float* st = reinterpret_cast<float*>(stage);
 #pragma unroll
-    for (int k = 0; k < C; ++k) row[k] = mu[k];
-    if (sc == 1 && a.bev) {
+        for (int k = 0; k < C; ++k) st[lane * C + k] = mu[k];
+        __syncwarp();
+        for (int i = lane; i < n * C; i += 32) rows[i] = st[i];
+        __syncwarp();
+    } else if (active && !over) {
+#pragma unroll
+        for (int k = 0; k < C; ++k) rows[lane * C + k] = mu[k];
+    }
+    if (sc == 1 && a.bev && active && !over) {
         const size_t plane = (size_t)g.dims[1] * g.dims[0];
         float* dst = a.bev + (size_t)r * C * plane + (size_t)y * g.dims[0] + x;
 #pragma unroll
@@ -398,16 +439,15 @@ __device__ __forceinline__ void write_voxel(const AccumArgs& a, int sc, const Sc
 
 // CTAs [0, ovf_blocks) serve cells over the cap, one warp per cell: the `cap` lowest point
 // indices are kept (keep-first-by-index), summed in fp64 and written as the voxel's mean; all of
-// the cell's points get their point_voxel entry.  The other CTAs stride over the occupied tiles
-// of both stores, one thread per word / cell: coordinates from the cell id, count, mean, BEV
-// cell; then the word / cell goes back to zero.
+// the cell's points get their point_voxel entry.  The other CTAs write the voxel rows.
 template <int C>
 __global__ void __launch_bounds__(kThreads)
 vox_finalize_kernel(const float* __restrict__ pts, long long total, AccumArgs a, int ovf_blocks) {
+    constexpr int kWarps = kThreads / 32;
+    const int lane = threadIdx.x & 31;
     if ((int)blockIdx.x < ovf_blocks) {
-        const int lane = threadIdx.x & 31;
         const int warp = (blockIdx.x * kThreads + threadIdx.x) >> 5;
-        const int nwarps = (ovf_blocks * kThreads) >> 5;
+        const int nwarps = ovf_blocks * kWarps;
         for (int sc = 0; sc < 2; ++sc) {
             const ScaleDev& g = a.s[sc];
             if (g.cap <= 0) continue;
@@ -450,9 +490,9 @@ vox_finalize_kernel(const float* __restrict__ pts, long long total, AccumArgs a,
                     const float mu = (float)(v / (double)g.cap);
                     a.mean[sc][(size_t)m * C + lane] = mu;
                     if (sc == 1 && a.bev) {
-                        uint32_t r = g.ovf_cell[j];
-                        const uint32_t x = r % g.dims[0]; r /= g.dims[0];
-                        const uint32_t y = r % g.dims[1]; r /= g.dims[1];
+                        uint32_t r = g.ovf_cell[j], x, y;
+                        g.div[0].divmod(r, r, x);
+                        g.div[1].divmod(r, r, y);
                         const size_t plane = (size_t)g.dims[1] * g.dims[0];
                         a.bev[((size_t)r * C + lane) * plane + (size_t)y * g.dims[0] + x] = mu;
                     }
@@ -461,75 +501,25 @@ vox_finalize_kernel(const float* __restrict__ pts, long long total, AccumArgs a,
         }
         return;
     }
-    // Voxel rows.  Occupied cells are first compacted into a shared list (their rows are
-    // consecutive: the first one's rank plus the list position), then the list is worked off one
-    // voxel per thread, so that accumulator reads and row writes are dense whatever the
-    // occupancy pattern.
-    __shared__ uint32_t s_cell[kThreads * 32];    // cell ids of one round; table mode: bit 31 = over the cap
-    __shared__ int s_warp[kThreads / 32];
-    __shared__ int s_first;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t t0 = a.ntiles_used[0], t1 = a.ntiles_used[1];
-    const uint32_t nblk = gridDim.x - ovf_blocks;
-    for (uint32_t v = blockIdx.x - ovf_blocks; v < t0 + t1; v += nblk) {
-        const int sc = v >= t0 ? 1 : 0;
-        const uint32_t tile = sc ? v - t0 : v;
+    // Voxel rows: a warp takes 32 consecutive rows of one scale at a time, reads their cell ids
+    // from the list the rank scan wrote, writes the rows and puts the cells' store words back to
+    // zero.  Every warp has its own batch, so the batches' memory latencies overlap.
+    __shared__ float4 s_stage[kWarps][64];
+    float4* stage = s_stage[threadIdx.x >> 5];
+    const int tot0 = a.s[0].totals[0], tot1 = a.s[1].totals[0];
+    const int nb0 = (tot0 + 31) >> 5, nb1 = (tot1 + 31) >> 5;
+    const int nwarps = ((int)gridDim.x - ovf_blocks) * kWarps;
+    for (int v = ((int)blockIdx.x - ovf_blocks) * kWarps + (threadIdx.x >> 5); v < nb0 + nb1; v += nwarps) {
+        const int sc = v >= nb0 ? 1 : 0;
+        const int mb = (sc ? v - nb0 : v) << 5;
         const ScaleDev& g = a.s[sc];
-        if (!g.tile_flag[tile]) continue;
-        const bool bitmap = g.mode == MODE_BITMAP;
-        const int rounds = bitmap ? 4 : 2;        // 1024 words or 512 cells per tile, 256 per round
-        for (int rnd = 0; rnd < rounds; ++rnd) {
-            uint32_t bits = 0u, id0 = 0u;
-            int rank = 0, k = 0;
-            if (bitmap) {
-                const uint32_t word = tile * (uint32_t)(4 * kThreads) + rnd * kThreads + threadIdx.x;
-                uint2* pp = reinterpret_cast<uint2*>(g.store) + word;
-                const uint2 pr = *pp;
-                if (pr.x) *pp = make_uint2(0u, 0u);
-                bits = pr.x; rank = (int)pr.y; id0 = word * 32u; k = __popc(bits);
-            } else {
-                const uint32_t cell = tile * (uint32_t)(2 * kThreads) + rnd * kThreads + threadIdx.x;
-                uint4* pq = reinterpret_cast<uint4*>(g.store) + cell;
-                const uint4 q = *pq;
-                if (q.x) *pq = make_uint4(0u, 0u, 0u, 0u);
-                bits = q.x ? 1u : 0u; rank = (int)q.y; k = (int)bits;
-                id0 = cell | ((g.cap > 0 && (int)q.x > g.cap) ? 0x80000000u : 0u);
-            }
-            // Exclusive position of this thread's cells in the round's list.
-            int inc = k;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                if (lane >= d) inc += y;
-            }
-            if (lane == 31) s_warp[warp] = inc;
-            __syncthreads();
-            int off = inc - k, total_k = 0;
-#pragma unroll
-            for (int w = 0; w < kThreads / 32; ++w) {
-                const int c = s_warp[w];
-                if (w < warp) off += c;
-                total_k += c;
-            }
-            if (k > 0 && off == 0) s_first = rank;   // exactly one thread owns the round's first voxel
-            if (bitmap) {
-                while (bits) {
-                    const int bit = __ffs(bits) - 1;
-                    bits &= bits - 1;
-                    s_cell[off++] = id0 + bit;
-                }
-            } else if (k) {
-                s_cell[off] = id0;
-            }
-            __syncthreads();
-            const int m0 = s_first;
-            for (int i = threadIdx.x; i < total_k; i += kThreads) {
-                const uint32_t c = s_cell[i];
-                if (bitmap) write_voxel<C>(a, sc, g, m0 + i, c, false);
-                else write_voxel<C>(a, sc, g, m0 + i, c & 0x7FFFFFFFu, (c >> 31) != 0u);
-            }
-            __syncthreads();
+        const int n = min(32, (sc ? tot1 : tot0) - mb);
+        const uint32_t entry = lane < n ? g.cell_list[mb + lane] : 0u;
+        if (lane < n) {
+            if (g.mode == MODE_BITMAP) *reinterpret_cast<uint2*>(g.store + 2 * (size_t)(entry >> 5)) = make_uint2(0u, 0u);
+            else *reinterpret_cast<uint4*>(g.store + 4 * (size_t)(entry & 0x7FFFFFFFu)) = make_uint4(0u, 0u, 0u, 0u);
         }
+        write_batch<C>(a, sc, mb, n, entry, stage);
     }
 }
 
@@ -546,8 +536,8 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
         sa.s[s] = h->scale[s];
         aa.s[s] = h->scale[s];
         const uint64_t cells = (uint64_t)B * h->scale[s].cells;
-        const uint64_t per_tile = h->scale[s].mode == MODE_BITMAP ? kBitmapTileCells : kTableTileCells;
-        sa.ntiles_used[s] = aa.ntiles_used[s] = (uint32_t)((cells + per_tile - 1) / per_tile);
+        const uint64_t per_group = h->scale[s].mode == MODE_BITMAP ? kBitmapGroupCells : kTableGroupCells;
+        sa.ngroups_used[s] = aa.ngroups_used[s] = (uint32_t)((cells + per_group - 1) / per_group);
         sa.capacity[s] = aa.capacity[s] = capacity[s];
         aa.coords[s] = d_coords[s];
         aa.counts[s] = d_counts[s];
@@ -558,10 +548,11 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     sa.num_voxels = d_num_voxels;
     sa.status = h->d_status;
     sa.part = h->d_scan_part;
+    sa.warp_ofs = h->d_scan_warp_ofs;
     aa.bev = d_bev;
-    // Split the cooperative grid between the scales in proportion to their tile counts.
+    // Split the cooperative grid between the scales in proportion to their group counts.
     const int G = h->scan_blocks;
-    const double share = (double)sa.ntiles_used[0] / (double)((uint64_t)sa.ntiles_used[0] + sa.ntiles_used[1] + 1);
+    const double share = (double)sa.ngroups_used[0] / (double)((uint64_t)sa.ngroups_used[0] + sa.ngroups_used[1] + 1);
     sa.g0 = min(G - 1, max(1, (int)(share * G)));
 
     const size_t bev_n = d_bev ? (size_t)B * C * h->scale[1].dims[1] * h->scale[1].dims[0] : 0;
@@ -589,10 +580,9 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
             vox_accum_kernel<C><<<ptiles, kThreads, 0, st>>>(d_points, total, N, aa);
         }
         {
-            // Which tiles hold voxels is only known on the device: a fixed grid strides over them.
+            // The number of voxels is only known on the device: a fixed grid strides over them.
             const int ovf_blocks = any_cap ? kOvfBlocks : 0;
-            const uint32_t tiles = sa.ntiles_used[0] + sa.ntiles_used[1];
-            const int vox_blocks = (int)min((uint32_t)(148 * 8), max(tiles, 1u));
+            const int vox_blocks = (int)min((long long)148 * 8, (2 * total + 32 * 8 - 1) / (32 * 8) + 1);
             LaunchScope ls(h, K_VOX_FINALIZE, st);
             vox_finalize_kernel<C><<<ovf_blocks + vox_blocks, kThreads, 0, st>>>(d_points, total, aa, ovf_blocks);
         }
@@ -609,7 +599,7 @@ int voxel_scan_max_blocks() {
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, vox_scan_kernel, kThreads, 0) != cudaSuccess) return 0;
     int coop = 0;
     if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return 0;
-    return sms * min(per_sm, 4);
+    return min(sms * min(per_sm, 4), kMaxScanBlocks);
 }
 
 int launch_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* const d_coords[2],
