@@ -1,9 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the EMC2 data bridge + dispatch on B200.
 
-A step is one pass of the whole hot path (emc2_voxelize, emc2_project_gather,
-emc2_route_dispatch back to back on one stream) over one batch of synthetic
-frames.  Default workload: the nuScenes-shaped 6-camera batch (4 frames of
+A step is one pass of the whole hot path (emc2_bridge_run: voxelize, project +
+gather, route + dispatch; the three stage calls back to back are timed as well)
+over one batch of synthetic frames.  Default workload: the nuScenes-shaped 6-camera batch (4 frames of
 300,000 points), the configuration the roofline target is quoted on.
 
     python bench.py --gpus 1 --steps 20 --warmup 5
@@ -231,8 +231,11 @@ def run_ours(args, w):
     texels = distinct_texels(w, bufs["pg"])
     abytes = algorithmic_bytes(w, B, N, int(nv[0]), int(nv[1]), texels)
 
-    def step():
+    def step():                                            # emc2_bridge_run: the whole path in one call
         br.run(d["points"], d["proj"], d["feat"], bufs)
+
+    def staged_step():                                     # the same work as three stage calls
+        br.run_staged(d["points"], d["proj"], d["feat"], bufs)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -244,6 +247,10 @@ def run_ours(args, w):
     secs = max_over_ranks(time_steps(step, args.steps, sync, barrier))
     launches = sum(n for n, _ in br.profile_read(reset=True).values())
     br.status()
+    for _ in range(3):
+        staged_step()
+    staged_secs = max_over_ranks(time_steps(staged_step, args.steps, sync, barrier))
+    br.profile_read(reset=True)
 
     # End to end: pinned host inputs copied in every step, small results read back every step.
     e2e_in = {k: torch.empty_like(v) for k, v in d.items()}
@@ -274,7 +281,7 @@ def run_ours(args, w):
     br.profile_enable(True)
     prof_steps = max(3, min(args.steps, 10))
     for _ in range(prof_steps):
-        step()
+        staged_step()                                      # kernels one after another: clean per-kernel times
     sync()
     prof = br.profile_read(reset=True)
     br.profile_enable(False)
@@ -317,6 +324,7 @@ def run_ours(args, w):
                    "l2": "inputs and outputs of a step exceed L2 (no flush)" if abytes["total"] > 2 * L2_BYTES
                          else "working set fits in L2 (latency-bound workload, no flush)"},
         "mpoints_per_s": fps * N / 1e6,
+        "staged_ms_per_step": staged_secs / args.steps * 1e3,
         "bridge_algorithmic_bytes_per_step": abytes,
         "bridge_gbs": total_gbs, "bridge_frac_of_8tbs": total_gbs / NOMINAL_HBM_GBS,
         f"bridge_frac_of_{peak_kind}_copy": total_gbs / peak,

@@ -137,6 +137,22 @@ int emc2_route_dispatch(emc2_bridge_t* bridge, int32_t B, int32_t N, const float
                         int32_t* d_offsets, int32_t* d_perm, float* d_points_out, float* d_feat_out,
                         void* cuda_stream);
 
+/* The whole bridge in one call (all four stages; Sec. 3.1 - 3.2, with the overlap of independent
+ * work that Sec. 3.6 asks of the system).  Arguments, outputs, layouts and errors are exactly those
+ * of emc2_voxelize, emc2_project_gather and emc2_route_dispatch called in that order with the same
+ * buffers; d_vis_mask and d_gathered of stage 2 feed stages 3 - 4.  Stage 1 does not depend on
+ * stages 2 - 4, so the library runs it on a stream of its own (created with the handle, highest
+ * priority) beside them: it starts once the work already queued on `cuda_stream` has finished,
+ * and `cuda_stream` waits for it before the call's work counts as complete.  Seen from
+ * `cuda_stream` the call therefore behaves like the three calls, only shorter.  No allocation,
+ * no host synchronisation. */
+int emc2_bridge_run(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_points, const float* d_proj,
+                    const float* d_feat, int32_t* const d_coords[2], int32_t* const d_counts[2],
+                    float* const d_mean[2], int32_t* const d_point_voxel[2], const int32_t capacity[2],
+                    int32_t* d_num_voxels, float* d_bev, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
+                    float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
+                    float* d_points_out, float* d_feat_out, void* cuda_stream);
+
 /* Stages 3 and 4 for callers that must not allocate device memory (the paper has no counterpart;
  * this is a packaging variant of emc2_route_dispatch).
  *

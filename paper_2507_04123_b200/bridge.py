@@ -33,6 +33,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_status", "emc2_bridge_destroy", "emc2_status_string", "emc2_bridge_last_cuda_error",
     "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
+    "emc2_bridge_run",
 )
 
 
@@ -75,6 +76,8 @@ def load_library() -> ctypes.CDLL:
     lib.emc2_voxelize.argtypes = [vp, i32, i32, vp, P(vp), P(vp), P(vp), P(vp), P(i32), vp, vp, vp]
     lib.emc2_project_gather.argtypes = [vp, i32, i32] + [vp] * 8
     lib.emc2_route_dispatch.argtypes = [vp, i32, i32] + [vp] * 9
+    lib.emc2_bridge_run.argtypes = ([vp, i32, i32, vp, vp, vp, P(vp), P(vp), P(vp), P(vp), P(i32), vp, vp]
+                                    + [vp] * 4 + [vp] * 5 + [vp])
     lib.emc2_route_dispatch_static.argtypes = [P(Emc2Config), i32, i32] + [vp] * 9
     lib.emc2_bridge_status.argtypes = [vp, vp]
     lib.emc2_bridge_destroy.argtypes = [vp]
@@ -289,14 +292,63 @@ class Bridge:
         return rc
 
     # ------------------------------------------------------------------ whole path
-    def run(self, points: torch.Tensor, proj: torch.Tensor, feat: torch.Tensor,
-            bufs: Optional[Dict[str, object]] = None) -> Dict[str, object]:
+    def _alloc_vox(self, B, N, C, cap, want_point_voxel=True, want_bev=True):
+        dev = self.device
+        return {
+            "coords": [torch.empty((max(cap[s], 1), 4), dtype=torch.int32, device=dev) for s in range(2)],
+            "counts": [torch.empty((max(cap[s], 1),), dtype=torch.int32, device=dev) for s in range(2)],
+            "mean": [torch.empty((max(cap[s], 1), C), dtype=torch.float32, device=dev) for s in range(2)],
+            "point_voxel": [torch.empty((B, N), dtype=torch.int32, device=dev) for _ in range(2)]
+            if want_point_voxel else None,
+            "num_voxels": torch.empty((2,), dtype=torch.int32, device=dev),
+            "bev": torch.empty((B, C, self.cfg.grid[1].dims[1], self.cfg.grid[1].dims[0]),
+                               dtype=torch.float32, device=dev) if want_bev else None,
+        }
+
+    def run_staged(self, points: torch.Tensor, proj: torch.Tensor, feat: torch.Tensor,
+                   bufs: Optional[Dict[str, object]] = None) -> Dict[str, object]:
         """The three stage calls back to back on the current stream (no host sync)."""
         bufs = bufs if bufs is not None else {}
         bufs["vox"] = self.voxelize(points, out=bufs.get("vox"))
         bufs["pg"] = self.project_gather(points, proj, feat, out=bufs.get("pg"))
         pg = bufs["pg"]
         bufs["rd"] = self.route_dispatch(points, pg["vis_mask"], pg["gathered"], out=bufs.get("rd"))
+        return bufs
+
+    def run(self, points: torch.Tensor, proj: torch.Tensor, feat: torch.Tensor,
+            bufs: Optional[Dict[str, object]] = None) -> Dict[str, object]:
+        """emc2_bridge_run: all stages in one call; same outputs as :meth:`run_staged`."""
+        B, N, C = points.shape
+        c = self.cfg
+        _check(points, torch.float32, (B, N, c.point_floats), "points", self.device)
+        _check(proj, torch.float32, (B, c.num_cameras, 3, 4), "proj", self.device)
+        _check(feat, torch.float32, (B, c.num_cameras, c.feat_h, c.feat_w, c.feat_c), "feat", self.device)
+        if bufs is None:
+            dev = self.device
+            bufs = {"vox": self._alloc_vox(B, N, C, [B * N, B * N]),
+                    "pg": {"uvd": torch.empty((B, N, 3), dtype=torch.float32, device=dev),
+                           "vis_mask": torch.empty((B, N), dtype=torch.uint8, device=dev),
+                           "cam": torch.empty((B, N), dtype=torch.int8, device=dev),
+                           "gathered": torch.empty((B, N, c.feat_c), dtype=torch.float32, device=dev)},
+                    "rd": {"expert": torch.empty((B, N), dtype=torch.uint8, device=dev),
+                           "offsets": torch.empty((B, c.num_experts + 1), dtype=torch.int32, device=dev),
+                           "perm": torch.empty((B, N), dtype=torch.int32, device=dev),
+                           "points_out": torch.empty_like(points),
+                           "feat_out": torch.empty((B, N, c.feat_c), dtype=torch.float32, device=dev)}}
+        vox, pg, rd = bufs["vox"], bufs["pg"], bufs["rd"]
+        arr = ctypes.c_void_p * 2
+        pv = vox["point_voxel"]
+        cap = [int(vox["coords"][s].shape[0]) for s in range(2)]
+        rc = self.lib.emc2_bridge_run(
+            self._h, B, N, points.data_ptr(), proj.data_ptr(), feat.data_ptr(),
+            arr(*[t.data_ptr() for t in vox["coords"]]), arr(*[t.data_ptr() for t in vox["counts"]]),
+            arr(*[t.data_ptr() for t in vox["mean"]]),
+            arr(*[t.data_ptr() for t in pv]) if pv is not None else None,
+            (ctypes.c_int32 * 2)(*cap), vox["num_voxels"].data_ptr(), _ptr(vox["bev"]),
+            pg["uvd"].data_ptr(), pg["vis_mask"].data_ptr(), pg["cam"].data_ptr(), pg["gathered"].data_ptr(),
+            rd["expert"].data_ptr(), rd["offsets"].data_ptr(), rd["perm"].data_ptr(),
+            rd["points_out"].data_ptr(), rd["feat_out"].data_ptr(), self._stream())
+        self._raise(rc, "emc2_bridge_run")
         return bufs
 
     # ------------------------------------------------------------------ measurement aids

@@ -198,6 +198,12 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     h->d_tile_counts = reinterpret_cast<int*>(base + o_tc);
     h->d_tile_base = reinterpret_cast<int*>(base + o_tb);
     h->d_status = reinterpret_cast<int*>(base + o_status);
+    int prio_lo = 0, prio_hi = 0;
+    e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+    if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, prio_hi);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+    if (e != cudaSuccess) { emc2_bridge_destroy(h); return EMC2_ERR_CUDA; }
     *out = h;
     return EMC2_OK;
 }
@@ -262,6 +268,38 @@ int emc2_route_dispatch(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_p
                                  d_points_out, d_feat_out, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points, const float* d_proj,
+                    const float* d_feat, int32_t* const d_coords[2], int32_t* const d_counts[2],
+                    float* const d_mean[2], int32_t* const d_point_voxel[2], const int32_t capacity[2],
+                    int32_t* d_num_voxels, float* d_bev, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
+                    float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
+                    float* d_points_out, float* d_feat_out, void* cuda_stream) {
+    // The stage calls validate before they enqueue anything; a host-detected error in stage 2 or
+    // 3 - 4 leaves stage 1 enqueued, exactly as three separate calls would.
+    if (!h) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaEventRecord(h->ev_fork, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->side, h->ev_fork, 0);
+    if (e != cudaSuccess) return check_cuda(h, e);
+    int rc = emc2_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity, d_num_voxels,
+                           d_bev, h->side);
+    int rc2 = EMC2_OK;
+    if (rc == EMC2_OK) {
+        rc2 = emc2_project_gather(h, B, N, d_points, d_proj, d_feat, d_uvd, d_vis_mask, d_cam, d_gathered, st);
+        if (rc2 == EMC2_OK)
+            rc2 = emc2_route_dispatch(h, B, N, d_points, d_vis_mask, d_gathered, d_expert, d_offsets, d_perm,
+                                      d_points_out, d_feat_out, st);
+    }
+    // Join even after an error, so that `cuda_stream` never runs ahead of stage 1.
+    e = cudaEventRecord(h->ev_join, h->side);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, h->ev_join, 0);
+    if (rc != EMC2_OK) return rc;
+    if (rc2 != EMC2_OK) return rc2;
+    return check_cuda(h, e);
+}
+
 int emc2_bridge_status(emc2_bridge_t* h, void* cuda_stream) {
     if (!h) return EMC2_ERR_INVALID_ARG;
     DeviceGuard guard(h->cfg.device);
@@ -283,6 +321,9 @@ int emc2_bridge_destroy(emc2_bridge_t* h) {
     int rc = EMC2_OK;
     for (ProfRec& r : h->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (cudaEvent_t e : h->event_pool) cudaEventDestroy(e);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->side) cudaStreamDestroy(h->side);
     if (h->slab && cudaFree(h->slab) != cudaSuccess) rc = EMC2_ERR_CUDA;
     delete h;
     return rc;

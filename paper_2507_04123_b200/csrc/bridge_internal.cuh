@@ -103,6 +103,8 @@ struct emc2_bridge {
     int* d_scan_warp_ofs = nullptr;  // [scan_blocks * 8][3] per-warp offsets inside their CTA
     int scan_blocks = 0;           // CTAs of the cooperative rank scan (all co-resident)
     int max_tiles = 0;
+    cudaStream_t side = nullptr;   // stream of stage 1 inside emc2_bridge_run
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     int last_cuda_error = 0;
     bool profiling = false;
     int64_t launches[emc2::K_KINDS] = {0};

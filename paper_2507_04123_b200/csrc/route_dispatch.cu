@@ -4,8 +4,8 @@
 // offsets are exclusive prefix sums (Sec. 3.6).
 //
 // Three launches: (1) expert ids plus one histogram per 256-point tile, counted with warp
-// ballots; (2) a small scan that turns tile histograms into per-frame expert offsets and
-// per-tile bases; (3) one CTA per tile ranks its points inside the tile with ballots and
+// ballots; (2) a small scan, one warp per expert, that turns tile histograms into per-frame
+// expert offsets and per-tile bases; (3) one CTA per tile ranks its points inside the tile with ballots and
 // popcounts, writes the permutation and moves the 16/20-byte point rows and the 256/320-byte
 // feature rows with coalesced 128-bit accesses.
 #include <cmath>
@@ -26,77 +26,80 @@ struct RouteArgs {
     uint8_t lut[16];
 };
 
-// grid = (tiles per frame, B); tiles never straddle frames.
+constexpr int kHistTiles = 4;         // tiles one CTA of route_hist_kernel takes (independent loads per thread)
+
+// grid = (ceil(tiles per frame / kHistTiles), B); tiles never straddle frames.  Thread t takes
+// point t of each of the CTA's tiles, so its loads are independent; one histogram per tile.
 template <int C>
-__global__ void __launch_bounds__(kThreads) route_hist_kernel(RouteArgs a) {
-    __shared__ __align__(16) float sp[kTile * C];
-    __shared__ int hist[EMC2_MAX_EXPERTS];
-    const int b = blockIdx.y, tile = blockIdx.x, t = threadIdx.x;
-    const int i0 = tile * kTile;
-    const int npts = min(kTile, a.N - i0);
-    const size_t g0 = (size_t)b * a.N + i0;
-    // Frames start on a 16-byte boundary only if N*C is a multiple of 4 floats.
-    const float* src = a.pts + g0 * C;
-    if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
-        load_tile_f32(src, npts * C, sp);
-    } else {
-        for (int i = t; i < npts * C; i += kThreads) sp[i] = __ldg(src + i);
-    }
-    if (t < EMC2_MAX_EXPERTS) hist[t] = 0;
-    __syncthreads();
-    int e = -1;
-    if (t < npts) {
-        const float x = sp[t * C], y = sp[t * C + 1];
-        const float r2 = __fmaf_rn(x, x, __fmul_rn(y, y));
-        int bucket = 0;
-        for (int k = 0; k < a.T; ++k) bucket += (r2 >= a.thr2[k]) ? 1 : 0;
-        e = a.lut[(a.vis[g0 + t] != 0 ? 8 : 0) + bucket];
-        a.expert[g0 + t] = (uint8_t)e;
-    }
-    const int lane = t & 31;
-    for (int k = 0; k < a.E; ++k) {
-        const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
-        if (lane == 0 && m) atomicAdd(&hist[k], __popc(m));
+__global__ void __launch_bounds__(kThreads) route_hist_kernel(const __grid_constant__ RouteArgs a) {
+    __shared__ int hist[kHistTiles][EMC2_MAX_EXPERTS];
+    const int b = blockIdx.y, t = threadIdx.x, lane = t & 31;
+    const int tile0 = blockIdx.x * kHistTiles;
+    if (t < kHistTiles * EMC2_MAX_EXPERTS) hist[t / EMC2_MAX_EXPERTS][t % EMC2_MAX_EXPERTS] = 0;
+    float x[kHistTiles], y[kHistTiles];
+    unsigned vis[kHistTiles];
+#pragma unroll
+    for (int u = 0; u < kHistTiles; ++u) {
+        const int i = (tile0 + u) * kTile + t;
+        x[u] = y[u] = 0.0f;
+        vis[u] = 0u;
+        if (i < a.N) {
+            const size_t gi = (size_t)b * a.N + i;
+            const float2 xy = C == 4 ? *reinterpret_cast<const float2*>(a.pts + gi * 4)
+                                     : make_float2(__ldg(a.pts + gi * C), __ldg(a.pts + gi * C + 1));
+            x[u] = xy.x; y[u] = xy.y;
+            vis[u] = a.vis[gi];
+        }
     }
     __syncthreads();
-    if (t < a.E) a.tile_counts[((size_t)b * a.tiles + tile) * a.E + t] = hist[t];
+#pragma unroll
+    for (int u = 0; u < kHistTiles; ++u) {
+        const int i = (tile0 + u) * kTile + t;
+        int e = -1;
+        if (i < a.N) {
+            const float r2 = __fmaf_rn(x[u], x[u], __fmul_rn(y[u], y[u]));
+            int bucket = 0;
+            for (int k = 0; k < a.T; ++k) bucket += (r2 >= a.thr2[k]) ? 1 : 0;
+            e = a.lut[(vis[u] != 0u ? 8 : 0) + bucket];
+            a.expert[(size_t)b * a.N + i] = (uint8_t)e;
+        }
+        for (int k = 0; k < a.E; ++k) {
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
+            if (lane == 0 && m) atomicAdd(&hist[u][k], __popc(m));
+        }
+    }
+    __syncthreads();
+    if (t < kHistTiles * EMC2_MAX_EXPERTS) {
+        const int u = t / EMC2_MAX_EXPERTS, k = t % EMC2_MAX_EXPERTS;
+        if (tile0 + u < a.tiles && k < a.E)
+            a.tile_counts[((size_t)b * a.tiles + tile0 + u) * a.E + k] = hist[u][k];
+    }
 }
 
-// One CTA per frame.  For each expert: exclusive scan of its tile counts.  Then offsets.
+template <int C>
+void launch_hist(const RouteArgs& ra, int B, cudaStream_t st) {
+    const dim3 grid((ra.tiles + kHistTiles - 1) / kHistTiles, B);
+    route_hist_kernel<C><<<grid, kThreads, 0, st>>>(ra);
+}
+
+// One CTA per frame, one warp per expert at a time, no CTA barrier inside the loops.  First the
+// per-expert totals give the frame's offsets, then each warp turns its expert's tile counts into
+// exclusive bases that start at the expert's offset.
 __global__ void __launch_bounds__(kThreads)
 route_scan_kernel(const int* __restrict__ tile_counts, int* __restrict__ tile_base, int32_t* offsets,
                   int tiles, int E, int N) {
-    __shared__ int wsum[kThreads / 32];
-    __shared__ int carry;
+    constexpr int kWarps = kThreads / 32;
     __shared__ int etot[EMC2_MAX_EXPERTS + 1];
     const int b = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int* cnt = tile_counts + (size_t)b * tiles * E;
     int* base = tile_base + (size_t)b * tiles * E;
-    for (int e = 0; e < E; ++e) {
-        if (t == 0) carry = 0;
-        __syncthreads();
-        for (int s = 0; s < tiles; s += kThreads) {
-            const int i = s + t;
-            const int v = i < tiles ? cnt[(size_t)i * E + e] : 0;
-            int x = v;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
-                if (lane >= d) x += y;
-            }
-            if (lane == 31) wsum[warp] = x;
-            __syncthreads();
-            int wb = 0;
-            for (int w = 0; w < warp; ++w) wb += wsum[w];
-            const int c0 = carry;
-            if (i < tiles) base[(size_t)i * E + e] = c0 + wb + x - v;   // still relative to the expert
-            __syncthreads();
-            if (t == kThreads - 1) carry = c0 + wb + x;
-            __syncthreads();
-        }
-        if (t == 0) etot[e] = carry;
-        __syncthreads();
+    for (int e = warp; e < E; e += kWarps) {
+        int v = 0;
+        for (int i = lane; i < tiles; i += 32) v += cnt[(size_t)i * E + e];
+        v = warp_sum(v);
+        if (lane == 0) etot[e] = v;
     }
+    __syncthreads();
     if (t == 0) {
         int run = 0;
         for (int e = 0; e < E; ++e) { const int c = etot[e]; etot[e] = run; run += c; }
@@ -104,7 +107,21 @@ route_scan_kernel(const int* __restrict__ tile_counts, int* __restrict__ tile_ba
     }
     __syncthreads();
     if (t <= E) offsets[(size_t)b * (E + 1) + t] = etot[t];
-    for (int i = t; i < tiles * E; i += kThreads) base[i] += etot[i % E];
+    for (int e = warp; e < E; e += kWarps) {
+        int carry = etot[e];
+        for (int s = 0; s < tiles; s += 32) {
+            const int i = s + lane;
+            const int v = i < tiles ? cnt[(size_t)i * E + e] : 0;
+            int x = v;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
+                if (lane >= d) x += y;
+            }
+            if (i < tiles) base[(size_t)i * E + e] = carry + x - v;
+            carry += __shfl_sync(0xFFFFFFFFu, x, 31);
+        }
+    }
 }
 
 struct ScatterArgs {
@@ -214,8 +231,7 @@ int launch_route_dispatch(emc2_bridge* h, int B, int N, const float* d_points, c
     for (int k = 0; k < 16; ++k) ra.lut[k] = c.lut[k >> 3][k & 7];
     if (tiles > 0) {
         LaunchScope ls(h, K_ROUTE_HIST, st);
-        if (c.point_floats == 4) route_hist_kernel<4><<<grid, kThreads, 0, st>>>(ra);
-        else route_hist_kernel<5><<<grid, kThreads, 0, st>>>(ra);
+        if (c.point_floats == 4) launch_hist<4>(ra, B, st); else launch_hist<5>(ra, B, st);
     }
     {
         LaunchScope ls(h, K_ROUTE_SCAN, st);
@@ -320,8 +336,7 @@ extern "C" int emc2_route_dispatch_static(const emc2_config_t* config, int32_t B
             for (int k = 0; k < EMC2_MAX_THRESHOLDS; ++k)
                 ra.thr2[k] = k < c.num_thresholds ? c.thresholds[k] * c.thresholds[k] : 0.0f;
             for (int k = 0; k < 16; ++k) ra.lut[k] = c.lut[k >> 3][k & 7];
-            if (c.point_floats == 4) route_hist_kernel<4><<<grid, kThreads, 0, st>>>(ra);
-            else route_hist_kernel<5><<<grid, kThreads, 0, st>>>(ra);
+            if (c.point_floats == 4) launch_hist<4>(ra, B, st); else launch_hist<5>(ra, B, st);
         }
         route_scan_kernel<<<B, kThreads, 0, st>>>(tile_counts, tile_base, d_offsets, tiles, E, N);
         if (tiles > 0) {
