@@ -58,10 +58,22 @@ def algorithmic_bytes(w, B, N, m0, m1, texels):
 
 
 def kernel_bytes(w, B, N, texels):
-    """Algorithmic bytes of the two row-moving kernels, per launch."""
+    """Algorithmic bytes of the row-moving kernels, per launch."""
     pb, fb = 4 * w.C, 4 * w.feat_c
     return {"project_gather": B * N * pb + B * w.K * 48 + fb * texels + B * N * (12 + 1 + 1 + fb),
-            "dispatch_scatter": B * N * (1 + pb + fb) + B * N * (4 + pb + fb)}
+            "dispatch_scatter": B * N * (1 + pb + fb) + B * N * (4 + pb + fb),
+            # one-call path: reads points, uvd, camera, expert and the texels; writes the permutation,
+            # the point rows and every feature row twice (gathered and feat_out)
+            "gather_scatter": B * N * (pb + 12 + 1 + 1) + fb * texels + B * N * (4 + pb + 2 * fb)}
+
+
+def one_call_bytes(w, B, N, m0, m1, texels):
+    """Bytes the one-call path must move: as the staged count, minus the read-back of `gathered`,
+    of the mask and of the point rows that stages 3 - 4 no longer need, plus the re-read of uvd/cam."""
+    pb, fb = 4 * w.C, 4 * w.feat_c
+    staged = algorithmic_bytes(w, B, N, m0, m1, texels)
+    proj = B * N * pb + B * w.K * 48 + B * N * (12 + 1 + 1 + 1)
+    return staged["voxelize"] + proj + kernel_bytes(w, B, N, texels)["gather_scatter"] + B * (w.num_experts + 1) * 4
 
 
 def distinct_texels(w, pg):
@@ -280,8 +292,11 @@ def run_ours(args, w):
     br.profile_read(reset=True)
     br.profile_enable(True)
     prof_steps = max(3, min(args.steps, 10))
+    br.set_overlap(False)                                  # kernels one after another: clean per-kernel times
     for _ in range(prof_steps):
-        staged_step()                                      # kernels one after another: clean per-kernel times
+        step()
+    sync()
+    br.set_overlap(True)
     sync()
     prof = br.profile_read(reset=True)
     br.profile_enable(False)
@@ -326,6 +341,7 @@ def run_ours(args, w):
         "mpoints_per_s": fps * N / 1e6,
         "staged_ms_per_step": staged_secs / args.steps * 1e3,
         "bridge_algorithmic_bytes_per_step": abytes,
+        "one_call_bytes_per_step": one_call_bytes(w, B, N, int(nv[0]), int(nv[1]), texels),
         "bridge_gbs": total_gbs, "bridge_frac_of_8tbs": total_gbs / NOMINAL_HBM_GBS,
         f"bridge_frac_of_{peak_kind}_copy": total_gbs / peak,
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_source": peak_kind,

@@ -140,7 +140,9 @@ int emc2_route_dispatch(emc2_bridge_t* bridge, int32_t B, int32_t N, const float
 /* The whole bridge in one call (all four stages; Sec. 3.1 - 3.2, with the overlap of independent
  * work that Sec. 3.6 asks of the system).  Arguments, outputs, layouts and errors are exactly those
  * of emc2_voxelize, emc2_project_gather and emc2_route_dispatch called in that order with the same
- * buffers; d_vis_mask and d_gathered of stage 2 feed stages 3 - 4.  Stage 1 does not depend on
+ * buffers.  Stages 2 - 4 run as one pass: the expert id is computed beside the projection, and
+ * every feature row is blended once and stored both at its row of d_gathered and at its slot of
+ * d_feat_out, so the rows are not read back.  Stage 1 does not depend on
  * stages 2 - 4, so the library runs it on a stream of its own (created with the handle, highest
  * priority) beside them: it starts once the work already queued on `cuda_stream` has finished,
  * and `cuda_stream` waits for it before the call's work counts as complete.  Seen from
@@ -152,6 +154,11 @@ int emc2_bridge_run(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_
                     int32_t* d_num_voxels, float* d_bev, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
                     float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
                     float* d_points_out, float* d_feat_out, void* cuda_stream);
+
+/* Turns the side stream of emc2_bridge_run off (0) or on (non-zero, the default).  Off, every
+ * kernel of the call is enqueued on `cuda_stream` itself, one after another: for callers that
+ * want no second stream, and for timing kernels one at a time. */
+int emc2_bridge_set_overlap(emc2_bridge_t* bridge, int enable);
 
 /* Stages 3 and 4 for callers that must not allocate device memory (the paper has no counterpart;
  * this is a packaging variant of emc2_route_dispatch).

@@ -33,7 +33,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_status", "emc2_bridge_destroy", "emc2_status_string", "emc2_bridge_last_cuda_error",
     "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
-    "emc2_bridge_run",
+    "emc2_bridge_run", "emc2_bridge_set_overlap",
 )
 
 
@@ -80,6 +80,7 @@ def load_library() -> ctypes.CDLL:
                                     + [vp] * 4 + [vp] * 5 + [vp])
     lib.emc2_route_dispatch_static.argtypes = [P(Emc2Config), i32, i32] + [vp] * 9
     lib.emc2_bridge_status.argtypes = [vp, vp]
+    lib.emc2_bridge_set_overlap.argtypes = [vp, ctypes.c_int]
     lib.emc2_bridge_destroy.argtypes = [vp]
     lib.emc2_status_string.argtypes = [ctypes.c_int]
     lib.emc2_status_string.restype = ctypes.c_char_p
@@ -283,6 +284,10 @@ class Bridge:
                                           self._stream())
         self._raise(rc, "emc2_route_dispatch")
         return out
+
+    def set_overlap(self, enable: bool) -> None:
+        """emc2_bridge_set_overlap: stage 1 of :meth:`run` beside stages 2 - 4 (default) or after them."""
+        self._raise(self.lib.emc2_bridge_set_overlap(self._h, int(enable)), "emc2_bridge_set_overlap")
 
     def status(self, raise_on_error: bool = True) -> int:
         """emc2_bridge_status: waits for the current stream, returns the sticky device status."""

@@ -9,7 +9,7 @@ namespace emc2 {
 
 static const char* const kKernelNames[K_KINDS] = {
     "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
-    "project_gather", "route_hist", "route_scan", "dispatch_scatter"};
+    "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
     if (e == cudaSuccess) return EMC2_OK;
@@ -280,24 +280,45 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
     DeviceGuard guard(h->cfg.device);
     if (!guard.ok) return EMC2_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    cudaError_t e = cudaEventRecord(h->ev_fork, st);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->side, h->ev_fork, 0);
-    if (e != cudaSuccess) return check_cuda(h, e);
+    cudaStream_t vox_st = h->overlap ? h->side : st;
+    cudaError_t e = cudaSuccess;
+    if (h->overlap) {
+        e = cudaEventRecord(h->ev_fork, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->side, h->ev_fork, 0);
+        if (e != cudaSuccess) return check_cuda(h, e);
+    }
     int rc = emc2_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity, d_num_voxels,
-                           d_bev, h->side);
+                           d_bev, vox_st);
     int rc2 = EMC2_OK;
-    if (rc == EMC2_OK) {
-        rc2 = emc2_project_gather(h, B, N, d_points, d_proj, d_feat, d_uvd, d_vis_mask, d_cam, d_gathered, st);
-        if (rc2 == EMC2_OK)
-            rc2 = emc2_route_dispatch(h, B, N, d_points, d_vis_mask, d_gathered, d_expert, d_offsets, d_perm,
-                                      d_points_out, d_feat_out, st);
+    if (rc == EMC2_OK && B > 0) {
+        // The checks of emc2_project_gather and emc2_route_dispatch, then one pass over the rows.
+        if (!d_offsets) rc2 = EMC2_ERR_INVALID_ARG;
+        else if (N > 0 && (!d_points || !d_proj || !d_feat || !d_uvd || !d_vis_mask || !d_cam || !d_gathered ||
+                           !d_expert || !d_perm || !d_points_out || !d_feat_out))
+            rc2 = EMC2_ERR_INVALID_ARG;
+        else if (!aligned16(d_points) || !aligned16(d_feat) || !aligned16(d_gathered) || !aligned16(d_feat_out))
+            rc2 = EMC2_ERR_INVALID_ARG;
+        else if (N > 0 && (d_points_out == d_points || d_feat_out == d_gathered))
+            rc2 = EMC2_ERR_INVALID_ARG;
+        else
+            rc2 = launch_project_route_gather_dispatch(h, B, N, d_points, d_proj, d_feat, d_uvd, d_vis_mask, d_cam,
+                                                       d_gathered, d_expert, d_offsets, d_perm, d_points_out,
+                                                       d_feat_out, st);
     }
     // Join even after an error, so that `cuda_stream` never runs ahead of stage 1.
-    e = cudaEventRecord(h->ev_join, h->side);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, h->ev_join, 0);
+    if (h->overlap) {
+        e = cudaEventRecord(h->ev_join, h->side);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, h->ev_join, 0);
+    }
     if (rc != EMC2_OK) return rc;
     if (rc2 != EMC2_OK) return rc2;
     return check_cuda(h, e);
+}
+
+int emc2_bridge_set_overlap(emc2_bridge_t* h, int enable) {
+    if (!h) return EMC2_ERR_INVALID_ARG;
+    h->overlap = enable != 0;
+    return EMC2_OK;
 }
 
 int emc2_bridge_status(emc2_bridge_t* h, void* cuda_stream) {

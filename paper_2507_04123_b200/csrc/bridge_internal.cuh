@@ -25,6 +25,8 @@ enum KernelKind {
     K_VOX_ACCUM,
     K_VOX_FINALIZE,
     K_PROJECT_GATHER,
+    K_PROJECT_ROUTE,
+    K_GATHER_SCATTER,
     K_ROUTE_HIST,
     K_ROUTE_SCAN,
     K_DISPATCH_SCATTER,
@@ -83,6 +85,13 @@ struct ScaleDev {
     int* totals;            // [0] voxels, [1] cells over the cap, [2] points in cells over the cap
 };
 
+// Routing tables as the kernels take them (Sec. 3.2 distance rule, per point with visibility).
+struct RouteParams {
+    int T, E;
+    float thr2[EMC2_MAX_THRESHOLDS];    // squared thresholds
+    uint8_t lut[16];                    // [visible ? 8 : 0] + number of thresholds reached -> expert
+};
+
 struct ProfRec {
     int kind;
     cudaEvent_t a, b;
@@ -103,6 +112,7 @@ struct emc2_bridge {
     int* d_scan_warp_ofs = nullptr;  // [scan_blocks * 8][3] per-warp offsets inside their CTA
     int scan_blocks = 0;           // CTAs of the cooperative rank scan (all co-resident)
     int max_tiles = 0;
+    bool overlap = true;           // emc2_bridge_run puts stage 1 on `side`
     cudaStream_t side = nullptr;   // stream of stage 1 inside emc2_bridge_run
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     int last_cuda_error = 0;
@@ -138,6 +148,23 @@ int launch_project_gather(emc2_bridge* h, int B, int N, const float* d_points, c
 int launch_route_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const uint8_t* d_vis_mask,
                           const float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
                           float* d_points_out, float* d_feat_out, cudaStream_t st);
+
+inline RouteParams route_params(const emc2_bridge* h) {
+    RouteParams rp;
+    rp.T = h->cfg.num_thresholds;
+    rp.E = h->cfg.num_experts;
+    for (int k = 0; k < EMC2_MAX_THRESHOLDS; ++k) rp.thr2[k] = h->thr2[k];
+    for (int k = 0; k < 16; ++k) rp.lut[k] = h->cfg.lut[k >> 3][k & 7];
+    return rp;
+}
+
+// Tile histograms (handle scratch) -> d_offsets and tile bases (handle scratch).
+void launch_route_scan(emc2_bridge* h, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st);
+// Stages 2 - 4 in one pass over the feature rows (the one-call path).
+int launch_project_route_gather_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj,
+                                         const float* d_feat, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
+                                         float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
+                                         float* d_points_out, float* d_feat_out, cudaStream_t st);
 
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__

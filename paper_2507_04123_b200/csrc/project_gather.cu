@@ -40,6 +40,69 @@ __device__ __forceinline__ float4 blend(const float4& f00, const float4& f01, co
     return o;
 }
 
+// Projection of one point into the K cameras of its frame (P: [K][3][4] row-major).
+struct Projected {
+    unsigned mask;      // bit k: visible in camera k
+    int best;           // lowest visible camera, -1 if none
+    float u, v, d;      // pixel and depth in `best`; (-1, -1, depth in camera 0 or 0) if none
+};
+
+__device__ __forceinline__ Projected project_point(const float* __restrict__ P, int K, float x, float y, float z,
+                                                    int W, int H, float min_depth) {
+    Projected r;
+    r.mask = 0u; r.best = -1; r.u = -1.0f; r.v = -1.0f; r.d = 0.0f;
+    float d0 = 0.0f;
+    for (int k = 0; k < K; ++k, P += 12) {
+        // Depth first: most cameras look away from a given point.
+        const float t2 = __fmaf_rn(__ldg(P + 8), x, __fmaf_rn(__ldg(P + 9), y, __fmaf_rn(__ldg(P + 10), z, __ldg(P + 11))));
+        if (k == 0) d0 = t2;
+        if (!(t2 > min_depth)) continue;
+        const float t0 = __fmaf_rn(__ldg(P + 0), x, __fmaf_rn(__ldg(P + 1), y, __fmaf_rn(__ldg(P + 2), z, __ldg(P + 3))));
+        const float t1 = __fmaf_rn(__ldg(P + 4), x, __fmaf_rn(__ldg(P + 5), y, __fmaf_rn(__ldg(P + 6), z, __ldg(P + 7))));
+        const float u = __fdiv_rn(t0, t2), v = __fdiv_rn(t1, t2);
+        if (!((u >= 0.0f) && (u < (float)W) && (v >= 0.0f) && (v < (float)H))) continue;
+        r.mask |= 1u << k;
+        if (r.best < 0) { r.best = k; r.u = u; r.v = v; r.d = t2; }
+    }
+    if (r.best < 0) r.d = isfinite(d0) ? d0 : 0.0f;
+    return r;
+}
+
+// Tap record of a point seen by camera `cam` of frame b at pixel (u, v): {float4 index of tap
+// (y0, x0), clamp flags, wx, wy}; kZeroRow in .x for a point no camera sees.
+__device__ __forceinline__ uint4 tap_record(int b, int cam, float u, float v, int K, int Hf, int Wf, int cf4,
+                                            float inv_stride) {
+    uint4 rec = make_uint4(kZeroRow, 0u, 0u, 0u);
+    if (cam >= 0) {
+        // Texel coordinates: the stride is a power of two, so the scaling is exact.
+        const float fx = u * inv_stride, fy = v * inv_stride;
+        const float flx = floorf(fx), fly = floorf(fy);
+        int x0 = (int)flx, y0 = (int)fly;
+        const int x1 = min(x0 + 1, Wf - 1), y1 = min(y0 + 1, Hf - 1);
+        x0 = min(x0, Wf - 1);
+        y0 = min(y0, Hf - 1);
+        const uint32_t map = ((uint32_t)b * K + cam) * Hf;
+        rec.x = ((map + y0) * Wf + x0) * (uint32_t)cf4;
+        rec.y = (uint32_t)(x1 - x0) | ((uint32_t)(y1 - y0) << 1);
+        rec.z = __float_as_uint(fx - flx);
+        rec.w = __float_as_uint(fy - fly);
+    }
+    return rec;
+}
+
+// Blended feature column c of the row described by `rec` (zeros for kZeroRow).
+__device__ __forceinline__ float4 gather_column(const float4* __restrict__ feat, const uint4& rec, int c, uint32_t cf4,
+                                                uint32_t row_stride) {
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (rec.x != kZeroRow) {
+        const float4* p = feat + rec.x + c;
+        const uint32_t dx = (rec.y & 1u) ? cf4 : 0u, dy = (rec.y & 2u) ? row_stride : 0u;
+        const float4 f00 = __ldg(p), f01 = __ldg(p + dx), f10 = __ldg(p + dy), f11 = __ldg(p + dy + dx);
+        o = blend(f00, f01, f10, f11, __uint_as_float(rec.z), __uint_as_float(rec.w));
+    }
+    return o;
+}
+
 // CF4 > 0: Cf/4 known at compile time, blockDim.x == 16 * CF4.  CF4 == 0: any Cf, 256 threads.
 template <int C, int CF4>
 __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) project_gather_kernel(PgArgs a) {
@@ -58,41 +121,11 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) project_gather_
         const float x = sp[t * C], y = sp[t * C + 1], z = sp[t * C + 2];
         const long long gi = g0 + t;
         const int b = (int)(gi / a.N);
-        const float* P = a.proj + (size_t)b * a.K * 12;
-        unsigned mask = 0;
-        int best = -1;
-        float bu = -1.0f, bv = -1.0f, bd = 0.0f, d0 = 0.0f;
-        for (int k = 0; k < a.K; ++k, P += 12) {
-            const float t0 = __fmaf_rn(__ldg(P + 0), x, __fmaf_rn(__ldg(P + 1), y, __fmaf_rn(__ldg(P + 2), z, __ldg(P + 3))));
-            const float t1 = __fmaf_rn(__ldg(P + 4), x, __fmaf_rn(__ldg(P + 5), y, __fmaf_rn(__ldg(P + 6), z, __ldg(P + 7))));
-            const float t2 = __fmaf_rn(__ldg(P + 8), x, __fmaf_rn(__ldg(P + 9), y, __fmaf_rn(__ldg(P + 10), z, __ldg(P + 11))));
-            if (k == 0) d0 = t2;
-            if (!(t2 > a.min_depth)) continue;
-            const float u = __fdiv_rn(t0, t2), v = __fdiv_rn(t1, t2);
-            const bool vis = (u >= 0.0f) && (u < (float)a.W) && (v >= 0.0f) && (v < (float)a.H);
-            if (!vis) continue;
-            mask |= 1u << k;
-            if (best < 0) { best = k; bu = u; bv = v; bd = t2; }
-        }
-        if (best < 0) bd = isfinite(d0) ? d0 : 0.0f;
-        suvd[t * 3] = bu; suvd[t * 3 + 1] = bv; suvd[t * 3 + 2] = bd;
-        a.vis[gi] = (uint8_t)mask;
-        a.cam[gi] = (int8_t)best;
-        uint4 rec = make_uint4(kZeroRow, 0u, 0u, 0u);
-        if (best >= 0) {
-            // Texel coordinates: stride is a power of two, so the scaling is exact.
-            const float fx = bu * a.inv_stride, fy = bv * a.inv_stride;
-            const float flx = floorf(fx), fly = floorf(fy);
-            int x0 = (int)flx, y0 = (int)fly;
-            const int x1 = min(x0 + 1, a.Wf - 1), y1 = min(y0 + 1, a.Hf - 1);
-            x0 = min(x0, a.Wf - 1);
-            y0 = min(y0, a.Hf - 1);
-            const uint32_t map = ((uint32_t)b * a.K + best) * a.Hf;
-            rec.x = ((map + y0) * a.Wf + x0) * (uint32_t)cf4;
-            rec.y = (uint32_t)(x1 - x0) | ((uint32_t)(y1 - y0) << 1);
-            rec.z = __float_as_uint(fx - flx);
-            rec.w = __float_as_uint(fy - fly);
-        }
+        const Projected pr = project_point(a.proj + (size_t)b * a.K * 12, a.K, x, y, z, a.W, a.H, a.min_depth);
+        suvd[t * 3] = pr.u; suvd[t * 3 + 1] = pr.v; suvd[t * 3 + 2] = pr.d;
+        a.vis[gi] = (uint8_t)pr.mask;
+        a.cam[gi] = (int8_t)pr.best;
+        const uint4 rec = tap_record(b, pr.best, pr.u, pr.v, a.K, a.Hf, a.Wf, cf4, a.inv_stride);
         srow[t] = rec;
     }
     __syncthreads();
@@ -108,30 +141,170 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) project_gather_
         for (int j = 0; j < kTile / 16; ++j) {
             const int r = r0 + 16 * j;
             if (r >= npts) break;
-            const uint4 rec = srow[r];
-            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (rec.x != kZeroRow) {
-                const float4* p = a.feat + rec.x + c;
-                const uint32_t dx = (rec.y & 1u) ? (uint32_t)CF4 : 0u, dy = (rec.y & 2u) ? dyv : 0u;
-                const float4 f00 = __ldg(p), f01 = __ldg(p + dx), f10 = __ldg(p + dy), f11 = __ldg(p + dy + dx);
-                o = blend(f00, f01, f10, f11, __uint_as_float(rec.z), __uint_as_float(rec.w));
-            }
-            __stcs(out + r * CF4 + c, o);
+            __stcs(out + r * CF4 + c, gather_column(a.feat, srow[r], c, (uint32_t)CF4, dyv));
         }
     } else {
         const int items = npts * cf4;
         for (int i = t; i < items; i += blockDim.x) {
             const int r = i / cf4, c = i - r * cf4;
-            const uint4 rec = srow[r];
-            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (rec.x != kZeroRow) {
-                const float4* p = a.feat + rec.x + c;
-                const uint32_t dx = (rec.y & 1u) ? (uint32_t)cf4 : 0u, dy = (rec.y & 2u) ? dyv : 0u;
-                const float4 f00 = __ldg(p), f01 = __ldg(p + dx), f10 = __ldg(p + dy), f11 = __ldg(p + dy + dx);
-                o = blend(f00, f01, f10, f11, __uint_as_float(rec.z), __uint_as_float(rec.w));
-            }
-            __stcs(out + i, o);
+            __stcs(out + i, gather_column(a.feat, srow[r], c, (uint32_t)cf4, dyv));
         }
+    }
+}
+
+// ------------------------------------------------------------------ stages 2 - 4 in one pass
+// The one-call path (emc2_bridge_run) does not send the gathered rows through memory twice.
+//   project_route   per 256-point tile of a frame: projection, mask, camera, uvd, and - since the
+//                   mask is now known - the expert id and the tile's expert histogram.
+//   route_scan      tile histograms -> frame offsets and tile bases (shared with the staged path).
+//   gather_scatter  per tile: stable rank of every point inside its expert's segment, then each
+//                   feature row is blended once and stored twice, at its own row of `gathered`
+//                   and at its slot of `feat_out`; point rows and the permutation go along.
+// Outputs are those of the staged calls, bit for bit.
+struct PrArgs {
+    const float* pts;
+    const float* proj;
+    float* uvd;
+    uint8_t* vis;
+    int8_t* cam;
+    uint8_t* expert;
+    int* tile_counts;     // [B, tiles, E]
+    int N, tiles, K, H, W;
+    float min_depth;
+    RouteParams rp;
+};
+
+// grid = (tiles per frame, B); tiles never straddle frames.
+template <int C>
+__global__ void __launch_bounds__(kThreads) project_route_kernel(const __grid_constant__ PrArgs a) {
+    __shared__ float suvd[kTile * 3];
+    __shared__ int hist[EMC2_MAX_EXPERTS];
+    const int b = blockIdx.y, tile = blockIdx.x, t = threadIdx.x, lane = t & 31;
+    const int i0 = tile * kTile;
+    const int npts = min(kTile, a.N - i0);
+    const size_t g0 = (size_t)b * a.N + i0;
+    if (t < EMC2_MAX_EXPERTS) hist[t] = 0;
+    int e = -1;
+    if (t < npts) {
+        const float* p = a.pts + (g0 + t) * C;
+        float x, y, z;
+        if (C == 4) {
+            const float4 q = __ldg(reinterpret_cast<const float4*>(p));
+            x = q.x; y = q.y; z = q.z;
+        } else {
+            x = __ldg(p); y = __ldg(p + 1); z = __ldg(p + 2);
+        }
+        const Projected pr = project_point(a.proj + (size_t)b * a.K * 12, a.K, x, y, z, a.W, a.H, a.min_depth);
+        suvd[t * 3] = pr.u; suvd[t * 3 + 1] = pr.v; suvd[t * 3 + 2] = pr.d;
+        a.vis[g0 + t] = (uint8_t)pr.mask;
+        a.cam[g0 + t] = (int8_t)pr.best;
+        const float r2 = __fmaf_rn(x, x, __fmul_rn(y, y));
+        int bucket = 0;
+        for (int k = 0; k < a.rp.T; ++k) bucket += (r2 >= a.rp.thr2[k]) ? 1 : 0;
+        e = a.rp.lut[(pr.mask != 0u ? 8 : 0) + bucket];
+        a.expert[g0 + t] = (uint8_t)e;
+    }
+    __syncthreads();
+    for (int i = t; i < npts * 3; i += kThreads) a.uvd[g0 * 3 + i] = suvd[i];
+    for (int k = 0; k < a.rp.E; ++k) {
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
+        if (lane == 0 && m) atomicAdd(&hist[k], __popc(m));
+    }
+    __syncthreads();
+    if (t < a.rp.E) a.tile_counts[((size_t)b * a.tiles + tile) * a.rp.E + t] = hist[t];
+}
+
+struct GsArgs {
+    const float* pts;
+    const float* uvd;
+    const int8_t* cam;
+    const uint8_t* expert;
+    const int* tile_base;     // [B, tiles, E]
+    const float4* feat;
+    int32_t* perm;
+    float* pts_out;
+    float4* gathered;
+    float4* feat_out;
+    int N, tiles, E, K, Hf, Wf, cf4;
+    float inv_stride;
+};
+
+// CF4 > 0: Cf/4 known at compile time, blockDim.x == 16 * CF4.  CF4 == 0: any Cf, 256 threads.
+template <int C, int CF4>
+__global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) gather_scatter_kernel(const __grid_constant__ GsArgs a) {
+    __shared__ uint4 srow[kTile];
+    __shared__ int sdest[kTile];
+    __shared__ int wcnt[kTile / 32][EMC2_MAX_EXPERTS];
+    const int b = blockIdx.y, tile = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int i0 = tile * kTile;
+    const int npts = min(kTile, a.N - i0);
+    const size_t f0 = (size_t)b * a.N;        // first row of the frame
+    const size_t g0 = f0 + i0;
+    const int cf4 = CF4 > 0 ? CF4 : a.cf4;
+
+    // Stable rank inside the tile by ballots per expert, and the tap record of every point.
+    int e = -1, rank = 0;
+    if (t < kTile) {
+        if (t < npts) {
+            e = (int)a.expert[g0 + t];
+            const float u = a.uvd[(g0 + t) * 3], v = a.uvd[(g0 + t) * 3 + 1];
+            srow[t] = tap_record(b, (int)a.cam[g0 + t], u, v, a.K, a.Hf, a.Wf, cf4, a.inv_stride);
+        }
+        for (int k = 0; k < a.E; ++k) {
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
+            if (e == k) rank = __popc(m & ((1u << lane) - 1u));
+            if (lane == 0) wcnt[warp][k] = __popc(m);
+        }
+    }
+    __syncthreads();
+    if (t < npts) {
+        int before = 0;
+        for (int w = 0; w < warp; ++w) before += wcnt[w][e];
+        const int d = a.tile_base[((size_t)b * a.tiles + tile) * a.E + e] + before + rank;
+        sdest[t] = d;
+        a.perm[f0 + d] = i0 + t;
+    }
+    __syncthreads();
+
+    // Point rows: the tile's source floats are contiguous.
+    const float* psrc = a.pts + g0 * C;
+    float* pdst = a.pts_out + f0 * C;
+    for (int i = t; i < npts * C; i += blockDim.x) {
+        const int r = i / C, c = i - r * C;
+        pdst[(size_t)sdest[r] * C + c] = __ldg(psrc + i);
+    }
+    // Feature rows: 16 rows x Cf/4 columns of threads; blended once, stored at both places.
+    float4* out = a.gathered + g0 * cf4;
+    float4* fdst = a.feat_out + f0 * cf4;
+    const uint32_t dyv = (uint32_t)a.Wf * cf4;
+    if (CF4 > 0) {
+        const int c = t % CF4, r0 = t / CF4;
+#pragma unroll 4
+        for (int j = 0; j < kTile / 16; ++j) {
+            const int r = r0 + 16 * j;
+            if (r >= npts) break;
+            const float4 o = gather_column(a.feat, srow[r], c, (uint32_t)CF4, dyv);
+            __stcs(out + r * CF4 + c, o);
+            __stcs(fdst + (size_t)sdest[r] * CF4 + c, o);
+        }
+    } else {
+        const int items = npts * cf4;
+        for (int i = t; i < items; i += blockDim.x) {
+            const int r = i / cf4, c = i - r * cf4;
+            const float4 o = gather_column(a.feat, srow[r], c, (uint32_t)cf4, dyv);
+            __stcs(out + i, o);
+            __stcs(fdst + (size_t)sdest[r] * cf4 + c, o);
+        }
+    }
+}
+
+template <int C>
+void launch_gs(emc2_bridge* h, const GsArgs& a, dim3 grid, cudaStream_t st) {
+    LaunchScope ls(h, K_GATHER_SCATTER, st);
+    switch (a.cf4) {
+        case 16: gather_scatter_kernel<C, 16><<<grid, 16 * 16, 0, st>>>(a); break;
+        case 20: gather_scatter_kernel<C, 20><<<grid, 16 * 20, 0, st>>>(a); break;
+        default: gather_scatter_kernel<C, 0><<<grid, kThreads, 0, st>>>(a); break;
     }
 }
 
@@ -162,6 +335,39 @@ int launch_project_gather(emc2_bridge* h, int B, int N, const float* d_points, c
     const int tiles = (int)((a.total + kTile - 1) / kTile);
     if (tiles == 0) return EMC2_OK;
     if (c.point_floats == 4) launch_c<4>(h, a, tiles, st); else launch_c<5>(h, a, tiles, st);
+    return check_cuda(h, cudaGetLastError());
+}
+
+int launch_project_route_gather_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj,
+                                         const float* d_feat, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
+                                         float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
+                                         float* d_points_out, float* d_feat_out, cudaStream_t st) {
+    const emc2_config_t& c = h->cfg;
+    if (B == 0) return EMC2_OK;
+    const int tiles = (N + kTile - 1) / kTile;
+    const dim3 grid(tiles > 0 ? tiles : 1, B);
+    if (tiles > 0) {
+        PrArgs pa;
+        pa.pts = d_points; pa.proj = d_proj; pa.uvd = d_uvd; pa.vis = d_vis_mask; pa.cam = d_cam;
+        pa.expert = d_expert; pa.tile_counts = h->d_tile_counts;
+        pa.N = N; pa.tiles = tiles; pa.K = c.num_cameras; pa.H = c.img_h; pa.W = c.img_w;
+        pa.min_depth = c.min_depth;
+        pa.rp = route_params(h);
+        LaunchScope ls(h, K_PROJECT_ROUTE, st);
+        if (c.point_floats == 4) project_route_kernel<4><<<grid, kThreads, 0, st>>>(pa);
+        else project_route_kernel<5><<<grid, kThreads, 0, st>>>(pa);
+    }
+    launch_route_scan(h, B, tiles, N, d_offsets, st);
+    if (tiles > 0) {
+        GsArgs ga;
+        ga.pts = d_points; ga.uvd = d_uvd; ga.cam = d_cam; ga.expert = d_expert; ga.tile_base = h->d_tile_base;
+        ga.feat = reinterpret_cast<const float4*>(d_feat); ga.perm = d_perm; ga.pts_out = d_points_out;
+        ga.gathered = reinterpret_cast<float4*>(d_gathered); ga.feat_out = reinterpret_cast<float4*>(d_feat_out);
+        ga.N = N; ga.tiles = tiles; ga.E = c.num_experts; ga.K = c.num_cameras; ga.Hf = c.feat_h; ga.Wf = c.feat_w;
+        ga.cf4 = c.feat_c / 4;
+        ga.inv_stride = 1.0f / (float)c.feat_stride;
+        if (c.point_floats == 4) launch_gs<4>(h, ga, grid, st); else launch_gs<5>(h, ga, grid, st);
+    }
     return check_cuda(h, cudaGetLastError());
 }
 

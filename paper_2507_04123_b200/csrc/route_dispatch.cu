@@ -216,6 +216,11 @@ void launch_scatter(emc2_bridge* h, const ScatterArgs& a, dim3 grid, cudaStream_
 
 }  // namespace
 
+void launch_route_scan(emc2_bridge* h, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st) {
+    LaunchScope ls(h, K_ROUTE_SCAN, st);
+    route_scan_kernel<<<B, kThreads, 0, st>>>(h->d_tile_counts, h->d_tile_base, d_offsets, tiles, h->cfg.num_experts, N);
+}
+
 int launch_route_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const uint8_t* d_vis_mask,
                           const float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
                           float* d_points_out, float* d_feat_out, cudaStream_t st) {
