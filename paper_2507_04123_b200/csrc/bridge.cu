@@ -242,7 +242,8 @@ int emc2_project_gather(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_p
     if (B == 0 || N == 0) return EMC2_OK;   // nothing to write
     if (!d_points || !d_proj || !d_feat || !d_uvd || !d_vis_mask || !d_cam || !d_gathered)
         return EMC2_ERR_INVALID_ARG;
-    if (!aligned16(d_points) || !aligned16(d_feat) || !aligned16(d_gathered)) return EMC2_ERR_INVALID_ARG;
+    if (!aligned16(d_points) || !aligned16(d_proj) || !aligned16(d_feat) || !aligned16(d_gathered))
+        return EMC2_ERR_INVALID_ARG;
     DeviceGuard guard(h->cfg.device);
     if (!guard.ok) return EMC2_ERR_CUDA;
     return launch_project_gather(h, B, N, d_points, d_proj, d_feat, d_uvd, d_vis_mask, d_cam, d_gathered,
@@ -296,7 +297,8 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
         else if (N > 0 && (!d_points || !d_proj || !d_feat || !d_uvd || !d_vis_mask || !d_cam || !d_gathered ||
                            !d_expert || !d_perm || !d_points_out || !d_feat_out))
             rc2 = EMC2_ERR_INVALID_ARG;
-        else if (!aligned16(d_points) || !aligned16(d_feat) || !aligned16(d_gathered) || !aligned16(d_feat_out))
+        else if (!aligned16(d_points) || !aligned16(d_proj) || !aligned16(d_feat) || !aligned16(d_gathered) ||
+                 !aligned16(d_feat_out))
             rc2 = EMC2_ERR_INVALID_ARG;
         else if (N > 0 && (d_points_out == d_points || d_feat_out == d_gathered))
             rc2 = EMC2_ERR_INVALID_ARG;

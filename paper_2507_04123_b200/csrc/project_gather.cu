@@ -47,25 +47,52 @@ struct Projected {
     float u, v, d;      // pixel and depth in `best`; (-1, -1, depth in camera 0 or 0) if none
 };
 
-__device__ __forceinline__ Projected project_point(const float* __restrict__ P, int K, float x, float y, float z,
+// `P` points to the frame's matrices as float4 rows in shared memory.  The visibility decision is
+// the one of the plain definition (fp32 fma chains, IEEE divide, compare), but the divide is only
+// executed where it can matter: comparing the numerators with bounds scaled by the depth settles
+// every pixel that is not within 0.01 px of an image edge, and only the chosen camera's (u, v) is
+// divided out.  A warp of scattered points therefore does not walk the divide once per camera.
+__device__ __forceinline__ Projected project_point(const float4* P, int K, float x, float y, float z,
                                                     int W, int H, float min_depth) {
     Projected r;
     r.mask = 0u; r.best = -1; r.u = -1.0f; r.v = -1.0f; r.d = 0.0f;
-    float d0 = 0.0f;
-    for (int k = 0; k < K; ++k, P += 12) {
-        // Depth first: most cameras look away from a given point.
-        const float t2 = __fmaf_rn(__ldg(P + 8), x, __fmaf_rn(__ldg(P + 9), y, __fmaf_rn(__ldg(P + 10), z, __ldg(P + 11))));
+    float d0 = 0.0f, b0 = 0.0f, b1 = 0.0f;
+    const float fw = (float)W, fh = (float)H;
+    for (int k = 0; k < K; ++k) {
+        const float4 p0 = P[3 * k], p1 = P[3 * k + 1], p2 = P[3 * k + 2];
+        const float t2 = __fmaf_rn(p2.x, x, __fmaf_rn(p2.y, y, __fmaf_rn(p2.z, z, p2.w)));
+        const float t0 = __fmaf_rn(p0.x, x, __fmaf_rn(p0.y, y, __fmaf_rn(p0.z, z, p0.w)));
+        const float t1 = __fmaf_rn(p1.x, x, __fmaf_rn(p1.y, y, __fmaf_rn(p1.z, z, p1.w)));
         if (k == 0) d0 = t2;
-        if (!(t2 > min_depth)) continue;
-        const float t0 = __fmaf_rn(__ldg(P + 0), x, __fmaf_rn(__ldg(P + 1), y, __fmaf_rn(__ldg(P + 2), z, __ldg(P + 3))));
-        const float t1 = __fmaf_rn(__ldg(P + 4), x, __fmaf_rn(__ldg(P + 5), y, __fmaf_rn(__ldg(P + 6), z, __ldg(P + 7))));
-        const float u = __fdiv_rn(t0, t2), v = __fdiv_rn(t1, t2);
-        if (!((u >= 0.0f) && (u < (float)W) && (v >= 0.0f) && (v < (float)H))) continue;
-        r.mask |= 1u << k;
-        if (r.best < 0) { r.best = k; r.u = u; r.v = v; r.d = t2; }
+        const bool front = t2 > min_depth;        // false for NaN
+        // 0.001 < u < W - 0.01 and the like, multiplied through by the (positive) depth.
+        const float lo = t2 * 1e-3f, hx = t2 * (fw - 1e-2f), hy = t2 * (fh - 1e-2f);
+        const float ox = t2 * (fw + 1e-2f), oy = t2 * (fh + 1e-2f);
+        const bool in_sure = (t0 > lo) && (t0 < hx) && (t1 > lo) && (t1 < hy);
+        const bool out_sure = (t0 < -lo) || (t0 > ox) || (t1 < -lo) || (t1 > oy);
+        bool vis = front && in_sure;
+        if (front && !in_sure && !out_sure) {     // within a hair of an edge, or not finite: decide exactly
+            const float u = __fdiv_rn(t0, t2), v = __fdiv_rn(t1, t2);
+            vis = (u >= 0.0f) && (u < fw) && (v >= 0.0f) && (v < fh);
+        }
+        if (vis) {
+            r.mask |= 1u << k;
+            if (r.best < 0) { r.best = k; b0 = t0; b1 = t1; r.d = t2; }
+        }
     }
-    if (r.best < 0) r.d = isfinite(d0) ? d0 : 0.0f;
+    if (r.best >= 0) {
+        r.u = __fdiv_rn(b0, r.d);
+        r.v = __fdiv_rn(b1, r.d);
+    } else {
+        r.d = isfinite(d0) ? d0 : 0.0f;
+    }
     return r;
+}
+
+// Copies the K 3x4 matrices of frame b into shared memory (K * 3 float4 rows).
+__device__ __forceinline__ void load_proj(const float* __restrict__ proj, int b, int K, float4* sP) {
+    const float4* src = reinterpret_cast<const float4*>(proj) + (size_t)b * K * 3;
+    for (int i = threadIdx.x; i < K * 3; i += blockDim.x) sP[i] = __ldg(src + i);
 }
 
 // Tap record of a point seen by camera `cam` of frame b at pixel (u, v): {float4 index of tap
@@ -109,10 +136,17 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) project_gather_
     __shared__ __align__(16) float sp[kTile * C];
     __shared__ float suvd[kTile * 3];
     __shared__ uint4 srow[kTile];          // {tap (y0,x0) as a float4 index, clamp flags, wx, wy}
+    __shared__ float4 sP[2][EMC2_MAX_CAMERAS * 3];   // matrices of the (at most two, if N >= 256) frames of the tile
 
     const long long g0 = (long long)blockIdx.x * kTile;
     const int npts = (int)min((long long)kTile, a.total - g0);
     load_tile_f32(a.pts + g0 * C, npts * C, sp);
+    const int bfirst = (int)(g0 / a.N);
+    const int nframes = (int)((g0 + npts - 1) / a.N) - bfirst + 1;
+    if (nframes <= 2) {
+        load_proj(a.proj, bfirst, a.K, sP[0]);
+        if (nframes == 2) load_proj(a.proj, bfirst + 1, a.K, sP[1]);
+    }
     __syncthreads();
 
     const int t = threadIdx.x;
@@ -121,7 +155,9 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) project_gather_
         const float x = sp[t * C], y = sp[t * C + 1], z = sp[t * C + 2];
         const long long gi = g0 + t;
         const int b = (int)(gi / a.N);
-        const Projected pr = project_point(a.proj + (size_t)b * a.K * 12, a.K, x, y, z, a.W, a.H, a.min_depth);
+        // Tiny frames (N < 256) can put more than two frames in a tile: read those from global memory.
+        const float4* P = nframes <= 2 ? sP[b - bfirst] : reinterpret_cast<const float4*>(a.proj) + (size_t)b * a.K * 3;
+        const Projected pr = project_point(P, a.K, x, y, z, a.W, a.H, a.min_depth);
         suvd[t * 3] = pr.u; suvd[t * 3 + 1] = pr.v; suvd[t * 3 + 2] = pr.d;
         a.vis[gi] = (uint8_t)pr.mask;
         a.cam[gi] = (int8_t)pr.best;
@@ -179,11 +215,14 @@ template <int C>
 __global__ void __launch_bounds__(kThreads) project_route_kernel(const __grid_constant__ PrArgs a) {
     __shared__ float suvd[kTile * 3];
     __shared__ int hist[EMC2_MAX_EXPERTS];
+    __shared__ float4 sP[EMC2_MAX_CAMERAS * 3];
     const int b = blockIdx.y, tile = blockIdx.x, t = threadIdx.x, lane = t & 31;
+    load_proj(a.proj, b, a.K, sP);
     const int i0 = tile * kTile;
     const int npts = min(kTile, a.N - i0);
     const size_t g0 = (size_t)b * a.N + i0;
     if (t < EMC2_MAX_EXPERTS) hist[t] = 0;
+    __syncthreads();
     int e = -1;
     if (t < npts) {
         const float* p = a.pts + (g0 + t) * C;
@@ -194,7 +233,7 @@ __global__ void __launch_bounds__(kThreads) project_route_kernel(const __grid_co
         } else {
             x = __ldg(p); y = __ldg(p + 1); z = __ldg(p + 2);
         }
-        const Projected pr = project_point(a.proj + (size_t)b * a.K * 12, a.K, x, y, z, a.W, a.H, a.min_depth);
+        const Projected pr = project_point(sP, a.K, x, y, z, a.W, a.H, a.min_depth);
         suvd[t * 3] = pr.u; suvd[t * 3 + 1] = pr.v; suvd[t * 3 + 2] = pr.d;
         a.vis[g0 + t] = (uint8_t)pr.mask;
         a.cam[g0 + t] = (int8_t)pr.best;

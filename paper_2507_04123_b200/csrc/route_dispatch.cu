@@ -4,7 +4,7 @@
 // offsets are exclusive prefix sums (Sec. 3.6).
 //
 // Three launches: (1) expert ids plus one histogram per 256-point tile, counted with warp
-// ballots; (2) a small scan, one warp per expert, that turns tile histograms into per-frame
+// ballots; (2) a small scan, one CTA per frame, that turns tile histograms into per-frame
 // expert offsets and per-tile bases; (3) one CTA per tile ranks its points inside the tile with ballots and
 // popcounts, writes the permutation and moves the 16/20-byte point rows and the 256/320-byte
 // feature rows with coalesced 128-bit accesses.
@@ -82,44 +82,72 @@ void launch_hist(const RouteArgs& ra, int B, cudaStream_t st) {
     route_hist_kernel<C><<<grid, kThreads, 0, st>>>(ra);
 }
 
-// One CTA per frame, one warp per expert at a time, no CTA barrier inside the loops.  First the
-// per-expert totals give the frame's offsets, then each warp turns its expert's tile counts into
-// exclusive bases that start at the expert's offset.
-__global__ void __launch_bounds__(kThreads)
+constexpr int kScanThreads = 1024;
+
+// One CTA of 1024 threads per frame.  Every thread owns a run of consecutive tiles and loads all
+// their counts up front; per expert, a CTA-wide exclusive scan of the run totals gives the run's
+// base, the expert totals give the frame's offsets, and the bases are written in one sweep.
+__global__ void __launch_bounds__(kScanThreads)
 route_scan_kernel(const int* __restrict__ tile_counts, int* __restrict__ tile_base, int32_t* offsets,
                   int tiles, int E, int N) {
-    constexpr int kWarps = kThreads / 32;
+    constexpr int kWarps = kScanThreads / 32;
+    __shared__ int wsum[EMC2_MAX_EXPERTS][kWarps];
     __shared__ int etot[EMC2_MAX_EXPERTS + 1];
     const int b = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int* cnt = tile_counts + (size_t)b * tiles * E;
     int* base = tile_base + (size_t)b * tiles * E;
-    for (int e = warp; e < E; e += kWarps) {
-        int v = 0;
-        for (int i = lane; i < tiles; i += 32) v += cnt[(size_t)i * E + e];
-        v = warp_sum(v);
-        if (lane == 0) etot[e] = v;
+    const int per = (tiles + kScanThreads - 1) / kScanThreads;
+    const int lo = min(tiles, t * per), hi = min(tiles, lo + per);
+    int run[EMC2_MAX_EXPERTS];            // this thread's total, then its exclusive base, per expert
+#pragma unroll
+    for (int e = 0; e < EMC2_MAX_EXPERTS; ++e) run[e] = 0;
+    for (int i = lo; i < hi; ++i) {
+#pragma unroll
+        for (int e = 0; e < EMC2_MAX_EXPERTS; ++e)
+            if (e < E) run[e] += cnt[(size_t)i * E + e];
+    }
+#pragma unroll
+    for (int e = 0; e < EMC2_MAX_EXPERTS; ++e) {
+        if (e >= E) break;
+        int x = run[e];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
+            if (lane >= d) x += y;
+        }
+        if (lane == 31) wsum[e][warp] = x;
+        run[e] = x - run[e];              // exclusive inside the warp
+    }
+    __syncthreads();
+    if (warp < E) {                       // warp e scans the warp totals of expert e
+        int x = wsum[warp][lane];
+        const int v = x;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
+            if (lane >= d) x += y;
+        }
+        wsum[warp][lane] = x - v;
+        if (lane == 31) etot[warp] = x;
     }
     __syncthreads();
     if (t == 0) {
-        int run = 0;
-        for (int e = 0; e < E; ++e) { const int c = etot[e]; etot[e] = run; run += c; }
-        etot[E] = run;
+        int acc = 0;
+        for (int e = 0; e < E; ++e) { const int c = etot[e]; etot[e] = acc; acc += c; }
+        etot[E] = acc;
     }
     __syncthreads();
     if (t <= E) offsets[(size_t)b * (E + 1) + t] = etot[t];
-    for (int e = warp; e < E; e += kWarps) {
-        int carry = etot[e];
-        for (int s = 0; s < tiles; s += 32) {
-            const int i = s + lane;
-            const int v = i < tiles ? cnt[(size_t)i * E + e] : 0;
-            int x = v;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
-                if (lane >= d) x += y;
+    for (int e = 0; e < EMC2_MAX_EXPERTS; ++e)
+        if (e < E) run[e] += etot[e] + wsum[e][warp];
+    for (int i = lo; i < hi; ++i) {
+#pragma unroll
+        for (int e = 0; e < EMC2_MAX_EXPERTS; ++e) {
+            if (e < E) {
+                base[(size_t)i * E + e] = run[e];
+                run[e] += cnt[(size_t)i * E + e];
             }
-            if (i < tiles) base[(size_t)i * E + e] = carry + x - v;
-            carry += __shfl_sync(0xFFFFFFFFu, x, 31);
         }
     }
 }
@@ -218,7 +246,7 @@ void launch_scatter(emc2_bridge* h, const ScatterArgs& a, dim3 grid, cudaStream_
 
 void launch_route_scan(emc2_bridge* h, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st) {
     LaunchScope ls(h, K_ROUTE_SCAN, st);
-    route_scan_kernel<<<B, kThreads, 0, st>>>(h->d_tile_counts, h->d_tile_base, d_offsets, tiles, h->cfg.num_experts, N);
+    route_scan_kernel<<<B, kScanThreads, 0, st>>>(h->d_tile_counts, h->d_tile_base, d_offsets, tiles, h->cfg.num_experts, N);
 }
 
 int launch_route_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const uint8_t* d_vis_mask,
@@ -240,7 +268,7 @@ int launch_route_dispatch(emc2_bridge* h, int B, int N, const float* d_points, c
     }
     {
         LaunchScope ls(h, K_ROUTE_SCAN, st);
-        route_scan_kernel<<<B, kThreads, 0, st>>>(h->d_tile_counts, h->d_tile_base, d_offsets, tiles, E, N);
+        route_scan_kernel<<<B, kScanThreads, 0, st>>>(h->d_tile_counts, h->d_tile_base, d_offsets, tiles, E, N);
     }
     if (tiles > 0) {
         ScatterArgs sa;
@@ -343,7 +371,7 @@ extern "C" int emc2_route_dispatch_static(const emc2_config_t* config, int32_t B
             for (int k = 0; k < 16; ++k) ra.lut[k] = c.lut[k >> 3][k & 7];
             if (c.point_floats == 4) launch_hist<4>(ra, B, st); else launch_hist<5>(ra, B, st);
         }
-        route_scan_kernel<<<B, kThreads, 0, st>>>(tile_counts, tile_base, d_offsets, tiles, E, N);
+        route_scan_kernel<<<B, kScanThreads, 0, st>>>(tile_counts, tile_base, d_offsets, tiles, E, N);
         if (tiles > 0) {
             ScatterArgs sa;
             sa.pts = d_points; sa.feat = reinterpret_cast<const float4*>(d_gathered); sa.expert = d_expert;
