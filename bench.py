@@ -307,11 +307,12 @@ def run_ours(args, w):
     dom_ms = per_kernel[dom]["ms_per_launch"]
     achieved = kb[dom] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
     traffic = None
-    try:
-        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
-            t = json.load(f).get(dom)
-            if t:
-                traffic = t["dram_bytes_per_point"] * B * N
+    try:                                                   # ncu DRAM counters, taken on this workload only
+        if w.config_id == 2:
+            with open(os.path.join(ROOT, "profiles", "dram_traffic_nuscenes.json")) as f:
+                t = json.load(f).get(dom)
+                if t:
+                    traffic = t["dram_bytes_per_point"] * B * N
     except Exception:
         pass
 
