@@ -186,7 +186,11 @@ __global__ void __launch_bounds__(kThreads) vox_scan_kernel(ScanArgs a) {
         Sector x[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u)
-            if (grp + u < hi) x[u] = load_sector(g.store, grp + u, lane);
+            if (grp + u < hi) {                   // streaming: most of the store is empty, keep it out of L2
+                const uint4* p = reinterpret_cast<const uint4*>(g.store) + ((size_t)(grp + u) * 32 + lane) * 2;
+                x[u].a = __ldcs(p);
+                x[u].b = __ldcs(p + 1);
+            }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             if (grp + u >= hi) break;
