@@ -288,8 +288,10 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
         if (e == cudaSuccess) e = cudaStreamWaitEvent(h->side, h->ev_fork, 0);
         if (e != cudaSuccess) return check_cuda(h, e);
     }
+    h->thin_scan = h->overlap;
     int rc = emc2_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity, d_num_voxels,
                            d_bev, vox_st);
+    h->thin_scan = false;
     int rc2 = EMC2_OK;
     if (rc == EMC2_OK && B > 0) {
         // The checks of emc2_project_gather and emc2_route_dispatch, then one pass over the rows.

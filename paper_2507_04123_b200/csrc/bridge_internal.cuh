@@ -111,6 +111,7 @@ struct emc2_bridge {
     int* d_scan_part = nullptr;    // [scan_blocks][3] per-CTA totals of the voxel rank scan
     int* d_scan_warp_ofs = nullptr;  // [scan_blocks * 8][3] per-warp offsets inside their CTA
     int scan_blocks = 0;           // CTAs of the cooperative rank scan (all co-resident)
+    bool thin_scan = false;        // set while emc2_bridge_run enqueues stage 1 beside stages 2 - 4
     int max_tiles = 0;
     bool overlap = true;           // emc2_bridge_run puts stage 1 on `side`
     cudaStream_t side = nullptr;   // stream of stage 1 inside emc2_bridge_run

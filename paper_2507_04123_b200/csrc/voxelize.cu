@@ -38,7 +38,7 @@ namespace emc2 {
 namespace {
 
 constexpr int kStatusCapacity = 1;
-constexpr int kPtsPerThread = 4;                      // independent points per thread (memory-level parallelism)
+constexpr int kPtsPerThread = 2;                      // independent points per thread (memory-level parallelism)
 constexpr int kBigTile = kThreads * kPtsPerThread;    // points per CTA in the two per-point passes
 constexpr int kOvfBlocks = 296;                       // CTAs of vox_finalize that serve cells over the cap
 
@@ -328,7 +328,7 @@ vox_accum_kernel(const float* __restrict__ pts, long long total, int N, AccumArg
     __syncthreads();
     const int b0 = (int)(g0 / N);
     const int i0 = (int)(g0 - (long long)b0 * N);
-    // All rank lookups first, so that a thread has eight loads in flight.
+    // All rank lookups first, so that a thread has its loads in flight together.
     Slot slot[2][kPtsPerThread];
     int cx[2][kPtsPerThread], cy[2][kPtsPerThread], cz[2][kPtsPerThread];
 #pragma unroll
@@ -555,7 +555,9 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     sa.warp_ofs = h->d_scan_warp_ofs;
     aa.bev = d_bev;
     // Split the cooperative grid between the scales in proportion to their group counts.
-    const int G = h->scan_blocks;
+    // Beside stages 2 - 4 (emc2_bridge_run) a thinner grid leaves them more of each SM and the
+    // step as a whole is shorter, although this kernel alone takes longer.
+    const int G = h->thin_scan ? max(2, h->scan_blocks / 2) : h->scan_blocks;
     const double share = (double)sa.ngroups_used[0] / (double)((uint64_t)sa.ngroups_used[0] + sa.ngroups_used[1] + 1);
     sa.g0 = min(G - 1, max(1, (int)(share * G)));
 
