@@ -288,7 +288,14 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
         if (e == cudaSuccess) e = cudaStreamWaitEvent(h->side, h->ev_fork, 0);
         if (e != cudaSuccess) return check_cuda(h, e);
     }
-    h->thin_scan = h->overlap;
+    // A thinner rank scan leaves stages 2 - 4 more of each SM; it pays while the scan's streaming
+    // read of the cell stores is small beside the feature rows those stages move.
+    {
+        double store_bytes = 0.0;
+        for (int s = 0; s < 2; ++s)
+            store_bytes += (double)B * h->scale[s].cells * (h->scale[s].mode == MODE_BITMAP ? 0.25 : 16.0);
+        h->thin_scan = h->overlap && 2.0 * store_bytes < (double)B * N * h->cfg.feat_c * 4.0;
+    }
     int rc = emc2_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity, d_num_voxels,
                            d_bev, vox_st);
     h->thin_scan = false;

@@ -45,6 +45,46 @@ def test_ragged_shapes(b200, oracle, B, N):
         run_case(b200, oracle, base.with_shape(B, N), repeat=2, staged=(N % 2 == 0))
 
 
+def test_one_call_without_the_side_stream(b200, oracle):
+    w = gen.NUSCENES.with_shape(2, 20000)
+    batch = gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    br = b200.Bridge(b200.config_from_workload(w))
+    br.set_overlap(False)                        # every kernel on the caller's stream
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    bufs = br.run(d["points"], d["proj"], d["feat"], bufs)
+    br.status()
+    compare_bridge(w, ref, bufs)
+    br.set_overlap(True)
+    bufs = br.run(d["points"], d["proj"], d["feat"], bufs)
+    br.status()
+    compare_bridge(w, ref, bufs)
+    br.close()
+
+
+def test_one_call_on_a_side_stream_of_the_caller(b200, oracle):
+    # The call must order itself after work already queued on the caller's stream and be complete,
+    # stage 1 included, for work queued after it on that stream.
+    w = gen.KITTI.with_shape(2, 30000)
+    batch = gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    br = b200.Bridge(b200.config_from_workload(w))
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        d = {k: torch.from_numpy(v).pin_memory().to("cuda", non_blocking=True) for k, v in batch.items()}
+        bufs = br.run(d["points"], d["proj"], d["feat"])
+        host = {"nv": bufs["vox"]["num_voxels"].to("cpu", non_blocking=True),
+                "bev": bufs["vox"]["bev"].to("cpu", non_blocking=True)}
+    s.synchronize()
+    assert host["nv"].tolist() == [ref["vox0"]["num_voxels"], ref["vox1"]["num_voxels"]]
+    assert np.array_equal(host["bev"].numpy() != 0, ref["bev"] != 0)
+    with torch.cuda.stream(s):
+        br.status()
+    compare_bridge(w, ref, bufs)
+    br.close()
+
+
 def test_sweep_cell_with_six_cameras(b200, oracle):
     run_case(b200, oracle, gen.SWEEP.with_shape(2, 65536))
 
