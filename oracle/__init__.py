@@ -129,6 +129,17 @@ def dispatch(expert: np.ndarray, points: np.ndarray, gathered: np.ndarray, num_e
     return offsets, perm, pout, fout
 
 
+def scene_route(offsets: np.ndarray, priority: Sequence[int], min_points: int = 1) -> np.ndarray:
+    """Scene-level expert per frame from the dispatch offsets (Sec. 3.2)."""
+    offsets = np.ascontiguousarray(offsets, np.int32)
+    B, E1 = offsets.shape
+    pr = np.ascontiguousarray(priority, np.uint8)
+    assert len(pr) == E1 - 1
+    out = np.empty(B, np.int32)
+    lib().emc2o_scene_route(B, E1 - 1, _p(offsets, _I), _p(pr, _U8), int(min_points), _p(out, _I))
+    return out
+
+
 def bridge(w, batch: Dict[str, np.ndarray]) -> Dict[str, object]:
     """All four stages on one batch of a workload description (emc2_gen.Workload)."""
     pts, proj, feat = batch["points"], batch["proj"], batch["feat"]

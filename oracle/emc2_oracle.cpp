@@ -226,3 +226,24 @@ void emc2o_dispatch(int B, int N, int C, int Cf, int E, const uint8_t* expert, c
 }
 
 }  // extern "C"
+
+// Scene-level choice of the Scenario-Adaptive Dispatcher (Sec. 3.2): a scene goes to the most
+// demanding expert that any of its objects asks for (close-and-distinct scenes to the
+// latency-prioritised expert, scenes with some harder object to the next one, and so on).  Per
+// point, that is the expert of highest priority among those that own at least `min_points`
+// points of the frame; ties go to the lowest expert id; -1 if no expert qualifies.
+// offsets [B, E+1] as written by the dispatch; priority [E]; scene_expert [B].
+extern "C" void emc2o_scene_route(int B, int E, const int32_t* offsets, const uint8_t* priority, int min_points,
+                                  int32_t* scene_expert) {
+    if (min_points < 1) min_points = 1;
+    for (int b = 0; b < B; ++b) {
+        const int32_t* off = offsets + (size_t)b * (E + 1);
+        int best = -1;
+        for (int e = 0; e < E; ++e) {
+            const int count = off[e + 1] - off[e];
+            if (count < min_points) continue;
+            if (best < 0 || priority[e] > priority[best]) best = e;
+        }
+        scene_expert[b] = best;
+    }
+}

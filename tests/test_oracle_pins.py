@@ -416,3 +416,33 @@ def test_dense_frame_recipe_hits_the_stated_occupancy(oracle):
     assert 150 <= r["counts"].max() <= 300
     capped = oracle.voxelize(pts, g.min, g.voxel, g.dims, g.max_points)
     assert capped["counts"].max() == 32 and (r["counts"] > 32).sum() > 100
+
+
+# ------------------------------------------------------------------ scene-level dispatch (Sec. 3.2)
+def test_scene_route_follows_the_three_cases_of_the_dispatcher(oracle):
+    # Experts 0 / 1 / 2 stand for the latency-prioritised, versatile and accuracy-prioritised
+    # experts, in rising priority.  A scene whose points all ask for expert 0 stays with expert 0;
+    # one point asking for a harder expert moves the whole scene.
+    pr = (0, 1, 2)
+    off = np.array([[0, 100, 100, 100],      # all close and distinct
+                    [0, 99, 100, 100],       # one mixed-visibility point
+                    [0, 50, 99, 100],        # one distant and uncertain point
+                    [0, 0, 0, 0],            # empty frame
+                    [0, 0, 0, 7]], np.int32)
+    assert list(oracle.scene_route(off, pr)) == [0, 1, 2, -1, 2]
+    # "some" can be given a size: with min_points = 2 single stragglers no longer move the scene
+    assert list(oracle.scene_route(off, pr, min_points=2)) == [0, 0, 1, -1, 2]
+    # priority is a table, not the expert id: ties go to the lowest id
+    assert list(oracle.scene_route(off[:3], (5, 5, 1))) == [0, 0, 0]
+    assert list(oracle.scene_route(off[:3], (0, 2, 1))) == [0, 1, 1]
+
+
+def test_scene_route_from_points_built_around_the_threshold(oracle):
+    # KITTI-style threshold of Sec. 4.1: D = 23.5 m; experts: 0 near, 1 far.
+    D = 23.5
+    near = [(5.0, 1.0), (10.0, -3.0), (nxt(D, 0), 0.0)]
+    for rows, want in ((near, 0), (near + [(D, 0.0)], 1), ([(40.0, 0.0)], 1)):
+        pts = _pts(rows)
+        ex = oracle.route(pts, np.ones((1, len(rows)), np.uint8), (D,), ((0, 1), (0, 1)))
+        off, _, _, _ = oracle.dispatch(ex, pts, np.zeros((1, len(rows), 4), F32), 2)
+        assert list(oracle.scene_route(off, (0, 1))) == [want]
