@@ -155,6 +155,18 @@ int emc2_bridge_run(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_
                     float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
                     float* d_points_out, float* d_feat_out, void* cuda_stream);
 
+/* Scene-level choice of the Scenario-Adaptive Dispatcher (Sec. 3.2): a scene is served by the most
+ * demanding expert that any of its objects asks for.  Per point: for every frame b the expert of
+ * highest priority[e] among the experts that own at least max(1, min_points) points of the frame
+ * (their counts are offsets[b][e+1] - offsets[b][e]); ties go to the lowest expert id; -1 if no
+ * expert qualifies.
+ *   d_offsets       int32 [B, E+1]  as written by emc2_route_dispatch / emc2_bridge_run
+ *   priority        uint8 [E]       HOST array, larger = more demanding expert
+ *   d_scene_expert  int32 [B]       output
+ * Enqueues one small kernel on `cuda_stream`. */
+int emc2_scene_route(emc2_bridge_t* bridge, int32_t B, const int32_t* d_offsets, const uint8_t* priority,
+                     int32_t min_points, int32_t* d_scene_expert, void* cuda_stream);
+
 /* Turns the side stream of emc2_bridge_run off (0) or on (non-zero, the default).  Off, every
  * kernel of the call is enqueued on `cuda_stream` itself, one after another: for callers that
  * want no second stream, and for timing kernels one at a time. */

@@ -33,7 +33,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_status", "emc2_bridge_destroy", "emc2_status_string", "emc2_bridge_last_cuda_error",
     "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
-    "emc2_bridge_run", "emc2_bridge_set_overlap",
+    "emc2_bridge_run", "emc2_bridge_set_overlap", "emc2_scene_route",
 )
 
 
@@ -80,6 +80,7 @@ def load_library() -> ctypes.CDLL:
                                     + [vp] * 4 + [vp] * 5 + [vp])
     lib.emc2_route_dispatch_static.argtypes = [P(Emc2Config), i32, i32] + [vp] * 9
     lib.emc2_bridge_status.argtypes = [vp, vp]
+    lib.emc2_scene_route.argtypes = [vp, i32, vp, P(ctypes.c_uint8), i32, vp, vp]
     lib.emc2_bridge_set_overlap.argtypes = [vp, ctypes.c_int]
     lib.emc2_bridge_destroy.argtypes = [vp]
     lib.emc2_status_string.argtypes = [ctypes.c_int]
@@ -283,6 +284,21 @@ class Bridge:
                                           out["points_out"].data_ptr(), out["feat_out"].data_ptr(),
                                           self._stream())
         self._raise(rc, "emc2_route_dispatch")
+        return out
+
+    def scene_route(self, offsets: torch.Tensor, priority: Sequence[int], min_points: int = 1,
+                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """emc2_scene_route: one expert per frame from the dispatch offsets."""
+        B = offsets.shape[0]
+        _check(offsets, torch.int32, (B, self.cfg.num_experts + 1), "offsets", self.device)
+        if len(priority) != self.cfg.num_experts:
+            raise ValueError("priority needs one entry per expert")
+        if out is None:
+            out = torch.empty((B,), dtype=torch.int32, device=self.device)
+        pr = (ctypes.c_uint8 * len(priority))(*priority)
+        rc = self.lib.emc2_scene_route(self._h, B, offsets.data_ptr(), pr, int(min_points), out.data_ptr(),
+                                       self._stream())
+        self._raise(rc, "emc2_scene_route")
         return out
 
     def set_overlap(self, enable: bool) -> None:

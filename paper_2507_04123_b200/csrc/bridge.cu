@@ -9,7 +9,7 @@ namespace emc2 {
 
 static const char* const kKernelNames[K_KINDS] = {
     "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
-    "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter"};
+    "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
     if (e == cudaSuccess) return EMC2_OK;
@@ -324,6 +324,17 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
     if (rc != EMC2_OK) return rc;
     if (rc2 != EMC2_OK) return rc2;
     return check_cuda(h, e);
+}
+
+int emc2_scene_route(emc2_bridge_t* h, int32_t B, const int32_t* d_offsets, const uint8_t* priority,
+                     int32_t min_points, int32_t* d_scene_expert, void* cuda_stream) {
+    if (!h || B < 0 || B > h->cfg.max_batch || !priority) return EMC2_ERR_INVALID_ARG;
+    if (B == 0) return EMC2_OK;
+    if (!d_offsets || !d_scene_expert) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_scene_route(h, B, d_offsets, priority, min_points, d_scene_expert,
+                              static_cast<cudaStream_t>(cuda_stream));
 }
 
 int emc2_bridge_set_overlap(emc2_bridge_t* h, int enable) {

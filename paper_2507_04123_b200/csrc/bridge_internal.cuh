@@ -30,6 +30,7 @@ enum KernelKind {
     K_ROUTE_HIST,
     K_ROUTE_SCAN,
     K_DISPATCH_SCATTER,
+    K_SCENE_ROUTE,
     K_KINDS
 };
 
@@ -159,6 +160,8 @@ inline RouteParams route_params(const emc2_bridge* h) {
     return rp;
 }
 
+int launch_scene_route(emc2_bridge* h, int B, const int32_t* d_offsets, const uint8_t* priority, int min_points,
+                       int32_t* d_scene_expert, cudaStream_t st);
 // Tile histograms (handle scratch) -> d_offsets and tile bases (handle scratch).
 void launch_route_scan(emc2_bridge* h, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st);
 // Stages 2 - 4 in one pass over the feature rows (the one-call path).

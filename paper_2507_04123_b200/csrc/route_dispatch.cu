@@ -244,6 +244,43 @@ void launch_scatter(emc2_bridge* h, const ScatterArgs& a, dim3 grid, cudaStream_
 
 }  // namespace
 
+namespace {
+
+struct SceneArgs {
+    const int32_t* offsets;
+    int32_t* scene_expert;
+    int B, E, min_points;
+    uint8_t priority[EMC2_MAX_EXPERTS];
+};
+
+// One thread per frame: the expert of highest priority that owns enough points (Sec. 3.2).
+__global__ void scene_route_kernel(const __grid_constant__ SceneArgs a) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= a.B) return;
+    const int32_t* off = a.offsets + (size_t)b * (a.E + 1);
+    int best = -1, best_pr = -1;
+    for (int e = 0; e < a.E; ++e) {
+        const int count = off[e + 1] - off[e];
+        if (count >= a.min_points && (int)a.priority[e] > best_pr) { best = e; best_pr = a.priority[e]; }
+    }
+    a.scene_expert[b] = best;
+}
+
+}  // namespace
+
+int launch_scene_route(emc2_bridge* h, int B, const int32_t* d_offsets, const uint8_t* priority, int min_points,
+                       int32_t* d_scene_expert, cudaStream_t st) {
+    SceneArgs a;
+    a.offsets = d_offsets; a.scene_expert = d_scene_expert;
+    a.B = B; a.E = h->cfg.num_experts; a.min_points = min_points < 1 ? 1 : min_points;
+    for (int e = 0; e < EMC2_MAX_EXPERTS; ++e) a.priority[e] = e < a.E ? priority[e] : 0;
+    {
+        LaunchScope ls(h, K_SCENE_ROUTE, st);
+        scene_route_kernel<<<(B + 31) / 32, 32, 0, st>>>(a);
+    }
+    return check_cuda(h, cudaGetLastError());
+}
+
 void launch_route_scan(emc2_bridge* h, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st) {
     LaunchScope ls(h, K_ROUTE_SCAN, st);
     route_scan_kernel<<<B, kScanThreads, 0, st>>>(h->d_tile_counts, h->d_tile_base, d_offsets, tiles, h->cfg.num_experts, N);

@@ -85,6 +85,28 @@ def test_one_call_on_a_side_stream_of_the_caller(b200, oracle):
     br.close()
 
 
+def test_scene_route_matches_the_oracle(b200, oracle):
+    w = gen.NUSCENES.with_shape(5, 4000)
+    batch = gen.make_batch(w)
+    p = batch["points"]
+    p[1, :, :2] *= 0.2                           # everything near: no far expert in this frame
+    p[2, :, 0] = -400.0                          # everything beyond 50 m and invisible
+    p[3, 1:, :2] *= 0.1
+    p[3, 0, :3] = (60.0, 0.0, 0.0)               # a single far point
+    ref = oracle.bridge(w, batch)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    for pr, mp in (((0, 1, 2, 3), 1), ((0, 1, 2, 3), 2), ((3, 2, 1, 0), 1), ((1, 1, 1, 1), 1), ((0, 2, 1, 2), 50)):
+        got = np_(br.scene_route(bufs["rd"]["offsets"], pr, mp))
+        assert np.array_equal(got, oracle.scene_route(ref["offsets"], pr, mp)), (pr, mp)
+    assert len(set(oracle.scene_route(ref["offsets"], (0, 1, 2, 3), 1).tolist())) > 1
+    empty = torch.zeros((5, w.num_experts + 1), dtype=torch.int32, device="cuda")
+    assert (np_(br.scene_route(empty, (0, 1, 2, 3))) == -1).all()
+    br.status()
+    br.close()
+
+
 def test_sweep_cell_with_six_cameras(b200, oracle):
     run_case(b200, oracle, gen.SWEEP.with_shape(2, 65536))
 
