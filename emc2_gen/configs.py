@@ -53,6 +53,7 @@ class Workload:
     num_experts: int
     lut: Tuple[Tuple[int, ...], Tuple[int, ...]]   # [visible?][distance bucket]
     xy_range: Tuple[float, float, float, float] = (0.0, 70.4, -40.0, 40.0)
+    feat_offset: float = 0.0            # pixel position of texel 0 (non-zero for pooled maps)
 
     @property
     def K(self) -> int:

@@ -86,14 +86,23 @@ def project(points: np.ndarray, proj: np.ndarray, H: int, W: int, min_depth: flo
     return uvd, mask, cam
 
 
-def gather(uvd: np.ndarray, cam: np.ndarray, feat: np.ndarray, stride: int) -> np.ndarray:
+def pool(feat: np.ndarray, p: int) -> np.ndarray:
+    """p x p average pooling of channels-last feature maps (Sec. 3.5, Multiscale Pooling)."""
+    feat = _f32(feat)
+    B, K, Hf, Wf, Cf = feat.shape
+    out = np.empty((B, K, -(-Hf // p), -(-Wf // p), Cf), np.float32)
+    lib().emc2o_pool(B, K, Hf, Wf, Cf, int(p), _p(feat, _F), _p(out, _F))
+    return out
+
+
+def gather(uvd: np.ndarray, cam: np.ndarray, feat: np.ndarray, stride: int, offset: float = 0.0) -> np.ndarray:
     uvd, feat = _f32(uvd), _f32(feat)
     cam = np.ascontiguousarray(cam, np.int8)
     B, N, _ = uvd.shape
     _, K, Hf, Wf, Cf = feat.shape
     out = np.empty((B, N, Cf), np.float32)
-    lib().emc2o_gather(B, N, K, Hf, Wf, Cf, int(stride), _p(uvd, _F), _p(cam, _I8), _p(feat, _F),
-                       _p(out, _F))
+    lib().emc2o_gather(B, N, K, Hf, Wf, Cf, int(stride), ctypes.c_float(offset), _p(uvd, _F), _p(cam, _I8),
+                       _p(feat, _F), _p(out, _F))
     return out
 
 
@@ -151,7 +160,7 @@ def bridge(w, batch: Dict[str, np.ndarray]) -> Dict[str, object]:
                      out["vox1"]["mean"])
     uvd, mask, cam = project(pts, proj, w.img_h, w.img_w, w.min_depth)
     out["uvd"], out["vis_mask"], out["cam"] = uvd, mask, cam
-    out["gathered"] = gather(uvd, cam, feat, w.feat_stride)
+    out["gathered"] = gather(uvd, cam, feat, w.feat_stride, getattr(w, "feat_offset", 0.0))
     out["expert"] = route(pts, mask, w.thresholds, w.lut)
     off, perm, pout, fout = dispatch(out["expert"], pts, out["gathered"], w.num_experts)
     out["offsets"], out["perm"], out["points_out"], out["feat_out"] = off, perm, pout, fout

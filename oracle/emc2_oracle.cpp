@@ -154,8 +154,10 @@ void emc2o_project(int B, int N, int C, int K, const float* points, const float*
 // feat [B,K,Hf,Wf,Cf].  Texel (j,i) is the sample at pixel (j*s, i*s); taps
 // are edge-clamped; points with cam = -1 get an all-zero row (Fig. 5: no match
 // -> zero-filled features).  The blend is evaluated in double and rounded once.
-void emc2o_gather(int B, int N, int K, int Hf, int Wf, int Cf, int stride, const float* uvd,
+void emc2o_gather(int B, int N, int K, int Hf, int Wf, int Cf, int stride, float offset, const float* uvd,
                   const int8_t* cam, const float* feat, float* gathered) {
+    // `offset` is the pixel position of texel 0 (0 for a plain strided map; (p - 1) / 2 * s for a
+    // map that was average-pooled p x p, whose texels sit at the centres of their windows).
     const double inv = 1.0 / (double)stride;
     for (int b = 0; b < B; ++b)
         for (int i = 0; i < N; ++i) {
@@ -165,12 +167,15 @@ void emc2o_gather(int B, int N, int K, int Hf, int Wf, int Cf, int stride, const
                 for (int c = 0; c < Cf; ++c) out[c] = 0.0f;
                 continue;
             }
-            double fx = (double)uvd[3 * g + 0] * inv, fy = (double)uvd[3 * g + 1] * inv;
+            // The subtraction is done in fp32 (one rounding), as the pixel coordinates are fp32.
+            double fx = (double)(uvd[3 * g + 0] - offset) * inv, fy = (double)(uvd[3 * g + 1] - offset) * inv;
             int x0 = (int)std::floor(fx), y0 = (int)std::floor(fy);
             double wx = fx - x0, wy = fy - y0;
             int x1 = std::min(x0 + 1, Wf - 1), y1 = std::min(y0 + 1, Hf - 1);
             x0 = std::min(x0, Wf - 1);
             y0 = std::min(y0, Hf - 1);
+            x0 = std::max(x0, 0); x1 = std::max(x1, 0);     // left of texel 0: clamp to the edge as well
+            y0 = std::max(y0, 0); y1 = std::max(y1, 0);
             const float* base = feat + ((size_t)b * K + cam[g]) * Hf * Wf * Cf;
             const float* f00 = base + ((size_t)y0 * Wf + x0) * Cf;
             const float* f01 = base + ((size_t)y0 * Wf + x1) * Cf;
@@ -182,6 +187,28 @@ void emc2o_gather(int B, int N, int K, int Hf, int Wf, int Cf, int stride, const
                 out[c] = (float)((1.0 - wy) * top + wy * bot);
             }
         }
+}
+
+// Multiscale Pooling of the image features (Sec. 3.5: image features are pooled, with a
+// user-chosen pooling size, before they are fused with LiDAR features, to relieve memory).
+// feat [B,K,Hf,Wf,Cf] channels-last -> pooled [B,K,ceil(Hf/p),ceil(Wf/p),Cf]: the mean over each
+// p x p window of texels; windows at the right / bottom edge hold fewer texels and average over
+// those they hold.
+void emc2o_pool(int B, int K, int Hf, int Wf, int Cf, int p, const float* feat, float* pooled) {
+    const int Hp = (Hf + p - 1) / p, Wp = (Wf + p - 1) / p;
+    for (int m = 0; m < B * K; ++m)
+        for (int J = 0; J < Hp; ++J)
+            for (int I = 0; I < Wp; ++I)
+                for (int c = 0; c < Cf; ++c) {
+                    double sum = 0.0;
+                    int n = 0;
+                    for (int j = J * p; j < std::min(Hf, J * p + p); ++j)
+                        for (int i = I * p; i < std::min(Wf, I * p + p); ++i) {
+                            sum += (double)feat[(((size_t)m * Hf + j) * Wf + i) * Cf + c];
+                            n += 1;
+                        }
+                    pooled[(((size_t)m * Hp + J) * Wp + I) * Cf + c] = (float)(sum / n);
+                }
 }
 
 // Stage 3: per-point routing (Sec. 3.2: near is "< D", far is ">= D").  Planar

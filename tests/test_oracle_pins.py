@@ -446,3 +446,61 @@ def test_scene_route_from_points_built_around_the_threshold(oracle):
         ex = oracle.route(pts, np.ones((1, len(rows)), np.uint8), (D,), ((0, 1), (0, 1)))
         off, _, _, _ = oracle.dispatch(ex, pts, np.zeros((1, len(rows), 4), F32), 2)
         assert list(oracle.scene_route(off, (0, 1))) == [want]
+
+
+# ------------------------------------------------------------------ Multiscale Pooling (Sec. 3.5)
+def test_pool_closed_forms(oracle):
+    rng = np.random.default_rng(11)
+    feat = rng.standard_normal((2, 3, 7, 10, 4)).astype(F32)
+    assert np.array_equal(oracle.pool(feat, 1), feat)                       # p = 1 is the identity
+    const = np.full((1, 1, 9, 9, 3), 2.5, F32)
+    assert np.array_equal(oracle.pool(const, 4), np.full((1, 1, 3, 3, 3), 2.5, F32))
+    # an affine map pools to its value at the window centre, ragged edge windows included
+    Hf, Wf = 7, 10
+    yy, xx = np.meshgrid(np.arange(Hf), np.arange(Wf), indexing="ij")
+    ramp = (0.5 * xx - 2.0 * yy + 1.0).astype(F32)[None, None, :, :, None]
+    got = oracle.pool(ramp, 3)[0, 0, :, :, 0]
+    assert got.shape == (3, 4)
+    for J in range(3):
+        for I in range(4):
+            ys, xs = range(3 * J, min(Hf, 3 * J + 3)), range(3 * I, min(Wf, 3 * I + 3))
+            cy, cx = (ys[0] + ys[-1]) / 2, (xs[0] + xs[-1]) / 2
+            assert abs(got[J, I] - (0.5 * cx - 2.0 * cy + 1.0)) < 1e-6
+
+
+def test_pool_against_avg_pool2d(oracle):
+    rng = np.random.default_rng(12)
+    feat = rng.standard_normal((2, 2, 94, 311, 8)).astype(F32)
+    for p in (2, 4, 5):
+        got = oracle.pool(feat, p)
+        x = torch.from_numpy(feat).double().permute(0, 1, 4, 2, 3).reshape(4, 8, 94, 311)
+        ref = torch.nn.functional.avg_pool2d(x, p, stride=p, ceil_mode=True, count_include_pad=False)
+        ref = ref.reshape(2, 2, 8, ref.shape[2], ref.shape[3]).permute(0, 1, 3, 4, 2).numpy()
+        assert got.shape == ref.shape and np.abs(got - ref).max() < 1e-6
+
+
+def test_gather_with_window_centre_offset(oracle):
+    # A map pooled p x p has its texels at the window centres: texel I sits at pixel
+    # (I * p + (p - 1) / 2) * s.  Sampling an affine image there reproduces it between the first and
+    # last centre and clamps outside, on the left as well as on the right.
+    s, p, Hp, Wp = 4, 4, 6, 9
+    S, off = s * p, (p - 1) / 2 * s
+    yy, xx = np.meshgrid(np.arange(Hp), np.arange(Wp), indexing="ij")
+    u_tex, v_tex = xx * S + off, yy * S + off                               # pixel position of each texel
+    feat = (0.25 * u_tex - 0.5 * v_tex + 3.0).astype(F32)[None, None, :, :, None]
+    rng = np.random.default_rng(13)
+    u = rng.uniform(off, (Wp - 1) * S + off, 200)
+    v = rng.uniform(off, (Hp - 1) * S + off, 200)
+    uvd = np.stack([u, v, np.ones(200)], 1).astype(F32)[None]
+    out = oracle.gather(uvd, np.zeros((1, 200), np.int8), feat, S, off)
+    want = 0.25 * uvd[0, :, 0].astype(np.float64) - 0.5 * uvd[0, :, 1].astype(np.float64) + 3.0
+    assert np.abs(out[0, :, 0] - want).max() < 1e-4
+    uvd = np.array([[[0.5, 40.0, 1.0], [(Wp - 1) * S + off + 5.0, 40.0, 1.0], [50.0, 1.0, 1.0]]], F32)
+    out = oracle.gather(uvd, np.zeros((1, 3), np.int8), feat, S, off)
+    assert np.isclose(out[0, 0, 0], 0.25 * off - 0.5 * 40.0 + 3.0)          # left of the first centre
+    assert np.isclose(out[0, 1, 0], 0.25 * ((Wp - 1) * S + off) - 0.5 * 40.0 + 3.0)
+    assert np.isclose(out[0, 2, 0], 0.25 * 50.0 - 0.5 * off + 3.0)          # above the first centre
+    # offset 0 is the plain strided map
+    a = oracle.gather(uvd, np.zeros((1, 3), np.int8), feat, S)
+    b = oracle.gather(uvd, np.zeros((1, 3), np.int8), feat, S, 0.0)
+    assert np.array_equal(a, b)
