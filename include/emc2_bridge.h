@@ -84,6 +84,10 @@ typedef struct {
     float thresholds[EMC2_MAX_THRESHOLDS]; /* ascending planar ranges in metres */
     int32_t num_experts;                   /* E, 1..EMC2_MAX_EXPERTS */
     uint8_t lut[2][8]; /* expert = lut[visible ? 1 : 0][number of thresholds reached]; < E */
+    float feat_offset; /* pixel position of texel 0 along both axes: texel (j, i) is the sample at pixel
+                          (feat_offset + j*s, feat_offset + i*s).  0 for a plain strided map; (p-1)/2 * s0
+                          for a map that emc2_pool_features pooled p x p from stride s0 (then s = p*s0).
+                          Finite, >= 0. */
 } emc2_config_t;
 
 /* Validates the configuration, selects the device and allocates all scratch memory the stage
@@ -117,7 +121,8 @@ int emc2_voxelize(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_po
  *                                 or (-1, -1, depth in camera 0 [0 if not finite]) if none does
  *   d_vis_mask  uint8 [B, N]      bit k set iff depth_k > min_depth, 0 <= u < W and 0 <= v < H
  *   d_cam       int8  [B, N]      that camera, or -1
- *   d_gathered  float [B, N, Cf]  bilinear sample at (u/s, v/s), taps clamped to the map edge;
+ *   d_gathered  float [B, N, Cf]  bilinear sample at ((u - feat_offset)/s, (v - feat_offset)/s), taps
+ *                                 clamped to the map edge;
  *                                 all zeros for points no camera sees */
 int emc2_project_gather(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_points,
                         const float* d_proj, const float* d_feat, float* d_uvd, uint8_t* d_vis_mask,
@@ -154,6 +159,18 @@ int emc2_bridge_run(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_
                     int32_t* d_num_voxels, float* d_bev, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
                     float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
                     float* d_points_out, float* d_feat_out, void* cuda_stream);
+
+/* Multiscale Pooling of the image features (Sec. 3.5: image features are pooled, with a pooling size
+ * the user chooses, before they are fused with LiDAR features, to relieve memory).
+ *   d_feat    float [B, K, Hf, Wf, Cf]                    the handle's feature-map shape
+ *   d_pooled  float [B, K, ceil(Hf/p), ceil(Wf/p), Cf]    mean over each p x p window of texels; windows
+ *                                                         at the right / bottom edge average over the
+ *                                                         texels they hold
+ * p >= 1 (1 copies).  To sample the pooled maps, use a handle whose configuration has
+ * feat_h = ceil(Hf/p), feat_w = ceil(Wf/p), feat_stride = p * s (p a power of two) and
+ * feat_offset = (p - 1) / 2 * s, so that each pooled texel sits at the centre of its window. */
+int emc2_pool_features(emc2_bridge_t* bridge, int32_t B, int32_t p, const float* d_feat, float* d_pooled,
+                       void* cuda_stream);
 
 /* Scene-level choice of the Scenario-Adaptive Dispatcher (Sec. 3.2): a scene is served by the most
  * demanding expert that any of its objects asks for.  Per point: for every frame b the expert of

@@ -33,7 +33,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_status", "emc2_bridge_destroy", "emc2_status_string", "emc2_bridge_last_cuda_error",
     "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
-    "emc2_bridge_run", "emc2_bridge_set_overlap", "emc2_scene_route",
+    "emc2_bridge_run", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
 )
 
 
@@ -50,7 +50,8 @@ class Emc2Config(ctypes.Structure):
                 ("feat_h", ctypes.c_int32), ("feat_w", ctypes.c_int32), ("feat_c", ctypes.c_int32),
                 ("feat_stride", ctypes.c_int32), ("min_depth", ctypes.c_float),
                 ("num_thresholds", ctypes.c_int32), ("thresholds", ctypes.c_float * 7),
-                ("num_experts", ctypes.c_int32), ("lut", (ctypes.c_uint8 * 8) * 2)]
+                ("num_experts", ctypes.c_int32), ("lut", (ctypes.c_uint8 * 8) * 2),
+                ("feat_offset", ctypes.c_float)]
 
 
 class Emc2Error(RuntimeError):
@@ -80,6 +81,7 @@ def load_library() -> ctypes.CDLL:
                                     + [vp] * 4 + [vp] * 5 + [vp])
     lib.emc2_route_dispatch_static.argtypes = [P(Emc2Config), i32, i32] + [vp] * 9
     lib.emc2_bridge_status.argtypes = [vp, vp]
+    lib.emc2_pool_features.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.emc2_scene_route.argtypes = [vp, i32, vp, P(ctypes.c_uint8), i32, vp, vp]
     lib.emc2_bridge_set_overlap.argtypes = [vp, ctypes.c_int]
     lib.emc2_bridge_destroy.argtypes = [vp]
@@ -99,7 +101,7 @@ def load_library() -> ctypes.CDLL:
 def make_config(*, device: int, max_batch: int, max_points: int, point_floats: int, grids,
                 num_cameras: int, img_h: int, img_w: int, feat_h: int, feat_w: int, feat_c: int,
                 feat_stride: int, min_depth: float, thresholds: Sequence[float], num_experts: int,
-                lut: Sequence[Sequence[int]]) -> Emc2Config:
+                lut: Sequence[Sequence[int]], feat_offset: float = 0.0) -> Emc2Config:
     """Fills an emc2_config_t.  ``grids`` is two objects with min, voxel, dims, max_points."""
     c = Emc2Config()
     c.device, c.max_batch, c.max_points, c.point_floats = device, max_batch, max_points, point_floats
@@ -113,6 +115,7 @@ def make_config(*, device: int, max_batch: int, max_points: int, point_floats: i
     c.num_cameras, c.img_h, c.img_w = num_cameras, img_h, img_w
     c.feat_h, c.feat_w, c.feat_c, c.feat_stride = feat_h, feat_w, feat_c, feat_stride
     c.min_depth = min_depth
+    c.feat_offset = feat_offset
     c.num_thresholds = len(thresholds)
     for t, v in enumerate(thresholds):
         c.thresholds[t] = v
@@ -131,7 +134,7 @@ def config_from_workload(w, device: int = 0, max_batch: Optional[int] = None,
                        point_floats=w.C, grids=w.grids, num_cameras=w.K, img_h=w.img_h, img_w=w.img_w,
                        feat_h=w.feat_h, feat_w=w.feat_w, feat_c=w.feat_c, feat_stride=w.feat_stride,
                        min_depth=w.min_depth, thresholds=w.thresholds, num_experts=w.num_experts,
-                       lut=w.lut)
+                       lut=w.lut, feat_offset=getattr(w, "feat_offset", 0.0))
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -284,6 +287,19 @@ class Bridge:
                                           out["points_out"].data_ptr(), out["feat_out"].data_ptr(),
                                           self._stream())
         self._raise(rc, "emc2_route_dispatch")
+        return out
+
+    def pool_features(self, feat: torch.Tensor, p: int, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """emc2_pool_features: p x p average pooling of the handle's feature maps."""
+        c = self.cfg
+        B = feat.shape[0]
+        _check(feat, torch.float32, (B, c.num_cameras, c.feat_h, c.feat_w, c.feat_c), "feat", self.device)
+        shape = (B, c.num_cameras, -(-c.feat_h // p), -(-c.feat_w // p), c.feat_c)
+        if out is None:
+            out = torch.empty(shape, dtype=torch.float32, device=self.device)
+        _check(out, torch.float32, shape, "pooled", self.device)
+        rc = self.lib.emc2_pool_features(self._h, B, int(p), feat.data_ptr(), out.data_ptr(), self._stream())
+        self._raise(rc, "emc2_pool_features")
         return out
 
     def scene_route(self, offsets: torch.Tensor, priority: Sequence[int], min_points: int = 1,

@@ -9,7 +9,7 @@ namespace emc2 {
 
 static const char* const kKernelNames[K_KINDS] = {
     "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
-    "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route"};
+    "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
     if (e == cudaSuccess) return EMC2_OK;
@@ -90,6 +90,7 @@ int validate(const emc2_config_t& c) {
     if ((uint64_t)c.max_batch * c.num_cameras * c.feat_h * c.feat_w * (uint64_t)(c.feat_c / 4) > 0xFFFFFFF0ull)
         return EMC2_ERR_BAD_CONFIG;
     if (!(c.min_depth >= 0.0f)) return EMC2_ERR_BAD_CONFIG;
+    if (!(c.feat_offset >= 0.0f) || !std::isfinite(c.feat_offset)) return EMC2_ERR_BAD_CONFIG;
     if (c.num_thresholds < 0 || c.num_thresholds > EMC2_MAX_THRESHOLDS) return EMC2_ERR_BAD_CONFIG;
     for (int t = 0; t < c.num_thresholds; ++t) {
         if (!(c.thresholds[t] >= 0.0f) || !std::isfinite(c.thresholds[t])) return EMC2_ERR_BAD_CONFIG;
@@ -324,6 +325,17 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
     if (rc != EMC2_OK) return rc;
     if (rc2 != EMC2_OK) return rc2;
     return check_cuda(h, e);
+}
+
+int emc2_pool_features(emc2_bridge_t* h, int32_t B, int32_t p, const float* d_feat, float* d_pooled,
+                       void* cuda_stream) {
+    if (!h || B < 0 || B > h->cfg.max_batch || p < 1) return EMC2_ERR_INVALID_ARG;
+    if (B == 0) return EMC2_OK;
+    if (!d_feat || !d_pooled || !aligned16(d_feat) || !aligned16(d_pooled) || d_feat == d_pooled)
+        return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_pool_features(h, B, p, d_feat, d_pooled, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int emc2_scene_route(emc2_bridge_t* h, int32_t B, const int32_t* d_offsets, const uint8_t* priority,

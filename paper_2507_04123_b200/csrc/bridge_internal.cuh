@@ -31,6 +31,7 @@ enum KernelKind {
     K_ROUTE_SCAN,
     K_DISPATCH_SCATTER,
     K_SCENE_ROUTE,
+    K_POOL_FEATURES,
     K_KINDS
 };
 
@@ -160,6 +161,7 @@ inline RouteParams route_params(const emc2_bridge* h) {
     return rp;
 }
 
+int launch_pool_features(emc2_bridge* h, int B, int p, const float* d_feat, float* d_pooled, cudaStream_t st);
 int launch_scene_route(emc2_bridge* h, int B, const int32_t* d_offsets, const uint8_t* priority, int min_points,
                        int32_t* d_scene_expert, cudaStream_t st);
 // Tile histograms (handle scratch) -> d_offsets and tile bases (handle scratch).

@@ -24,7 +24,7 @@ struct PgArgs {
     float4* out;
     long long total;
     int N, K, H, W, Hf, Wf, cf4;
-    float min_depth, inv_stride;
+    float min_depth, inv_stride, offset;
 };
 
 constexpr uint32_t kZeroRow = 0xFFFFFFFFu;
@@ -98,16 +98,17 @@ __device__ __forceinline__ void load_proj(const float* __restrict__ proj, int b,
 // Tap record of a point seen by camera `cam` of frame b at pixel (u, v): {float4 index of tap
 // (y0, x0), clamp flags, wx, wy}; kZeroRow in .x for a point no camera sees.
 __device__ __forceinline__ uint4 tap_record(int b, int cam, float u, float v, int K, int Hf, int Wf, int cf4,
-                                            float inv_stride) {
+                                            float inv_stride, float offset) {
     uint4 rec = make_uint4(kZeroRow, 0u, 0u, 0u);
     if (cam >= 0) {
-        // Texel coordinates: the stride is a power of two, so the scaling is exact.
-        const float fx = u * inv_stride, fy = v * inv_stride;
+        // Texel coordinates: one fp32 subtraction, then an exact scaling (the stride is a power of
+        // two).  Taps are clamped to the map on every side.
+        const float fx = __fsub_rn(u, offset) * inv_stride, fy = __fsub_rn(v, offset) * inv_stride;
         const float flx = floorf(fx), fly = floorf(fy);
         int x0 = (int)flx, y0 = (int)fly;
-        const int x1 = min(x0 + 1, Wf - 1), y1 = min(y0 + 1, Hf - 1);
-        x0 = min(x0, Wf - 1);
-        y0 = min(y0, Hf - 1);
+        const int x1 = max(min(x0 + 1, Wf - 1), 0), y1 = max(min(y0 + 1, Hf - 1), 0);
+        x0 = max(min(x0, Wf - 1), 0);
+        y0 = max(min(y0, Hf - 1), 0);
         const uint32_t map = ((uint32_t)b * K + cam) * Hf;
         rec.x = ((map + y0) * Wf + x0) * (uint32_t)cf4;
         rec.y = (uint32_t)(x1 - x0) | ((uint32_t)(y1 - y0) << 1);
@@ -161,7 +162,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) project_gather_
         suvd[t * 3] = pr.u; suvd[t * 3 + 1] = pr.v; suvd[t * 3 + 2] = pr.d;
         a.vis[gi] = (uint8_t)pr.mask;
         a.cam[gi] = (int8_t)pr.best;
-        const uint4 rec = tap_record(b, pr.best, pr.u, pr.v, a.K, a.Hf, a.Wf, cf4, a.inv_stride);
+        const uint4 rec = tap_record(b, pr.best, pr.u, pr.v, a.K, a.Hf, a.Wf, cf4, a.inv_stride, a.offset);
         srow[t] = rec;
     }
     __syncthreads();
@@ -265,7 +266,7 @@ struct GsArgs {
     float4* gathered;
     float4* feat_out;
     int N, tiles, E, K, Hf, Wf, cf4;
-    float inv_stride;
+    float inv_stride, offset;
 };
 
 // CF4 > 0: Cf/4 known at compile time, blockDim.x == 16 * CF4.  CF4 == 0: any Cf, 256 threads.
@@ -287,7 +288,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) gather_scatter_
         if (t < npts) {
             e = (int)a.expert[g0 + t];
             const float u = a.uvd[(g0 + t) * 3], v = a.uvd[(g0 + t) * 3 + 1];
-            srow[t] = tap_record(b, (int)a.cam[g0 + t], u, v, a.K, a.Hf, a.Wf, cf4, a.inv_stride);
+            srow[t] = tap_record(b, (int)a.cam[g0 + t], u, v, a.K, a.Hf, a.Wf, cf4, a.inv_stride, a.offset);
         }
         for (int k = 0; k < a.E; ++k) {
             const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
@@ -347,6 +348,32 @@ void launch_gs(emc2_bridge* h, const GsArgs& a, dim3 grid, cudaStream_t st) {
     }
 }
 
+// ------------------------------------------------------------------ Multiscale Pooling (Sec. 3.5)
+// One thread per (pooled texel, float4 column); grid = (columns of a pooled row, pooled rows,
+// maps).  Consecutive threads read consecutive columns of the same input rows, so every load
+// covers whole 256/320-byte rows.  Streams the maps once.
+__global__ void __launch_bounds__(kThreads)
+pool_features_kernel(const float4* __restrict__ feat, float4* __restrict__ pooled, int Hf, int Wf, int Hp, int Wp,
+                     int cf4, int p) {
+    const int ic = blockIdx.x * kThreads + threadIdx.x;     // I * cf4 + c
+    if (ic >= Wp * cf4) return;
+    const int I = ic / cf4, c = ic - I * cf4;
+    const int J = blockIdx.y;
+    const size_t m = blockIdx.z;                            // map index b * K + k
+    const int j0 = J * p, j1 = min(Hf, j0 + p), i0 = I * p, i1 = min(Wf, i0 + p);
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = j0; j < j1; ++j) {
+        const float4* row = feat + ((m * Hf + j) * Wf + i0) * cf4 + c;
+#pragma unroll 4
+        for (int x = 0; x < i1 - i0; ++x) {
+            const float4 v = __ldcs(row + (size_t)x * cf4);
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+    }
+    const float inv = 1.0f / (float)((j1 - j0) * (i1 - i0));
+    pooled[((m * Hp + J) * Wp) * cf4 + ic] = make_float4(s.x * inv, s.y * inv, s.z * inv, s.w * inv);
+}
+
 template <int C>
 void launch_c(emc2_bridge* h, const PgArgs& a, int tiles, cudaStream_t st) {
     LaunchScope ls(h, K_PROJECT_GATHER, st);
@@ -371,6 +398,7 @@ int launch_project_gather(emc2_bridge* h, int B, int N, const float* d_points, c
     a.cf4 = c.feat_c / 4;
     a.min_depth = c.min_depth;
     a.inv_stride = 1.0f / (float)c.feat_stride;
+    a.offset = c.feat_offset;
     const int tiles = (int)((a.total + kTile - 1) / kTile);
     if (tiles == 0) return EMC2_OK;
     if (c.point_floats == 4) launch_c<4>(h, a, tiles, st); else launch_c<5>(h, a, tiles, st);
@@ -405,7 +433,22 @@ int launch_project_route_gather_dispatch(emc2_bridge* h, int B, int N, const flo
         ga.N = N; ga.tiles = tiles; ga.E = c.num_experts; ga.K = c.num_cameras; ga.Hf = c.feat_h; ga.Wf = c.feat_w;
         ga.cf4 = c.feat_c / 4;
         ga.inv_stride = 1.0f / (float)c.feat_stride;
+        ga.offset = c.feat_offset;
         if (c.point_floats == 4) launch_gs<4>(h, ga, grid, st); else launch_gs<5>(h, ga, grid, st);
+    }
+    return check_cuda(h, cudaGetLastError());
+}
+
+int launch_pool_features(emc2_bridge* h, int B, int p, const float* d_feat, float* d_pooled, cudaStream_t st) {
+    const emc2_config_t& c = h->cfg;
+    const int Hp = (c.feat_h + p - 1) / p, Wp = (c.feat_w + p - 1) / p, cf4 = c.feat_c / 4;
+    if (Hp > 65535) return EMC2_ERR_INVALID_ARG;           // grid limit: one pooled row per blockIdx.y
+    const dim3 grid((Wp * cf4 + kThreads - 1) / kThreads, Hp, B * c.num_cameras);
+    {
+        LaunchScope ls(h, K_POOL_FEATURES, st);
+        pool_features_kernel<<<grid, kThreads, 0, st>>>(reinterpret_cast<const float4*>(d_feat),
+                                                        reinterpret_cast<float4*>(d_pooled), c.feat_h, c.feat_w, Hp,
+                                                        Wp, cf4, p);
     }
     return check_cuda(h, cudaGetLastError());
 }

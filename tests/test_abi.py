@@ -30,9 +30,9 @@ def test_library_exports_every_declared_symbol(pkg):
 
 
 def test_config_struct_layout_matches_the_header(pkg):
-    # 4 ints, 2 grids of (3f, 3f, 3i, i), 7 ints, float, int, 7 floats, int, 16 bytes
+    # 4 ints, 2 grids of (3f, 3f, 3i, i), 7 ints, float, int, 7 floats, int, 16 bytes, float
     assert ctypes.sizeof(pkg.Emc2Grid) == 40
-    assert ctypes.sizeof(pkg.Emc2Config) == 16 + 80 + 28 + 4 + 4 + 28 + 4 + 16
+    assert ctypes.sizeof(pkg.Emc2Config) == 16 + 80 + 28 + 4 + 4 + 28 + 4 + 16 + 4
 
 
 def test_status_strings(pkg):

@@ -85,6 +85,33 @@ def test_one_call_on_a_side_stream_of_the_caller(b200, oracle):
     br.close()
 
 
+@pytest.mark.parametrize("p", [1, 2, 4])
+def test_multiscale_pooling_and_the_pooled_path(b200, oracle, p):
+    from dataclasses import replace
+    for base in (gen.KITTI.with_shape(2, 6000), gen.NUSCENES.with_shape(1, 9000)):
+        batch = gen.make_batch(base)
+        d = to_dev(batch)
+        br = b200.Bridge(b200.config_from_workload(base))
+        pooled = br.pool_features(d["feat"], p)
+        br.status()
+        want = oracle.pool(batch["feat"], p)
+        assert tuple(pooled.shape) == want.shape
+        assert np.abs(np_(pooled).astype(np.float64) - want).max() <= 1e-5
+        br.close()
+        # the whole bridge on the pooled maps: texels at the window centres, stride p * s
+        w = replace(base, feat_stride=base.feat_stride * p, feat_offset=(p - 1) / 2 * base.feat_stride)
+        assert (w.feat_h, w.feat_w) == want.shape[2:4]
+        pbatch = dict(batch, feat=want)
+        ref = oracle.bridge(w, pbatch)
+        br = b200.Bridge(b200.config_from_workload(w))
+        dp = to_dev(pbatch)
+        for step in (br.run, br.run_staged):
+            bufs = step(dp["points"], dp["proj"], dp["feat"])
+            br.status()
+            compare_bridge(w, ref, bufs)
+        br.close()
+
+
 def test_scene_route_matches_the_oracle(b200, oracle):
     w = gen.NUSCENES.with_shape(5, 4000)
     batch = gen.make_batch(w)
