@@ -4,7 +4,7 @@ import pytest
 import torch
 
 import emc2_gen as gen
-from parity import compare_bridge, np_, to_dev
+from parity import close, compare_bridge, np_, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -136,6 +136,61 @@ def test_scene_route_matches_the_oracle(b200, oracle):
 
 def test_sweep_cell_with_six_cameras(b200, oracle):
     run_case(b200, oracle, gen.SWEEP.with_shape(2, 65536))
+
+
+def test_largest_sweep_cell_on_sampled_frames(b200, oracle):
+    """32 frames x 524,288 points (the largest size a handle accepts), checked on two of the frames.
+
+    Frames are independent, so the oracle is run on the sampled frames alone and every output of
+    those frames is compared: voxel rows through their frame column, the rest by slicing."""
+    w = gen.SWEEP.with_shape(32, 524288)
+    sample = [5, 31]
+    pts = np.empty((w.B, w.N, w.C), np.float32)
+    for f in range(w.B):
+        pts[f] = gen.make_points(w, f % 4)               # four distinct clouds, repeated
+    pts[sample[1]] = gen.make_points(w, 7)               # and one frame of its own
+    proj = np.broadcast_to(gen.make_projection(w), (w.B, w.K, 3, 4)).copy()
+    fmap = gen.make_features(w, 0)
+    dev = "cuda"
+    d_pts, d_proj = torch.from_numpy(pts).to(dev), torch.from_numpy(proj).to(dev)
+    d_feat = torch.from_numpy(fmap).to(dev)[None].expand(w.B, -1, -1, -1, -1).contiguous()
+    br = b200.Bridge(b200.config_from_workload(w))
+    bufs = br.run(d_pts, d_proj, d_feat)
+    br.status()
+    sub = w.with_shape(len(sample), w.N)
+    ref = oracle.bridge(sub, {"points": pts[sample], "proj": proj[sample],
+                              "feat": np.broadcast_to(fmap, (len(sample),) + fmap.shape).copy()})
+    vox = bufs["vox"]
+    nv = np_(vox["num_voxels"])
+    for s in range(2):
+        coords = np_(vox["coords"][s])[:nv[s]]
+        counts = np_(vox["counts"][s])[:nv[s]]
+        mean = np_(vox["mean"][s])[:nv[s]]
+        pv = np_(vox["point_voxel"][s])
+        r = ref[f"vox{s}"]
+        for k, f in enumerate(sample):
+            rows = np.nonzero(coords[:, 0] == f)[0]
+            want = r["coords"][:, 0] == k
+            assert len(rows) == want.sum()
+            assert np.array_equal(coords[rows, 1:], r["coords"][want, 1:])
+            assert np.array_equal(counts[rows], r["counts"][want])
+            assert close(mean[rows], r["mean"][want])[0]
+            first = rows[0] if len(rows) else 0
+            base = np.nonzero(want)[0][0] if len(rows) else 0
+            got_pv, want_pv = pv[f], r["point_voxel"][k]
+            assert np.array_equal(got_pv >= 0, want_pv >= 0)
+            assert np.array_equal(got_pv[got_pv >= 0] - first, want_pv[want_pv >= 0] - base)
+    assert close(np_(vox["bev"][sample]), ref["bev"])[0]
+    pg, rd = bufs["pg"], bufs["rd"]
+    for name in ("vis_mask", "cam"):
+        assert np.array_equal(np_(pg[name][sample]), ref[name]), name
+    for name in ("expert", "offsets", "perm"):
+        assert np.array_equal(np_(rd[name][sample]), ref[name]), name
+    assert close(np_(pg["uvd"][sample]), ref["uvd"])[0]
+    assert close(np_(pg["gathered"][sample]), ref["gathered"])[0]
+    assert close(np_(rd["feat_out"][sample]), ref["feat_out"])[0]
+    assert np.array_equal(np_(rd["points_out"][sample]).view(np.uint32), ref["points_out"].view(np.uint32))
+    br.close()
 
 
 def test_degenerate_frames(b200, oracle):
