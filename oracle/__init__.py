@@ -138,6 +138,19 @@ def dispatch(expert: np.ndarray, points: np.ndarray, gathered: np.ndarray, num_e
     return offsets, perm, pout, fout
 
 
+def voxel_image(point_voxel: np.ndarray, num_voxels: int, vis_mask: np.ndarray, gathered: np.ndarray):
+    """Image features per voxel (Fig. 5): mean gathered row of the voxel's visible points, else zeros."""
+    pv = np.ascontiguousarray(point_voxel, np.int32).reshape(-1)
+    vis = np.ascontiguousarray(vis_mask, np.uint8).reshape(-1)
+    g = _f32(gathered).reshape(len(pv), -1)
+    M, Cf = int(num_voxels), g.shape[1]
+    out = np.empty((M, Cf), np.float32)
+    cnt = np.empty(M, np.int32)
+    lib().emc2o_voxel_image(ctypes.c_longlong(len(pv)), M, Cf, _p(pv, _I), _p(vis, _U8), _p(g, _F), _p(out, _F),
+                            _p(cnt, _I))
+    return out, cnt
+
+
 def scene_route(offsets: np.ndarray, priority: Sequence[int], min_points: int = 1) -> np.ndarray:
     """Scene-level expert per frame from the dispatch offsets (Sec. 3.2)."""
     offsets = np.ascontiguousarray(offsets, np.int32)

@@ -274,3 +274,25 @@ extern "C" void emc2o_scene_route(int B, int E, const int32_t* offsets, const ui
         scene_expert[b] = best;
     }
 }
+
+// Fusion by voxel (Fig. 5): the image features of the pixels that share a voxel's 3-D coordinate
+// go with that voxel; voxels without such pixels get zero-filled features.  Here the pixels with
+// a 3-D coordinate are the projected LiDAR points, so voxel m receives the mean of the gathered
+// rows of its kept points that some camera sees (vis_mask != 0), and a zero row if it has none.
+// point_voxel [B*N] (row of the point's voxel, -1 if none), vis_mask [B*N], gathered [B*N, Cf] ->
+// vox_img [M, Cf], vox_img_count [M] (points averaged).
+extern "C" void emc2o_voxel_image(long long total, int M, int Cf, const int32_t* point_voxel, const uint8_t* vis_mask,
+                                  const float* gathered, float* vox_img, int32_t* vox_img_count) {
+    std::vector<double> sums((size_t)M * Cf, 0.0);
+    for (int m = 0; m < M; ++m) vox_img_count[m] = 0;
+    for (long long i = 0; i < total; ++i) {
+        const int m = point_voxel[i];
+        if (m < 0 || m >= M || vis_mask[i] == 0) continue;
+        vox_img_count[m] += 1;
+        for (int c = 0; c < Cf; ++c) sums[(size_t)m * Cf + c] += (double)gathered[i * Cf + c];
+    }
+    for (int m = 0; m < M; ++m)
+        for (int c = 0; c < Cf; ++c)
+            vox_img[(size_t)m * Cf + c] =
+                vox_img_count[m] ? (float)(sums[(size_t)m * Cf + c] / (double)vox_img_count[m]) : 0.0f;
+}

@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) project_gather_
 
     float4* out = a.out + (size_t)g0 * cf4;
     const uint32_t dyv = (uint32_t)a.Wf * cf4;
-    if (CF4 > 0) {
+    if constexpr (CF4 > 0) {
         const int c = t % CF4, r0 = t / CF4;
 #pragma unroll 4
         for (int j = 0; j < kTile / 16; ++j) {
@@ -317,7 +317,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) gather_scatter_
     float4* out = a.gathered + g0 * cf4;
     float4* fdst = a.feat_out + f0 * cf4;
     const uint32_t dyv = (uint32_t)a.Wf * cf4;
-    if (CF4 > 0) {
+    if constexpr (CF4 > 0) {
         const int c = t % CF4, r0 = t / CF4;
 #pragma unroll 4
         for (int j = 0; j < kTile / 16; ++j) {

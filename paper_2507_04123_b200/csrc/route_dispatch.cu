@@ -207,7 +207,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) dispatch_scatte
     // eight rows (eight independent 128-bit streaming loads), then writes them to their slots.
     const float4* fsrc = a.feat + g0 * cf4;
     float4* fdst = a.feat_out + f0 * cf4;
-    if (CF4 > 0) {
+    if constexpr (CF4 > 0) {
         const int c = t % CF4, r0 = t / CF4;
 #pragma unroll
         for (int j0 = 0; j0 < kTile / 16; j0 += 8) {

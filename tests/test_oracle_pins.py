@@ -504,3 +504,33 @@ def test_gather_with_window_centre_offset(oracle):
     a = oracle.gather(uvd, np.zeros((1, 3), np.int8), feat, S)
     b = oracle.gather(uvd, np.zeros((1, 3), np.int8), feat, S, 0.0)
     assert np.array_equal(a, b)
+
+
+# ------------------------------------------------------------------ fusion by voxel (Fig. 5)
+def test_voxel_image_on_a_hand_built_frame(oracle):
+    # five points: voxel 0 holds points 0, 1 (visible) and 2 (not seen); voxel 1 holds only an unseen
+    # point; point 4 lies in no voxel.
+    pv = np.array([0, 0, 0, 1, -1], np.int32)
+    vis = np.array([1, 0x20, 0, 0, 1], np.uint8)
+    g = np.array([[1, 2], [3, 6], [100, 100], [7, 7], [9, 9]], F32)
+    img, cnt = oracle.voxel_image(pv, 2, vis, g)
+    assert list(cnt) == [2, 0]
+    assert np.array_equal(img, np.array([[2, 4], [0, 0]], F32))              # mean of rows 0 and 1; zero fill
+
+
+def test_voxel_image_against_index_add_on_a_generated_frame(oracle):
+    w = gen.NUSCENES.with_shape(2, 8000)
+    r = oracle.bridge(w, gen.make_batch(w))
+    for s in range(2):
+        v = r[f"vox{s}"]
+        img, cnt = oracle.voxel_image(v["point_voxel"], v["num_voxels"], r["vis_mask"], r["gathered"])
+        pv = torch.from_numpy(v["point_voxel"].reshape(-1).astype(np.int64))
+        ok = (pv >= 0) & torch.from_numpy(r["vis_mask"].reshape(-1) != 0)
+        sums = torch.zeros(v["num_voxels"], w.feat_c, dtype=torch.float64)
+        sums.index_add_(0, pv[ok], torch.from_numpy(r["gathered"].reshape(-1, w.feat_c)).double()[ok])
+        n = torch.zeros(v["num_voxels"], dtype=torch.float64).index_add_(0, pv[ok], torch.ones(int(ok.sum()), dtype=torch.float64))
+        assert np.array_equal(cnt, n.numpy().astype(np.int32))
+        want = torch.where(n[:, None] > 0, sums / n.clamp(min=1)[:, None], torch.zeros_like(sums)).numpy()
+        assert np.abs(img - want).max() < 1e-6
+        assert (cnt <= v["counts"]).all() and (cnt == 0).any() and (cnt > 1).any()
+        assert not img[cnt == 0].any()
