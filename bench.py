@@ -381,6 +381,24 @@ def run_ours(args, w):
     }
     if pool_info:
         line["multiscale_pooling"] = pool_info
+    if args.voxel_image:
+        # Fusion by voxel on the outputs of the step, per scale (three kernels each, timed together).
+        vi = {}
+        pg = bufs["pg"]
+        for sc in (0, 1):
+            out = br.voxel_image(bufs["vox"], sc, pg["vis_mask"], pg["gathered"])
+            fn = lambda: br.voxel_image(bufs["vox"], sc, pg["vis_mask"], pg["gathered"], out)
+            for _ in range(3):
+                fn()
+            secs_vi = time_steps(fn, args.steps, sync, barrier)
+            br.status()
+            M = int(nv[sc])
+            nvis = int(out["vox_img_count"][:M].sum().item())
+            vbytes = B * N * 5 + M * 4 + nvis * 4 * w.feat_c + M * (4 * w.feat_c + 4)
+            ms_vi = secs_vi / args.steps * 1e3
+            vi[f"scale{sc}"] = {"ms_per_call": ms_vi, "voxels": M, "visible_points": nvis,
+                                "algorithmic_bytes": vbytes, "achieved_gbs": vbytes / (ms_vi * 1e-3) / 1e9}
+        line["voxel_image"] = vi
     print(json.dumps(line), flush=True)
     if use_dist:
         dist.destroy_process_group()
@@ -431,6 +449,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--voxel-image", action="store_true", help="also time emc2_voxel_image (fusion by voxel)")
     ap.add_argument("--pool", type=int, default=1, help="Multiscale Pooling size p (power of two): pool the maps, "
                                                         "then run the bridge on the pooled maps")
     args = ap.parse_args()

@@ -172,6 +172,22 @@ int emc2_bridge_run(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_
 int emc2_pool_features(emc2_bridge_t* bridge, int32_t B, int32_t p, const float* d_feat, float* d_pooled,
                        void* cuda_stream);
 
+/* Fusion by voxel (Fig. 5: image features of the pixels that share a voxel's 3-D coordinate go with
+ * that voxel; voxels without such pixels get zero-filled features).  The pixels with a 3-D coordinate
+ * are the projected points, so for one voxel scale:
+ *   d_vox_img        float [capacity, Cf]  row m = mean of d_gathered over the points i with
+ *                                          d_point_voxel[i] == m and d_vis_mask[i] != 0; zeros if none
+ *   d_vox_img_count  int32 [capacity]      number of points averaged
+ * Inputs are outputs of the earlier stages for the SAME scale and batch: d_point_voxel [B, N],
+ * d_counts [capacity], d_num_voxels -> the scale's entry (DEVICE int32), d_vis_mask [B, N],
+ * d_gathered [B, N, Cf].  Rows past min(*d_num_voxels, capacity) are left untouched.  Concatenating
+ * [d_mean row | d_vox_img row] gives the fused voxel feature; the library leaves that to the consumer.
+ * Enqueues three kernels on `cuda_stream`; uses handle scratch, so calls on one handle must be
+ * ordered. */
+int emc2_voxel_image(emc2_bridge_t* bridge, int32_t B, int32_t N, int32_t capacity, const int32_t* d_point_voxel,
+                     const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
+                     const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, void* cuda_stream);
+
 /* Scene-level choice of the Scenario-Adaptive Dispatcher (Sec. 3.2): a scene is served by the most
  * demanding expert that any of its objects asks for.  Per point: for every frame b the expert of
  * highest priority[e] among the experts that own at least max(1, min_points) points of the frame

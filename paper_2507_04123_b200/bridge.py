@@ -34,6 +34,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
     "emc2_bridge_run", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
+    "emc2_voxel_image",
 )
 
 
@@ -81,6 +82,7 @@ def load_library() -> ctypes.CDLL:
                                     + [vp] * 4 + [vp] * 5 + [vp])
     lib.emc2_route_dispatch_static.argtypes = [P(Emc2Config), i32, i32] + [vp] * 9
     lib.emc2_bridge_status.argtypes = [vp, vp]
+    lib.emc2_voxel_image.argtypes = [vp, i32, i32, i32] + [vp] * 8
     lib.emc2_pool_features.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.emc2_scene_route.argtypes = [vp, i32, vp, P(ctypes.c_uint8), i32, vp, vp]
     lib.emc2_bridge_set_overlap.argtypes = [vp, ctypes.c_int]
@@ -287,6 +289,27 @@ class Bridge:
                                           out["points_out"].data_ptr(), out["feat_out"].data_ptr(),
                                           self._stream())
         self._raise(rc, "emc2_route_dispatch")
+        return out
+
+    def voxel_image(self, vox: Dict[str, object], scale: int, vis_mask: torch.Tensor, gathered: torch.Tensor,
+                    out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        """emc2_voxel_image for one scale of a :meth:`voxelize` result (needs its point_voxel)."""
+        B, N = vis_mask.shape
+        c = self.cfg
+        pv = vox["point_voxel"][scale]
+        counts = vox["counts"][scale]
+        cap = int(counts.shape[0])
+        _check(pv, torch.int32, (B, N), "point_voxel", self.device)
+        _check(vis_mask, torch.uint8, (B, N), "vis_mask", self.device)
+        _check(gathered, torch.float32, (B, N, c.feat_c), "gathered", self.device)
+        if out is None:
+            out = {"vox_img": torch.empty((cap, c.feat_c), dtype=torch.float32, device=self.device),
+                   "vox_img_count": torch.empty((cap,), dtype=torch.int32, device=self.device)}
+        nv = vox["num_voxels"]
+        rc = self.lib.emc2_voxel_image(self._h, B, N, cap, pv.data_ptr(), counts.data_ptr(),
+                                       nv.data_ptr() + 4 * scale, vis_mask.data_ptr(), gathered.data_ptr(),
+                                       out["vox_img"].data_ptr(), out["vox_img_count"].data_ptr(), self._stream())
+        self._raise(rc, "emc2_voxel_image")
         return out
 
     def pool_features(self, feat: torch.Tensor, p: int, out: Optional[torch.Tensor] = None) -> torch.Tensor:

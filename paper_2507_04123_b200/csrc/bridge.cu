@@ -9,7 +9,8 @@ namespace emc2 {
 
 static const char* const kKernelNames[K_KINDS] = {
     "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
-    "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features"};
+    "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features",
+    "vif_scan", "vif_fill", "vif_mean"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
     if (e == cudaSuccess) return EMC2_OK;
@@ -139,6 +140,8 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
 
     h->scan_blocks = voxel_scan_max_blocks();
     if (h->scan_blocks < 2) { delete h; return EMC2_ERR_CUDA; }
+    h->vif_scan_blocks = voxel_image_scan_max_blocks();
+    if (h->vif_scan_blocks < 1) { delete h; return EMC2_ERR_CUDA; }
 
     // Plan the slab: everything the stage calls need, allocated once.
     SlabPlan plan;
@@ -167,6 +170,10 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         o_tot[s] = plan.take(4 * sizeof(int));
     }
     const size_t o_part = plan.take((size_t)h->scan_blocks * 3 * sizeof(int));
+    const size_t o_vif_start = plan.take(maxpts * sizeof(int));
+    const size_t o_vif_cursor = plan.take(maxpts * sizeof(int));
+    const size_t o_vif_list = plan.take(maxpts * sizeof(int));
+    const size_t o_vif_part = plan.take((size_t)h->vif_scan_blocks * sizeof(int));
     const size_t o_wofs = plan.take((size_t)h->scan_blocks * (kThreads / 32) * 3 * sizeof(int));
     h->max_tiles = (c.max_points + kTile - 1) / kTile;
     const size_t tile_ints = (size_t)c.max_batch * h->max_tiles * c.num_experts;
@@ -195,6 +202,10 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         d.totals = reinterpret_cast<int*>(base + o_tot[s]);
     }
     h->d_scan_part = reinterpret_cast<int*>(base + o_part);
+    h->d_vif_start = reinterpret_cast<int*>(base + o_vif_start);
+    h->d_vif_cursor = reinterpret_cast<int*>(base + o_vif_cursor);
+    h->d_vif_list = reinterpret_cast<int*>(base + o_vif_list);
+    h->d_vif_part = reinterpret_cast<int*>(base + o_vif_part);
     h->d_scan_warp_ofs = reinterpret_cast<int*>(base + o_wofs);
     h->d_tile_counts = reinterpret_cast<int*>(base + o_tc);
     h->d_tile_base = reinterpret_cast<int*>(base + o_tb);
@@ -325,6 +336,22 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
     if (rc != EMC2_OK) return rc;
     if (rc2 != EMC2_OK) return rc2;
     return check_cuda(h, e);
+}
+
+int emc2_voxel_image(emc2_bridge_t* h, int32_t B, int32_t N, int32_t capacity, const int32_t* d_point_voxel,
+                     const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
+                     const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, void* cuda_stream) {
+    int rc = check_call(h, B, N);
+    if (rc != EMC2_OK) return rc;
+    if (capacity < 0 || !d_num_voxels) return EMC2_ERR_INVALID_ARG;
+    if (B == 0 || N == 0 || capacity == 0) return EMC2_OK;
+    if (!d_point_voxel || !d_counts || !d_vis_mask || !d_gathered || !d_vox_img || !d_vox_img_count)
+        return EMC2_ERR_INVALID_ARG;
+    if (!aligned16(d_gathered) || !aligned16(d_vox_img)) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_voxel_image(h, B, N, capacity, d_point_voxel, d_counts, d_num_voxels, d_vis_mask, d_gathered,
+                              d_vox_img, d_vox_img_count, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int emc2_pool_features(emc2_bridge_t* h, int32_t B, int32_t p, const float* d_feat, float* d_pooled,

@@ -32,6 +32,9 @@ enum KernelKind {
     K_DISPATCH_SCATTER,
     K_SCENE_ROUTE,
     K_POOL_FEATURES,
+    K_VIF_SCAN,
+    K_VIF_FILL,
+    K_VIF_MEAN,
     K_KINDS
 };
 
@@ -114,6 +117,11 @@ struct emc2_bridge {
     int* d_scan_warp_ofs = nullptr;  // [scan_blocks * 8][3] per-warp offsets inside their CTA
     int scan_blocks = 0;           // CTAs of the cooperative rank scan (all co-resident)
     bool thin_scan = false;        // set while emc2_bridge_run enqueues stage 1 beside stages 2 - 4
+    int* d_vif_start = nullptr;    // emc2_voxel_image: [max points] list starts, cursors, lists
+    int* d_vif_cursor = nullptr;
+    int* d_vif_list = nullptr;
+    int* d_vif_part = nullptr;     // [vif_scan_blocks]
+    int vif_scan_blocks = 0;
     int max_tiles = 0;
     bool overlap = true;           // emc2_bridge_run puts stage 1 on `side`
     cudaStream_t side = nullptr;   // stream of stage 1 inside emc2_bridge_run
@@ -161,6 +169,10 @@ inline RouteParams route_params(const emc2_bridge* h) {
     return rp;
 }
 
+int voxel_image_scan_max_blocks();
+int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t* d_point_voxel,
+                       const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
+                       const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st);
 int launch_pool_features(emc2_bridge* h, int B, int p, const float* d_feat, float* d_pooled, cudaStream_t st);
 int launch_scene_route(emc2_bridge* h, int B, const int32_t* d_offsets, const uint8_t* priority, int min_points,
                        int32_t* d_scene_expert, cudaStream_t st);

@@ -1,0 +1,168 @@
+// Fusion by voxel (Fig. 5): the image features of the pixels that share a voxel's 3-D coordinate
+// go with that voxel, voxels without such pixels get zero rows.  The pixels with a 3-D coordinate
+// are the projected LiDAR points, so voxel m receives the mean of the gathered rows of its kept
+// points that some camera sees.
+//
+// Rows are 256/320 bytes: adding them up with reductions would cost twenty 16-byte requests per
+// point.  Instead the points are listed per voxel and each voxel reads its points' rows whole:
+//   vif_scan   cooperative launch: exclusive prefix sum of the voxels' kept-point counts (the
+//              prefix-sum indexing of Sec. 3.6) -> start of every voxel's list; cursors cleared.
+//   vif_fill   every kept point takes a ticket in its voxel's list (one atomic with return).
+//   vif_mean   16 voxels x Cf/4 columns of threads per CTA: a voxel's threads walk its list and
+//              read each visible point's row with one contiguous 128-bit load per thread.
+#include <cooperative_groups.h>
+
+#include "bridge_internal.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace emc2 {
+namespace {
+
+struct VifArgs {
+    const int32_t* pv;          // [total] row of the point's voxel, -1 if none
+    const int32_t* counts;      // [M] kept points per voxel
+    const int32_t* num_voxels;  // device: voxels found by emc2_voxelize for this scale
+    const uint8_t* vis;         // [total]
+    const float4* gathered;     // [total, cf4]
+    float4* vox_img;            // [capacity, cf4]
+    int32_t* vox_cnt;           // [capacity]
+    int* start;                 // [capacity] first list slot of each voxel
+    int* cursor;                // [capacity]
+    int* list;                  // [total] point indices; bitwise complement for points no camera sees
+    int* part;                  // [gridDim.x]
+    long long total;
+    int capacity, cf4;
+};
+
+__device__ __forceinline__ int voxels_in_use(const VifArgs& a) { return min(*a.num_voxels, a.capacity); }
+
+// Every thread owns a run of consecutive voxels.  CTA totals, grid barrier, then the prefix.
+__global__ void __launch_bounds__(kThreads) vif_scan_kernel(VifArgs a) {
+    __shared__ int wsum[kThreads / 32];
+    __shared__ int s_base;
+    cg::grid_group grid = cg::this_grid();
+    const int M = voxels_in_use(a);
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const long long nthreads = (long long)gridDim.x * kThreads;
+    const int per = (int)((M + nthreads - 1) / nthreads);
+    const long long lo64 = ((long long)blockIdx.x * kThreads + t) * per;
+    const int lo = (int)min((long long)M, lo64), hi = (int)min((long long)M, lo64 + per);
+    int sum = 0;
+    for (int m = lo; m < hi; ++m) sum += a.counts[m];
+    int inc = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += y;
+    }
+    if (lane == 31) wsum[warp] = inc;
+    __syncthreads();
+    int before = 0, cta_total = 0;
+    for (int w = 0; w < kThreads / 32; ++w) {
+        if (w < warp) before += wsum[w];
+        cta_total += wsum[w];
+    }
+    if (t == 0) a.part[blockIdx.x] = cta_total;
+    grid.sync();
+    if (warp == 0) {
+        int v = 0;
+        for (int c = lane; c < (int)blockIdx.x; c += 32) v += a.part[c];
+        v = warp_sum(v);
+        if (lane == 0) s_base = v;
+    }
+    __syncthreads();
+    int run = s_base + before + inc - sum;
+    for (int m = lo; m < hi; ++m) {
+        a.start[m] = run;
+        a.cursor[m] = 0;
+        run += a.counts[m];
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) vif_fill_kernel(VifArgs a) {
+    const int M = voxels_in_use(a);
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < a.total; i += (long long)gridDim.x * kThreads) {
+        const int m = a.pv[i];
+        if (m < 0 || m >= M) continue;
+        const int pos = a.start[m] + atomicAdd(&a.cursor[m], 1);
+        a.list[pos] = a.vis[i] ? (int)i : ~(int)i;
+    }
+}
+
+// CF4 > 0: Cf/4 known at compile time, blockDim.x == 16 * CF4.  CF4 == 0: any Cf, 256 threads.
+template <int CF4>
+__global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_mean_kernel(VifArgs a) {
+    const int M = voxels_in_use(a);
+    const int cf4 = CF4 > 0 ? CF4 : a.cf4;
+    const int rows = (int)blockDim.x / cf4;                  // voxels a CTA handles at a time
+    const int r = (int)threadIdx.x / cf4, c = (int)threadIdx.x - r * cf4;
+    if (r >= rows) return;
+    for (int m = blockIdx.x * rows + r; m < M; m += gridDim.x * rows) {
+        const int s0 = a.start[m], n = a.counts[m];
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        int seen = 0;
+        for (int k = 0; k < n; ++k) {
+            const int i = a.list[s0 + k];
+            if (i < 0) continue;
+            const float4 v = __ldcs(a.gathered + (size_t)i * cf4 + c);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            seen += 1;
+        }
+        if (seen > 1) {
+            const float inv = 1.0f / (float)seen;
+            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        }
+        __stcs(a.vox_img + (size_t)m * cf4 + c, acc);
+        if (c == 0) a.vox_cnt[m] = seen;
+    }
+}
+
+}  // namespace
+
+int voxel_image_scan_max_blocks() {
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, vif_scan_kernel, kThreads, 0) != cudaSuccess) return 0;
+    return sms * min(per_sm, 2);
+}
+
+int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t* d_point_voxel,
+                       const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
+                       const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st) {
+    VifArgs a;
+    a.pv = d_point_voxel; a.counts = d_counts; a.num_voxels = d_num_voxels; a.vis = d_vis_mask;
+    a.gathered = reinterpret_cast<const float4*>(d_gathered);
+    a.vox_img = reinterpret_cast<float4*>(d_vox_img); a.vox_cnt = d_vox_img_count;
+    a.start = h->d_vif_start; a.cursor = h->d_vif_cursor; a.list = h->d_vif_list; a.part = h->d_vif_part;
+    a.total = (long long)B * N;
+    a.capacity = (int)min((long long)capacity, a.total);   // a voxel holds at least one point
+    a.cf4 = h->cfg.feat_c / 4;
+    if (a.total == 0 || a.capacity == 0) return EMC2_OK;
+    if (a.cf4 > kThreads) return EMC2_ERR_INVALID_ARG;      // a feature row must fit one CTA
+    {
+        LaunchScope ls(h, K_VIF_SCAN, st);
+        void* args[] = {&a};
+        cudaError_t e = cudaLaunchCooperativeKernel((const void*)vif_scan_kernel, dim3(h->vif_scan_blocks),
+                                                    dim3(kThreads), args, 0, st);
+        if (e != cudaSuccess) return check_cuda(h, e);
+    }
+    {
+        LaunchScope ls(h, K_VIF_FILL, st);
+        const int blocks = (int)min((long long)148 * 16, (a.total + kThreads - 1) / kThreads);
+        vif_fill_kernel<<<blocks, kThreads, 0, st>>>(a);
+    }
+    {
+        LaunchScope ls(h, K_VIF_MEAN, st);
+        const int blocks = (int)min((long long)148 * 16, ((long long)a.capacity + 15) / 16);
+        switch (a.cf4) {
+            case 16: vif_mean_kernel<16><<<blocks, 16 * 16, 0, st>>>(a); break;
+            case 20: vif_mean_kernel<20><<<blocks, 16 * 20, 0, st>>>(a); break;
+            default: vif_mean_kernel<0><<<blocks, kThreads, 0, st>>>(a); break;
+        }
+    }
+    return check_cuda(h, cudaGetLastError());
+}
+
+}  // namespace emc2

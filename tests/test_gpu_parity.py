@@ -112,6 +112,27 @@ def test_multiscale_pooling_and_the_pooled_path(b200, oracle, p):
         br.close()
 
 
+@pytest.mark.parametrize("cid,B,N", [(2, 2, 50_000), (1, 3, 33_333), (3, 1, 300_000), (2, 1, 1)])
+def test_image_features_per_voxel(b200, oracle, cid, B, N):
+    w = gen.workload(cid).with_shape(B, N)
+    batch = gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    for rep in range(2):                           # twice: the lists must not depend on old cursors
+        for s in range(2):
+            out = br.voxel_image(bufs["vox"], s, bufs["pg"]["vis_mask"], bufs["pg"]["gathered"])
+            br.status()
+            M = ref[f"vox{s}"]["num_voxels"]
+            want, cnt = oracle.voxel_image(ref[f"vox{s}"]["point_voxel"], M, ref["vis_mask"], ref["gathered"])
+            assert np.array_equal(np_(out["vox_img_count"])[:M], cnt), s
+            ok, mx, nbad = close(np_(out["vox_img"])[:M], want)
+            assert ok, f"scale {s}: max abs err {mx}, {nbad} outside tolerance"
+            assert not np_(out["vox_img"])[:M][cnt == 0].any()
+    br.close()
+
+
 def test_scene_route_matches_the_oracle(b200, oracle):
     w = gen.NUSCENES.with_shape(5, 4000)
     batch = gen.make_batch(w)
