@@ -151,6 +151,22 @@ def voxel_image(point_voxel: np.ndarray, num_voxels: int, vis_mask: np.ndarray, 
     return out, cnt
 
 
+def occlusion(points: np.ndarray, proj: np.ndarray, H: int, W: int, vis_mask: np.ndarray, cell: int,
+              margin: float):
+    """Depth-buffer occlusion per camera: (zbuf [B,K,Hz,Wz], occ_mask, clear_mask)."""
+    points, proj = _f32(points), _f32(proj)
+    B, N, C = points.shape
+    K = proj.shape[1]
+    vis = np.ascontiguousarray(vis_mask, np.uint8)
+    Hz, Wz = -(-H // cell), -(-W // cell)
+    zbuf = np.empty((B, K, Hz, Wz), np.float32)
+    occ = np.empty((B, N), np.uint8)
+    clear = np.empty((B, N), np.uint8)
+    lib().emc2o_occlusion(B, N, C, K, _p(points, _F), _p(proj, _F), H, W, _p(vis, _U8), int(cell),
+                          ctypes.c_float(margin), _p(zbuf, _F), _p(occ, _U8), _p(clear, _U8))
+    return zbuf, occ, clear
+
+
 def scene_route(offsets: np.ndarray, priority: Sequence[int], min_points: int = 1) -> np.ndarray:
     """Scene-level expert per frame from the dispatch offsets (Sec. 3.2)."""
     offsets = np.ascontiguousarray(offsets, np.int32)

@@ -296,3 +296,52 @@ extern "C" void emc2o_voxel_image(long long total, int M, int Cf, const int32_t*
             vox_img[(size_t)m * Cf + c] =
                 vox_img_count[m] ? (float)(sums[(size_t)m * Cf + c] / (double)vox_img_count[m]) : 0.0f;
 }
+
+// Occlusion test for the "occluded / out-of-view" bucket.  The paper names occlusion as a cause of
+// missing LiDAR detail (Sec. 3.2, case 3) but gives no test; this is the usual depth-buffer one.
+// Every camera image is cut into cells of `cell` x `cell` pixels (cell a power of two).  For each
+// camera that sees a point (bit k of vis_mask), the point falls into cell (floor(v/cell),
+// floor(u/cell)) with depth d, both from the same fp32 projection as emc2o_project.  zbuf holds the
+// smallest depth per cell.  The point is occluded in camera k iff d > zbuf + margin (fp32 add,
+// fp32 compare).  occ_mask bit k = occluded in camera k; clear_mask = vis_mask & ~occ_mask.
+// zbuf [B,K,Hz,Wz] with Hz = ceil(H/cell), Wz = ceil(W/cell); +infinity where no point falls.
+extern "C" void emc2o_occlusion(int B, int N, int C, int K, const float* points, const float* proj, int H, int W,
+                                const uint8_t* vis_mask, int cell, float margin, float* zbuf, uint8_t* occ_mask,
+                                uint8_t* clear_mask) {
+    const int Hz = (H + cell - 1) / cell, Wz = (W + cell - 1) / cell;
+    const float inv = 1.0f / (float)cell;
+    const size_t nz = (size_t)B * K * Hz * Wz;
+    for (size_t i = 0; i < nz; ++i) zbuf[i] = INFINITY;
+    std::vector<float> depth((size_t)B * N * K, 0.0f);
+    std::vector<int> where((size_t)B * N * K, -1);
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < N; ++i) {
+            const int64_t g = (int64_t)b * N + i;
+            const float x = points[g * C + 0], y = points[g * C + 1], z = points[g * C + 2];
+            for (int k = 0; k < K; ++k) {
+                if (!((vis_mask[g] >> k) & 1)) continue;
+                const float* P = proj + ((size_t)b * K + k) * 12;
+                float t[3];
+                for (int r = 0; r < 3; ++r)
+                    t[r] = std::fmaf(P[4 * r + 0], x,
+                                     std::fmaf(P[4 * r + 1], y, std::fmaf(P[4 * r + 2], z, P[4 * r + 3])));
+                const float u = t[0] / t[2], v = t[1] / t[2];
+                const int cx = std::min((int)std::floor(u * inv), Wz - 1), cy = std::min((int)std::floor(v * inv), Hz - 1);
+                const size_t c = (((size_t)b * K + k) * Hz + cy) * Wz + cx;
+                depth[g * K + k] = t[2];
+                where[g * K + k] = (int)c;
+                zbuf[c] = std::min(zbuf[c], t[2]);
+            }
+        }
+    for (int64_t g = 0; g < (int64_t)B * N; ++g) {
+        unsigned occ = 0;
+        for (int k = 0; k < K; ++k) {
+            const int c = where[g * K + k];
+            if (c < 0) continue;
+            const float lim = zbuf[c] + margin;
+            if (depth[g * K + k] > lim) occ |= 1u << k;
+        }
+        occ_mask[g] = (uint8_t)occ;
+        clear_mask[g] = (uint8_t)(vis_mask[g] & ~occ);
+    }
+}

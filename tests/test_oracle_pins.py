@@ -534,3 +534,50 @@ def test_voxel_image_against_index_add_on_a_generated_frame(oracle):
         assert np.abs(img - want).max() < 1e-6
         assert (cnt <= v["counts"]).all() and (cnt == 0).any() and (cnt > 1).any()
         assert not img[cnt == 0].any()
+
+
+# ------------------------------------------------------------------ depth-buffer occlusion
+def test_occlusion_on_hand_built_rays(oracle):
+    P, _ = _proj1(512.0, 256.0, 640.0, 128.0)            # 1280 x 512 image, principal point (640, 128)
+    rows = [(5.0, 0.0, 0.0),                             # on the optical axis, 5 m
+            (9.0, 0.0, 0.0),                             # same ray, 9 m: hidden by the first
+            (5.25, 0.0, 0.0),                            # same ray, inside the margin: not hidden
+            (9.0, -9.0 * 200 / 512, 0.0),                # 200 px to the right: another cell, alone there
+            (-3.0, 0.0, 0.0),                            # behind the camera: never occluded, never clear
+            (5.5, 0.0, 0.0)]                             # exactly first depth + margin: not hidden (strict >)
+    pts = _pts(rows)
+    _, vis, _ = oracle.project(pts, P, 512, 1280, 0.1)
+    zbuf, occ, clear = oracle.occlusion(pts, P, 512, 1280, vis, 16, 0.5)
+    assert zbuf.shape == (1, 1, 32, 80)
+    assert list(vis[0]) == [1, 1, 1, 1, 0, 1]
+    assert list(occ[0]) == [0, 1, 0, 0, 0, 0]
+    assert list(clear[0]) == [1, 0, 1, 1, 0, 1]
+    assert zbuf[0, 0, 128 // 16, 640 // 16] == 5.0 and zbuf[0, 0, 8, (640 + 200) // 16] == 9.0
+    assert np.isinf(zbuf).sum() == zbuf.size - 2
+    # a larger margin hides nothing; margin 0 hides everything behind the nearest point of a cell
+    assert not oracle.occlusion(pts, P, 512, 1280, vis, 16, 10.0)[1].any()
+    assert list(oracle.occlusion(pts, P, 512, 1280, vis, 16, 0.0)[1][0]) == [0, 1, 1, 0, 0, 1]
+
+
+def test_occlusion_against_brute_force(oracle):
+    w = gen.NUSCENES.with_shape(1, 400)
+    batch = gen.make_batch(w)
+    pts, P = batch["points"], batch["proj"]
+    pts[0, :, :2] *= 0.3                                  # crowd the points so that cells are shared
+    uvd, vis, cam = oracle.project(pts, P, w.img_h, w.img_w, w.min_depth)
+    cell, margin = 64, 0.75
+    zbuf, occ, clear = oracle.occlusion(pts, P, w.img_h, w.img_w, vis, cell, margin)
+    assert occ.any() and (clear != vis).any()
+    # brute force per camera: re-project each camera alone through the oracle's own projection
+    for k in range(w.K):
+        uk, vk, _ = oracle.project(pts, P[:, k:k + 1], w.img_h, w.img_w, w.min_depth)
+        seen = np.nonzero(vk[0])[0]
+        assert np.array_equal(vk[0] != 0, ((vis[0] >> k) & 1) != 0)
+        cx = np.floor(uk[0, :, 0] / cell).astype(int)
+        cy = np.floor(uk[0, :, 1] / cell).astype(int)
+        for i in seen:
+            same = [j for j in seen if cx[j] == cx[i] and cy[j] == cy[i]]
+            nearest = min(uk[0, j, 2] for j in same)
+            assert zbuf[0, k, cy[i], cx[i]] == nearest
+            assert bool((occ[0, i] >> k) & 1) == bool(uk[0, i, 2] > F32(nearest) + F32(margin))
+    assert np.array_equal(clear, vis & ~occ)
