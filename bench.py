@@ -381,6 +381,21 @@ def run_ours(args, w):
     }
     if pool_info:
         line["multiscale_pooling"] = pool_info
+    if args.occlusion:
+        # Depth-buffer occlusion on the step's visibility mask (three kernels, timed together).
+        cell = w.feat_stride
+        occ = br.occlusion(d["points"], d["proj"], bufs["pg"]["vis_mask"], cell, 0.5)
+        fn = lambda: br.occlusion(d["points"], d["proj"], bufs["pg"]["vis_mask"], cell, 0.5, occ)
+        for _ in range(3):
+            fn()
+        secs_oc = time_steps(fn, args.steps, sync, barrier)
+        br.status()
+        obytes = 2 * B * N * (4 * w.C + 1) + occ["zbuf"].numel() * 4 + 2 * B * N
+        ms_oc = secs_oc / args.steps * 1e3
+        line["occlusion"] = {"cell_px": cell, "margin_m": 0.5, "ms_per_call": ms_oc, "algorithmic_bytes": obytes,
+                             "achieved_gbs": obytes / (ms_oc * 1e-3) / 1e9,
+                             "occluded_share_of_visible": float((occ["occ_mask"] != 0).sum().item())
+                             / max(1.0, float((bufs["pg"]["vis_mask"] != 0).sum().item()))}
     if args.voxel_image:
         # Fusion by voxel on the outputs of the step, per scale (three kernels each, timed together).
         vi = {}
@@ -449,6 +464,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--occlusion", action="store_true", help="also time emc2_occlusion (depth-buffer test)")
     ap.add_argument("--voxel-image", action="store_true", help="also time emc2_voxel_image (fusion by voxel)")
     ap.add_argument("--pool", type=int, default=1, help="Multiscale Pooling size p (power of two): pool the maps, "
                                                         "then run the bridge on the pooled maps")

@@ -188,6 +188,23 @@ int emc2_voxel_image(emc2_bridge_t* bridge, int32_t B, int32_t N, int32_t capaci
                      const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
                      const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, void* cuda_stream);
 
+/* Occlusion test for the "occluded / out-of-view" bucket of the dispatcher (Sec. 3.2 names occlusion
+ * among the causes of missing LiDAR detail; the paper gives no test, this is a depth buffer).  Every
+ * camera image is cut into cells of cell x cell pixels (cell a power of two).  For each camera k that
+ * sees a point (bit k of d_vis_mask) the point falls into cell (floor(v/cell), floor(u/cell)) with its
+ * depth d; the buffer keeps the smallest depth per cell; the point is occluded in camera k iff
+ * d > buffer + margin (fp32).
+ *   d_vis_mask    uint8 [B, N]            from emc2_project_gather / emc2_bridge_run (same points, proj)
+ *   d_zbuf        float [B, K, Hz, Wz]    Hz = ceil(H/cell), Wz = ceil(W/cell); written: the smallest
+ *                                         depth per cell, +infinity where no point falls
+ *   d_occ_mask    uint8 [B, N]            bit k: occluded in camera k
+ *   d_clear_mask  uint8 [B, N]            d_vis_mask & ~d_occ_mask: pass this to emc2_route_dispatch in
+ *                                         place of d_vis_mask to route occluded points as not visible
+ * margin >= 0, metres.  Enqueues three kernels on `cuda_stream`. */
+int emc2_occlusion(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_points, const float* d_proj,
+                   const uint8_t* d_vis_mask, int32_t cell, float margin, float* d_zbuf, uint8_t* d_occ_mask,
+                   uint8_t* d_clear_mask, void* cuda_stream);
+
 /* Scene-level choice of the Scenario-Adaptive Dispatcher (Sec. 3.2): a scene is served by the most
  * demanding expert that any of its objects asks for.  Per point: for every frame b the expert of
  * highest priority[e] among the experts that own at least max(1, min_points) points of the frame

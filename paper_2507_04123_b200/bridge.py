@@ -34,7 +34,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
     "emc2_bridge_run", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
-    "emc2_voxel_image",
+    "emc2_voxel_image", "emc2_occlusion",
 )
 
 
@@ -82,6 +82,7 @@ def load_library() -> ctypes.CDLL:
                                     + [vp] * 4 + [vp] * 5 + [vp])
     lib.emc2_route_dispatch_static.argtypes = [P(Emc2Config), i32, i32] + [vp] * 9
     lib.emc2_bridge_status.argtypes = [vp, vp]
+    lib.emc2_occlusion.argtypes = [vp, i32, i32, vp, vp, vp, i32, ctypes.c_float, vp, vp, vp, vp]
     lib.emc2_voxel_image.argtypes = [vp, i32, i32, i32] + [vp] * 8
     lib.emc2_pool_features.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.emc2_scene_route.argtypes = [vp, i32, vp, P(ctypes.c_uint8), i32, vp, vp]
@@ -310,6 +311,25 @@ class Bridge:
                                        nv.data_ptr() + 4 * scale, vis_mask.data_ptr(), gathered.data_ptr(),
                                        out["vox_img"].data_ptr(), out["vox_img_count"].data_ptr(), self._stream())
         self._raise(rc, "emc2_voxel_image")
+        return out
+
+    def occlusion(self, points: torch.Tensor, proj: torch.Tensor, vis_mask: torch.Tensor, cell: int,
+                  margin: float, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        """emc2_occlusion: depth buffer per camera cell, occluded bits, mask of clear views."""
+        B, N, C = points.shape
+        c = self.cfg
+        _check(points, torch.float32, (B, N, c.point_floats), "points", self.device)
+        _check(proj, torch.float32, (B, c.num_cameras, 3, 4), "proj", self.device)
+        _check(vis_mask, torch.uint8, (B, N), "vis_mask", self.device)
+        if out is None:
+            shape = (B, c.num_cameras, -(-c.img_h // cell), -(-c.img_w // cell))
+            out = {"zbuf": torch.empty(shape, dtype=torch.float32, device=self.device),
+                   "occ_mask": torch.empty((B, N), dtype=torch.uint8, device=self.device),
+                   "clear_mask": torch.empty((B, N), dtype=torch.uint8, device=self.device)}
+        rc = self.lib.emc2_occlusion(self._h, B, N, points.data_ptr(), proj.data_ptr(), vis_mask.data_ptr(),
+                                     int(cell), float(margin), out["zbuf"].data_ptr(), out["occ_mask"].data_ptr(),
+                                     out["clear_mask"].data_ptr(), self._stream())
+        self._raise(rc, "emc2_occlusion")
         return out
 
     def pool_features(self, feat: torch.Tensor, p: int, out: Optional[torch.Tensor] = None) -> torch.Tensor:

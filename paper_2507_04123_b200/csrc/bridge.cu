@@ -10,7 +10,7 @@ namespace emc2 {
 static const char* const kKernelNames[K_KINDS] = {
     "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
     "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features",
-    "vif_scan", "vif_fill", "vif_mean"};
+    "vif_scan", "vif_fill", "vif_mean", "occl_fill", "occl_splat", "occl_test"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
     if (e == cudaSuccess) return EMC2_OK;
@@ -352,6 +352,21 @@ int emc2_voxel_image(emc2_bridge_t* h, int32_t B, int32_t N, int32_t capacity, c
     if (!guard.ok) return EMC2_ERR_CUDA;
     return launch_voxel_image(h, B, N, capacity, d_point_voxel, d_counts, d_num_voxels, d_vis_mask, d_gathered,
                               d_vox_img, d_vox_img_count, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int emc2_occlusion(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points, const float* d_proj,
+                   const uint8_t* d_vis_mask, int32_t cell, float margin, float* d_zbuf, uint8_t* d_occ_mask,
+                   uint8_t* d_clear_mask, void* cuda_stream) {
+    int rc = check_call(h, B, N);
+    if (rc != EMC2_OK) return rc;
+    if (!is_pow2(cell) || !(margin >= 0.0f) || !std::isfinite(margin)) return EMC2_ERR_INVALID_ARG;
+    if (B == 0) return EMC2_OK;
+    if (!d_zbuf || !d_proj || !aligned16(d_proj)) return EMC2_ERR_INVALID_ARG;
+    if (N > 0 && (!d_points || !d_vis_mask || !d_occ_mask || !d_clear_mask)) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_occlusion(h, B, N, d_points, d_proj, d_vis_mask, cell, margin, reinterpret_cast<uint32_t*>(d_zbuf),
+                            d_occ_mask, d_clear_mask, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int emc2_pool_features(emc2_bridge_t* h, int32_t B, int32_t p, const float* d_feat, float* d_pooled,

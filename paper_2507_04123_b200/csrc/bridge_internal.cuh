@@ -35,6 +35,9 @@ enum KernelKind {
     K_VIF_SCAN,
     K_VIF_FILL,
     K_VIF_MEAN,
+    K_OCCL_FILL,
+    K_OCCL_SPLAT,
+    K_OCCL_TEST,
     K_KINDS
 };
 
@@ -169,6 +172,9 @@ inline RouteParams route_params(const emc2_bridge* h) {
     return rp;
 }
 
+int launch_occlusion(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj,
+                     const uint8_t* d_vis_mask, int cell, float margin, uint32_t* d_zbuf, uint8_t* d_occ_mask,
+                     uint8_t* d_clear_mask, cudaStream_t st);
 int voxel_image_scan_max_blocks();
 int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t* d_point_voxel,
                        const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,

@@ -133,6 +133,35 @@ def test_image_features_per_voxel(b200, oracle, cid, B, N):
     br.close()
 
 
+@pytest.mark.parametrize("cid,B,N,cell,margin", [(2, 2, 120_000, 8, 0.5), (1, 3, 40_001, 4, 0.25),
+                                                 (3, 1, 300_000, 16, 1.0), (2, 1, 5000, 64, 0.0)])
+def test_occlusion_and_routing_of_occluded_points(b200, oracle, cid, B, N, cell, margin):
+    w = gen.workload(cid).with_shape(B, N)
+    batch = gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    zbuf, occ, clear = oracle.occlusion(batch["points"], batch["proj"], w.img_h, w.img_w, ref["vis_mask"], cell, margin)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    out = None
+    for _ in range(2):
+        out = br.occlusion(d["points"], d["proj"], bufs["pg"]["vis_mask"], cell, margin, out)
+    br.status()
+    assert np.array_equal(np_(out["zbuf"]).view(np.uint32), zbuf.view(np.uint32))      # exact, +inf included
+    assert np.array_equal(np_(out["occ_mask"]), occ)
+    assert np.array_equal(np_(out["clear_mask"]), clear)
+    assert occ.any()
+    # occluded points routed as not visible
+    rd = br.route_dispatch(d["points"], out["clear_mask"], bufs["pg"]["gathered"])
+    br.status()
+    ex = oracle.route(batch["points"], clear, w.thresholds, w.lut)
+    off, perm, _, _ = oracle.dispatch(ex, batch["points"], ref["gathered"], w.num_experts)
+    assert np.array_equal(np_(rd["expert"]), ex) and np.array_equal(np_(rd["offsets"]), off)
+    assert np.array_equal(np_(rd["perm"]), perm)
+    assert (ex != ref["expert"]).any()
+    br.close()
+
+
 def test_scene_route_matches_the_oracle(b200, oracle):
     w = gen.NUSCENES.with_shape(5, 4000)
     batch = gen.make_batch(w)
