@@ -18,9 +18,11 @@
  *     the caller, contiguous, row-major and 16-byte aligned.  Pointers named
  *     h_* or without prefix are HOST memory.  The library never frees or keeps
  *     a caller pointer after the call has been enqueued.
- *   - The three stage calls only enqueue kernels on `cuda_stream` (a
- *     cudaStream_t passed as void*, NULL = legacy default stream).  They do not
+ *   - Every call that takes `cuda_stream` (a cudaStream_t passed as void*,
+ *     NULL = legacy default stream) only enqueues kernels.  These calls do not
  *     allocate, do not synchronise and do not touch the host except to return.
+ *     Some kernels are cooperative launches (grid-wide barrier), which the
+ *     device must support; emc2_bridge_create() fails otherwise.
  *   - One handle serves one device and one stream at a time; it is not
  *     thread-safe.  Calls on the same handle must be ordered on the stream.
  *   - Errors are returned as negative emc2_status_t values.  Errors the host
@@ -46,7 +48,9 @@ typedef enum {
     EMC2_ERR_BAD_CONFIG = -2,  /* emc2_config_t rejected by emc2_bridge_create */
     EMC2_ERR_CUDA = -3,        /* a CUDA runtime call failed; see emc2_bridge_last_cuda_error */
     EMC2_ERR_CAPACITY = -4,    /* more unique voxels than capacity[s] (device-detected, sticky) */
-    EMC2_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (device-detected, sticky) */
+    EMC2_ERR_TIMEOUT = -5,     /* reserved: a bounded device-side wait gave up.  No kernel of this library
+                                  spins on another CTA (the only grid-wide waits are the barriers of
+                                  cooperative launches), so it is never returned at present */
     EMC2_ERR_INTERNAL = -6,
     EMC2_ERR_TOO_LARGE = -7    /* the call needs more scratch than a fixed-size scratch area holds */
 } emc2_status_t;

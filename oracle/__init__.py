@@ -86,6 +86,15 @@ def project(points: np.ndarray, proj: np.ndarray, H: int, W: int, min_depth: flo
     return uvd, mask, cam
 
 
+def channels_last(planar: np.ndarray) -> np.ndarray:
+    """[B,K,Cf,Hf,Wf] -> [B,K,Hf,Wf,Cf] (a copy)."""
+    planar = _f32(planar)
+    B, K, Cf, Hf, Wf = planar.shape
+    out = np.empty((B, K, Hf, Wf, Cf), np.float32)
+    lib().emc2o_channels_last(B * K, Cf, Hf, Wf, _p(planar, _F), _p(out, _F))
+    return out
+
+
 def pool(feat: np.ndarray, p: int) -> np.ndarray:
     """p x p average pooling of channels-last feature maps (Sec. 3.5, Multiscale Pooling)."""
     feat = _f32(feat)

@@ -345,3 +345,13 @@ extern "C" void emc2o_occlusion(int B, int N, int C, int K, const float* points,
         clear_mask[g] = (uint8_t)(vis_mask[g] & ~occ);
     }
 }
+
+// Layout change for callers whose image branch emits planar maps: [B,K,Cf,Hf,Wf] -> the
+// channels-last [B,K,Hf,Wf,Cf] the gather reads.  A pure copy.
+extern "C" void emc2o_channels_last(int maps, int Cf, int Hf, int Wf, const float* planar, float* last) {
+    for (int m = 0; m < maps; ++m)
+        for (int c = 0; c < Cf; ++c)
+            for (int j = 0; j < Hf; ++j)
+                for (int i = 0; i < Wf; ++i)
+                    last[(((size_t)m * Hf + j) * Wf + i) * Cf + c] = planar[(((size_t)m * Cf + c) * Hf + j) * Wf + i];
+}

@@ -581,3 +581,9 @@ def test_occlusion_against_brute_force(oracle):
             assert zbuf[0, k, cy[i], cx[i]] == nearest
             assert bool((occ[0, i] >> k) & 1) == bool(uk[0, i, 2] > F32(nearest) + F32(margin))
     assert np.array_equal(clear, vis & ~occ)
+
+
+def test_channels_last_is_numpys_transpose(oracle):
+    rng = np.random.default_rng(14)
+    x = rng.standard_normal((2, 3, 7, 5, 11)).astype(F32)
+    assert np.array_equal(oracle.channels_last(x), np.ascontiguousarray(x.transpose(0, 1, 3, 4, 2)))
