@@ -414,6 +414,22 @@ def run_ours(args, w):
             vi[f"scale{sc}"] = {"ms_per_call": ms_vi, "voxels": M, "visible_points": nvis,
                                 "algorithmic_bytes": vbytes, "achieved_gbs": vbytes / (ms_vi * 1e-3) / 1e9}
         line["voxel_image"] = vi
+    if args.channels_last:
+        # Planar maps -> channels-last, its own kernel timed alone (a pure copy: bytes = 2 x the maps).
+        planar = d["feat"].permute(0, 1, 4, 2, 3).contiguous()
+        cl = br.features_channels_last(planar)
+        assert torch.equal(cl, d["feat"])
+        fn = lambda: br.features_channels_last(planar, cl)
+        for _ in range(3):
+            fn()
+        secs_cl = time_steps(fn, args.steps, sync, barrier)
+        br.status()
+        cbytes = 2 * planar.numel() * 4
+        ms_cl = secs_cl / args.steps * 1e3
+        peak1, kind1 = measured_peak()
+        line["channels_last"] = {"ms_per_call": ms_cl, "algorithmic_bytes": cbytes,
+                                 "achieved_gbs": cbytes / (ms_cl * 1e-3) / 1e9,
+                                 f"frac_of_{kind1}_copy": cbytes / (ms_cl * 1e-3) / 1e9 / peak1}
     print(json.dumps(line), flush=True)
     if use_dist:
         dist.destroy_process_group()
@@ -465,6 +481,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--occlusion", action="store_true", help="also time emc2_occlusion (depth-buffer test)")
+    ap.add_argument("--channels-last", action="store_true", help="also time emc2_features_channels_last")
     ap.add_argument("--voxel-image", action="store_true", help="also time emc2_voxel_image (fusion by voxel)")
     ap.add_argument("--pool", type=int, default=1, help="Multiscale Pooling size p (power of two): pool the maps, "
                                                         "then run the bridge on the pooled maps")

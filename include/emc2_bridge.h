@@ -164,6 +164,13 @@ int emc2_bridge_run(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_
                     float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
                     float* d_points_out, float* d_feat_out, void* cuda_stream);
 
+/* Layout change for callers whose image branch (a ResNet in Sec. 3.1) emits planar maps: copies
+ * d_planar float [B, K, Cf, Hf, Wf] into d_feat float [B, K, Hf, Wf, Cf], the channels-last layout
+ * the gather reads (one tap = one contiguous row).  The handle's K, Hf, Wf, Cf apply; the two
+ * buffers must not overlap. */
+int emc2_features_channels_last(emc2_bridge_t* bridge, int32_t B, const float* d_planar, float* d_feat,
+                                void* cuda_stream);
+
 /* Multiscale Pooling of the image features (Sec. 3.5: image features are pooled, with a pooling size
  * the user chooses, before they are fused with LiDAR features, to relieve memory).
  *   d_feat    float [B, K, Hf, Wf, Cf]                    the handle's feature-map shape

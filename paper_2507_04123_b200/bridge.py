@@ -34,6 +34,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
     "emc2_bridge_run", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
+    "emc2_features_channels_last",
     "emc2_voxel_image", "emc2_occlusion",
 )
 
@@ -85,6 +86,7 @@ def load_library() -> ctypes.CDLL:
     lib.emc2_occlusion.argtypes = [vp, i32, i32, vp, vp, vp, i32, ctypes.c_float, vp, vp, vp, vp]
     lib.emc2_voxel_image.argtypes = [vp, i32, i32, i32] + [vp] * 8
     lib.emc2_pool_features.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.emc2_features_channels_last.argtypes = [vp, i32, vp, vp, vp]
     lib.emc2_scene_route.argtypes = [vp, i32, vp, P(ctypes.c_uint8), i32, vp, vp]
     lib.emc2_bridge_set_overlap.argtypes = [vp, ctypes.c_int]
     lib.emc2_bridge_destroy.argtypes = [vp]
@@ -330,6 +332,19 @@ class Bridge:
                                      int(cell), float(margin), out["zbuf"].data_ptr(), out["occ_mask"].data_ptr(),
                                      out["clear_mask"].data_ptr(), self._stream())
         self._raise(rc, "emc2_occlusion")
+        return out
+
+    def features_channels_last(self, planar: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """emc2_features_channels_last: [B,K,Cf,Hf,Wf] maps copied into the [B,K,Hf,Wf,Cf] layout."""
+        c = self.cfg
+        B = planar.shape[0]
+        _check(planar, torch.float32, (B, c.num_cameras, c.feat_c, c.feat_h, c.feat_w), "planar", self.device)
+        shape = (B, c.num_cameras, c.feat_h, c.feat_w, c.feat_c)
+        if out is None:
+            out = torch.empty(shape, dtype=torch.float32, device=self.device)
+        _check(out, torch.float32, shape, "feat", self.device)
+        rc = self.lib.emc2_features_channels_last(self._h, B, planar.data_ptr(), out.data_ptr(), self._stream())
+        self._raise(rc, "emc2_features_channels_last")
         return out
 
     def pool_features(self, feat: torch.Tensor, p: int, out: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -10,7 +10,8 @@ namespace emc2 {
 static const char* const kKernelNames[K_KINDS] = {
     "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
     "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features",
-    "vif_scan", "vif_fill", "vif_mean", "occl_fill", "occl_splat", "occl_test"};
+    "vif_scan", "vif_fill", "vif_mean", "occl_fill", "occl_splat", "occl_test",
+    "channels_last"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
     if (e == cudaSuccess) return EMC2_OK;
@@ -367,6 +368,17 @@ int emc2_occlusion(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points
     if (!guard.ok) return EMC2_ERR_CUDA;
     return launch_occlusion(h, B, N, d_points, d_proj, d_vis_mask, cell, margin, reinterpret_cast<uint32_t*>(d_zbuf),
                             d_occ_mask, d_clear_mask, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int emc2_features_channels_last(emc2_bridge_t* h, int32_t B, const float* d_planar, float* d_feat,
+                                void* cuda_stream) {
+    if (!h || B < 0 || B > h->cfg.max_batch) return EMC2_ERR_INVALID_ARG;
+    if (B == 0) return EMC2_OK;
+    if (!d_planar || !d_feat || !aligned16(d_planar) || !aligned16(d_feat) || d_planar == d_feat)
+        return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_channels_last(h, B, d_planar, d_feat, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int emc2_pool_features(emc2_bridge_t* h, int32_t B, int32_t p, const float* d_feat, float* d_pooled,

@@ -38,6 +38,7 @@ enum KernelKind {
     K_OCCL_FILL,
     K_OCCL_SPLAT,
     K_OCCL_TEST,
+    K_CHANNELS_LAST,
     K_KINDS
 };
 
@@ -179,6 +180,7 @@ int voxel_image_scan_max_blocks();
 int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t* d_point_voxel,
                        const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
                        const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st);
+int launch_channels_last(emc2_bridge* h, int B, const float* d_planar, float* d_feat, cudaStream_t st);
 int launch_pool_features(emc2_bridge* h, int B, int p, const float* d_feat, float* d_pooled, cudaStream_t st);
 int launch_scene_route(emc2_bridge* h, int B, const int32_t* d_offsets, const uint8_t* priority, int min_points,
                        int32_t* d_scene_expert, cudaStream_t st);

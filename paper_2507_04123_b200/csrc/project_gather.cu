@@ -348,6 +348,43 @@ void launch_gs(emc2_bridge* h, const GsArgs& a, dim3 grid, cudaStream_t st) {
     }
 }
 
+// ------------------------------------------------------------------ planar -> channels-last
+// Per map the planar data is a Cf x P matrix (P = Hf * Wf pixels) and the channels-last data its
+// transpose.  A CTA moves a tile of 64 channels x 128 pixels through shared memory:
+//   in   one warp per channel row, 32 consecutive pixels (128 B) per instruction;
+//   out  a warp instruction covers 4 pixels x 32 channels: eight lanes store 128 contiguous bytes
+//        of one pixel's row.  With a row stride of 129 words the column reads from the tile
+//        (bank = channel + pixel mod 32) are conflict-free.
+constexpr int kClChan = 64, kClPix = 128, kClStride = kClPix + 1;
+
+__global__ void __launch_bounds__(256)
+channels_last_kernel(const float* __restrict__ planar, float* __restrict__ last, int Cf, int P, int ptiles) {
+    __shared__ float tile[kClChan][kClStride];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const size_t m = blockIdx.x / ptiles;
+    const int p0 = (int)(blockIdx.x - m * ptiles) * kClPix;
+    const int c0 = blockIdx.y * kClChan;
+    const int nc = min(kClChan, Cf - c0);
+    const float* src = planar + (m * Cf + c0) * (size_t)P + p0;
+    for (int c = warp; c < nc; c += 8) {
+#pragma unroll
+        for (int j = 0; j < kClPix / 32; ++j) {
+            const int q = lane + 32 * j;
+            tile[c][q] = p0 + q < P ? __ldcs(src + (size_t)c * P + q) : 0.f;
+        }
+    }
+    __syncthreads();
+    float* dst = last + (m * P + p0) * (size_t)Cf + c0;
+    const int halves = (nc + 31) / 32;                      // 32-channel halves of the tile
+    const int c = 4 * (lane & 7), dq = lane >> 3;
+    for (int job = warp; job < halves * (kClPix / 4); job += 8) {
+        const int cc = c + 32 * (job % halves), q = 4 * (job / halves) + dq;
+        if (cc >= nc || p0 + q >= P) continue;              // Cf % 4 == 0: a whole float4 or none
+        const float4 v = make_float4(tile[cc][q], tile[cc + 1][q], tile[cc + 2][q], tile[cc + 3][q]);
+        __stcs(reinterpret_cast<float4*>(dst + (size_t)q * Cf + cc), v);
+    }
+}
+
 // ------------------------------------------------------------------ Multiscale Pooling (Sec. 3.5)
 // One thread per (pooled texel, float4 column); grid = (columns of a pooled row, pooled rows,
 // maps).  Consecutive threads read consecutive columns of the same input rows, so every load
@@ -436,6 +473,19 @@ int launch_project_route_gather_dispatch(emc2_bridge* h, int B, int N, const flo
         ga.offset = c.feat_offset;
         if (c.point_floats == 4) launch_gs<4>(h, ga, grid, st); else launch_gs<5>(h, ga, grid, st);
     }
+    return check_cuda(h, cudaGetLastError());
+}
+
+int launch_channels_last(emc2_bridge* h, int B, const float* d_planar, float* d_feat, cudaStream_t st) {
+    const emc2_config_t& c = h->cfg;
+    const long long P = (long long)c.feat_h * c.feat_w;
+    const long long ptiles = (P + kClPix - 1) / kClPix;
+    const long long ctas = (long long)B * c.num_cameras * ptiles;
+    const int ct = (c.feat_c + kClChan - 1) / kClChan;
+    if (P > 0x7FFFFFFFLL || ctas > 0x7FFFFFFFLL || ct > 65535) return EMC2_ERR_INVALID_ARG;
+    LaunchScope ls(h, K_CHANNELS_LAST, st);
+    const dim3 grid((unsigned)ctas, ct);
+    channels_last_kernel<<<grid, 256, 0, st>>>(d_planar, d_feat, c.feat_c, (int)P, (int)ptiles);
     return check_cuda(h, cudaGetLastError());
 }
 

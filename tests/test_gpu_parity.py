@@ -85,6 +85,22 @@ def test_one_call_on_a_side_stream_of_the_caller(b200, oracle):
     br.close()
 
 
+def test_planar_maps_to_channels_last(b200, oracle):
+    rng = np.random.default_rng(21)
+    from dataclasses import replace
+    # pixel counts with and without 16-byte aligned channel rows; channel counts that fill a
+    # 64-channel tile, leave a 16- and a 4-channel remainder, or are one half group
+    for base in (gen.KITTI.with_shape(2, 100), gen.NUSCENES.with_shape(1, 100), gen.TINY,
+                 replace(gen.NUSCENES.with_shape(1, 100), feat_c=68), replace(gen.TINY, feat_c=12),
+                 replace(gen.TINY, feat_c=4, img_w=1250)):
+        br = b200.Bridge(b200.config_from_workload(base))
+        planar = rng.standard_normal((base.B, base.K, base.feat_c, base.feat_h, base.feat_w)).astype(np.float32)
+        got = br.features_channels_last(torch.from_numpy(planar).cuda())
+        br.status()
+        assert np.array_equal(np_(got), oracle.channels_last(planar))
+        br.close()
+
+
 @pytest.mark.parametrize("p", [1, 2, 4])
 def test_multiscale_pooling_and_the_pooled_path(b200, oracle, p):
     from dataclasses import replace
