@@ -37,6 +37,7 @@ def lib() -> ctypes.CDLL:
     if _lib is None:
         _lib = ctypes.CDLL(build())
         _lib.emc2o_voxelize.restype = ctypes.c_int
+        _lib.emc2o_rulebook.restype = ctypes.c_longlong
     return _lib
 
 
@@ -185,6 +186,17 @@ def scene_route(offsets: np.ndarray, priority: Sequence[int], min_points: int = 
     out = np.empty(B, np.int32)
     lib().emc2o_scene_route(B, E1 - 1, _p(offsets, _I), _p(pr, _U8), int(min_points), _p(out, _I))
     return out
+
+
+def rulebook(coords: np.ndarray):
+    """3 x 3 x 3 submanifold rulebook of a voxel list [M, 4] (b, z, y, x): offsets [28], in, out."""
+    coords = np.ascontiguousarray(coords, np.int32)
+    M = coords.shape[0]
+    offsets = np.empty(28, np.int32)
+    rin = np.empty(27 * max(M, 1), np.int32)
+    rout = np.empty(27 * max(M, 1), np.int32)
+    n = lib().emc2o_rulebook(M, _p(coords, _I), _p(offsets, _I), _p(rin, _I), _p(rout, _I))
+    return offsets, rin[:n].copy(), rout[:n].copy()
 
 
 def bridge(w, batch: Dict[str, np.ndarray]) -> Dict[str, object]:

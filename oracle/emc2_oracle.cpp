@@ -16,9 +16,11 @@
 // Conventions: points are row-major float32 [B, N, C] with (x, y, z) first;
 // all indices are 32-bit; a "frame" is one b in [0, B).
 #include <algorithm>
+#include <array>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <map>
 #include <vector>
 
 namespace {
@@ -354,4 +356,36 @@ extern "C" void emc2o_channels_last(int maps, int Cf, int Hf, int Wf, const floa
             for (int j = 0; j < Hf; ++j)
                 for (int i = 0; i < Wf; ++i)
                     last[(((size_t)m * Hf + j) * Wf + i) * Cf + c] = planar[(((size_t)m * Cf + c) * Hf + j) * Wf + i];
+}
+
+// Rulebook of a 3 x 3 x 3 submanifold sparse convolution over a voxel list (the index structure
+// of the 3D sparse convolution of Sec. 3.5, which runs on the non-empty voxels only; Sec. 3.6
+// replaces its index search by prefix sums).  The paper gives neither the kernel size nor the
+// layout: this is the usual one.  Kernel offset k = (dz+1)*9 + (dy+1)*3 + (dx+1) with dz, dy, dx
+// in {-1, 0, 1}.  For every k, in ascending order of the output voxel m: if a voxel n of the same
+// frame sits at coords[m] + (dz, dy, dx), the pair (in = n, out = m) is appended.
+// coords [M, 4] rows (b, z, y, x), all different -> offsets [28] (pairs before offset k; [27] =
+// all pairs), rule_in / rule_out [<= 27 * M].  Returns the number of pairs.
+extern "C" long long emc2o_rulebook(int M, const int32_t* coords, int32_t* offsets, int32_t* rule_in,
+                                    int32_t* rule_out) {
+    std::map<std::array<int32_t, 4>, int32_t> where;
+    for (int m = 0; m < M; ++m)
+        where[{coords[4 * m], coords[4 * m + 1], coords[4 * m + 2], coords[4 * m + 3]}] = m;
+    long long pairs = 0;
+    int k = 0;
+    for (int dz = -1; dz <= 1; ++dz)
+        for (int dy = -1; dy <= 1; ++dy)
+            for (int dx = -1; dx <= 1; ++dx, ++k) {
+                offsets[k] = (int32_t)pairs;
+                for (int m = 0; m < M; ++m) {
+                    const int32_t* c = coords + 4 * m;
+                    auto it = where.find({c[0], c[1] + dz, c[2] + dy, c[3] + dx});
+                    if (it == where.end()) continue;
+                    rule_in[pairs] = it->second;
+                    rule_out[pairs] = m;
+                    pairs += 1;
+                }
+            }
+    offsets[27] = (int32_t)pairs;
+    return pairs;
 }

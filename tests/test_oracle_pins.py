@@ -587,3 +587,75 @@ def test_channels_last_is_numpys_transpose(oracle):
     rng = np.random.default_rng(14)
     x = rng.standard_normal((2, 3, 7, 5, 11)).astype(F32)
     assert np.array_equal(oracle.channels_last(x), np.ascontiguousarray(x.transpose(0, 1, 3, 4, 2)))
+
+
+# ---------------------------------------------------------------- sparse-convolution rulebook
+def _offset(k):
+    return k // 9 - 1, (k // 3) % 3 - 1, k % 3 - 1            # dz, dy, dx
+
+
+def test_rulebook_of_a_hand_built_list(oracle):
+    # three voxels of frame 0: a=(z0,y0,x0), b=(z0,y0,x1), c=(z0,y1,x1); one of frame 1 at a's place
+    coords = np.array([[0, 0, 0, 0], [0, 0, 0, 1], [0, 0, 1, 1], [1, 0, 0, 0]], np.int32)
+    off, rin, rout = oracle.rulebook(coords)
+    got = {k: list(zip(rin[off[k]:off[k + 1]].tolist(), rout[off[k]:off[k + 1]].tolist())) for k in range(27)}
+    want = {k: [] for k in range(27)}
+    want[13] = [(0, 0), (1, 1), (2, 2), (3, 3)]               # centre: every voxel with itself
+    want[14] = [(1, 0)]                                       # dx=+1: b is the +x neighbour of a
+    want[12] = [(0, 1)]                                       # dx=-1
+    want[16] = [(2, 1)]                                       # dy=+1: c above b
+    want[10] = [(1, 2)]                                       # dy=-1
+    want[17] = [(2, 0)]                                       # dy=+1, dx=+1: c diagonal of a
+    want[9] = [(0, 2)]                                        # dy=-1, dx=-1
+    assert got == want
+    assert off[0] == 0 and off[27] == 10
+
+
+def test_rulebook_against_brute_force(oracle):
+    rng = np.random.default_rng(31)
+    for trial in range(4):
+        cells = rng.integers(0, 5, size=(300, 4)).astype(np.int32)
+        cells[:, 0] = rng.integers(0, 2, size=300)
+        coords = np.unique(cells, axis=0)                     # also sorted, as the voxelizer writes them
+        if trial == 3:
+            coords = coords[rng.permutation(len(coords))]     # the definition does not need sorted rows
+        off, rin, rout = oracle.rulebook(coords)
+        pos = 0
+        for k in range(27):
+            dz, dy, dx = _offset(k)
+            assert off[k] == pos
+            for m in range(len(coords)):
+                target = coords[m] + np.array([0, dz, dy, dx], np.int32)
+                hits = np.nonzero((coords == target).all(axis=1))[0]
+                assert len(hits) <= 1
+                if len(hits):
+                    assert (rin[pos], rout[pos]) == (hits[0], m)
+                    pos += 1
+        assert off[27] == pos == len(rin) == len(rout)
+
+
+def test_rulebook_counts_of_a_full_block_and_symmetry(oracle):
+    a, b, c = 4, 3, 5                                         # z, y, x extent of a full block
+    zz, yy, xx = np.meshgrid(np.arange(a), np.arange(b), np.arange(c), indexing="ij")
+    coords = np.stack([np.zeros(a * b * c, np.int64), zz.ravel(), yy.ravel(), xx.ravel()], 1).astype(np.int32)
+    off, rin, rout = oracle.rulebook(coords)
+    for k in range(27):
+        dz, dy, dx = _offset(k)
+        assert off[k + 1] - off[k] == (a - abs(dz)) * (b - abs(dy)) * (c - abs(dx))
+        # the pairs of the opposite offset are these pairs swapped
+        here = set(zip(rin[off[k]:off[k + 1]].tolist(), rout[off[k]:off[k + 1]].tolist()))
+        there = set(zip(rout[off[26 - k]:off[27 - k]].tolist(), rin[off[26 - k]:off[27 - k]].tolist()))
+        assert here == there
+        assert np.all(np.diff(rout[off[k]:off[k + 1]]) > 0)   # ascending output voxel
+
+
+def test_rulebook_neighbours_are_scipys_chebyshev_pairs(oracle):
+    from scipy.spatial import cKDTree
+    rng = np.random.default_rng(32)
+    pts = np.unique(rng.integers(0, 12, size=(800, 3)), axis=0)
+    coords = np.concatenate([np.zeros((len(pts), 1), np.int64), pts], 1).astype(np.int32)
+    off, rin, rout = oracle.rulebook(coords)
+    mine = {(min(i, o), max(i, o)) for i, o in zip(rin.tolist(), rout.tolist()) if i != o}
+    theirs = {tuple(sorted(p)) for p in cKDTree(pts.astype(np.float64)).query_pairs(1.0, p=np.inf)}
+    assert mine == theirs
+    assert off[27] == 2 * len(theirs) + len(pts)
