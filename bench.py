@@ -414,6 +414,31 @@ def run_ours(args, w):
             vi[f"scale{sc}"] = {"ms_per_call": ms_vi, "voxels": M, "visible_points": nvis,
                                 "algorithmic_bytes": vbytes, "achieved_gbs": vbytes / (ms_vi * 1e-3) / 1e9}
         line["voxel_image"] = vi
+    if args.rulebook:
+        # Sparse-convolution rulebook of each scale's voxel list (five kernels, timed together).
+        rb = {}
+        for sc in (0, 1):
+            M = int(nv[sc])
+            out = br.rulebook(bufs["vox"], sc)
+            fn = lambda: br.rulebook(bufs["vox"], sc, out=out)
+            for _ in range(3):
+                fn()
+            secs_rb = time_steps(fn, args.steps, sync, barrier)
+            br.status()
+            br.profile_read(reset=True)
+            br.profile_enable(True)
+            for _ in range(5):
+                fn()
+            sync()
+            kern = {k: ms / n for k, (n, ms) in br.profile_read(reset=True).items() if n and k.startswith("rb_")}
+            br.profile_enable(False)
+            pairs = int(out["offsets"][27].item())
+            rbytes = 16 * M + 8 * pairs + 112            # the list read once, every pair written once
+            ms_rb = secs_rb / args.steps * 1e3
+            rb[f"scale{sc}"] = {"ms_per_call": ms_rb, "voxels": M, "pairs": pairs, "algorithmic_bytes": rbytes,
+                                "achieved_gbs": rbytes / (ms_rb * 1e-3) / 1e9,
+                                "pairs_per_s": pairs / (ms_rb * 1e-3), "kernel_ms": kern}
+        line["rulebook"] = rb
     if args.channels_last:
         # Planar maps -> channels-last, its own kernel timed alone (a pure copy: bytes = 2 x the maps).
         planar = d["feat"].permute(0, 1, 4, 2, 3).contiguous()
@@ -481,6 +506,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--occlusion", action="store_true", help="also time emc2_occlusion (depth-buffer test)")
+    ap.add_argument("--rulebook", action="store_true", help="also time emc2_rulebook (sparse-convolution rulebook)")
     ap.add_argument("--channels-last", action="store_true", help="also time emc2_features_channels_last")
     ap.add_argument("--voxel-image", action="store_true", help="also time emc2_voxel_image (fusion by voxel)")
     ap.add_argument("--pool", type=int, default=1, help="Multiscale Pooling size p (power of two): pool the maps, "

@@ -44,7 +44,8 @@ extern "C" {
 
 typedef enum {
     EMC2_OK = 0,
-    EMC2_ERR_INVALID_ARG = -1, /* null/misaligned pointer, B or N outside the configured maxima */
+    EMC2_ERR_INVALID_ARG = -1, /* null/misaligned pointer, B or N outside the configured maxima; from
+                                  emc2_bridge_status: a voxel list that is not one of its grid */
     EMC2_ERR_BAD_CONFIG = -2,  /* emc2_config_t rejected by emc2_bridge_create */
     EMC2_ERR_CUDA = -3,        /* a CUDA runtime call failed; see emc2_bridge_last_cuda_error */
     EMC2_ERR_CAPACITY = -4,    /* more unique voxels than capacity[s] (device-detected, sticky) */
@@ -182,6 +183,25 @@ int emc2_features_channels_last(emc2_bridge_t* bridge, int32_t B, const float* d
  * feat_offset = (p - 1) / 2 * s, so that each pooled texel sits at the centre of its window. */
 int emc2_pool_features(emc2_bridge_t* bridge, int32_t B, int32_t p, const float* d_feat, float* d_pooled,
                        void* cuda_stream);
+
+/* Rulebook of a 3 x 3 x 3 submanifold sparse convolution over one scale's voxel list: the index
+ * structure of the 3D sparse convolution that consumes the list (Sec. 3.5), built with prefix sums
+ * instead of an index search (Sec. 3.6).  The paper states neither kernel size nor layout; this is
+ * the usual one.  Kernel offset k = (dz+1)*9 + (dy+1)*3 + (dx+1), dz, dy, dx in {-1, 0, 1}.
+ *   d_rule_offsets  int32 [28]             pairs before offset k; [27] = all pairs (true count even
+ *                                          when it exceeds pair_capacity)
+ *   d_rule_in/out   int32 [pair_capacity]  for every k, in ascending out: the pairs (in = n, out = m)
+ *                                          with coords[n] = coords[m] + (0, dz, dy, dx), same frame
+ * d_coords int32 [capacity, 4] and d_num_voxels (DEVICE int32, the scale's entry) are emc2_voxelize's
+ * outputs for grid[scale]: rows (b, z, y, x) inside the grid, all different, in ascending order;
+ * min(*d_num_voxels, capacity) rows are used, capacity <= max_batch * max_points.  A list that
+ * breaks these rules makes EMC2_ERR_INVALID_ARG sticky (device-detected; the outputs are then
+ * undefined but in bounds).  27 * capacity pairs always suffice; with fewer, pairs past
+ * pair_capacity are not written and EMC2_ERR_CAPACITY becomes sticky.  Enqueues five kernels; uses
+ * the scale's handle scratch, so calls on one handle must be ordered. */
+int emc2_rulebook(emc2_bridge_t* bridge, int32_t scale, int32_t capacity, const int32_t* d_coords,
+                  const int32_t* d_num_voxels, int32_t* d_rule_offsets, int32_t* d_rule_in, int32_t* d_rule_out,
+                  int64_t pair_capacity, void* cuda_stream);
 
 /* Fusion by voxel (Fig. 5: image features of the pixels that share a voxel's 3-D coordinate go with
  * that voxel; voxels without such pixels get zero-filled features).  The pixels with a 3-D coordinate

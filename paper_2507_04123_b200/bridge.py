@@ -35,7 +35,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
     "emc2_bridge_run", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
     "emc2_features_channels_last",
-    "emc2_voxel_image", "emc2_occlusion",
+    "emc2_voxel_image", "emc2_occlusion", "emc2_rulebook",
 )
 
 
@@ -85,6 +85,7 @@ def load_library() -> ctypes.CDLL:
     lib.emc2_bridge_status.argtypes = [vp, vp]
     lib.emc2_occlusion.argtypes = [vp, i32, i32, vp, vp, vp, i32, ctypes.c_float, vp, vp, vp, vp]
     lib.emc2_voxel_image.argtypes = [vp, i32, i32, i32] + [vp] * 8
+    lib.emc2_rulebook.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, ctypes.c_int64, vp]
     lib.emc2_pool_features.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.emc2_features_channels_last.argtypes = [vp, i32, vp, vp, vp]
     lib.emc2_scene_route.argtypes = [vp, i32, vp, P(ctypes.c_uint8), i32, vp, vp]
@@ -313,6 +314,27 @@ class Bridge:
                                        nv.data_ptr() + 4 * scale, vis_mask.data_ptr(), gathered.data_ptr(),
                                        out["vox_img"].data_ptr(), out["vox_img_count"].data_ptr(), self._stream())
         self._raise(rc, "emc2_voxel_image")
+        return out
+
+    def rulebook(self, vox: Dict[str, object], scale: int, pair_capacity: Optional[int] = None,
+                 out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        """emc2_rulebook for one scale of a :meth:`voxelize` result: offsets [28], rule_in, rule_out."""
+        coords = vox["coords"][scale]
+        cap = int(coords.shape[0])
+        _check(coords, torch.int32, (cap, 4), "coords", self.device)
+        if out is None:
+            pairs = 27 * cap if pair_capacity is None else int(pair_capacity)
+            out = {"offsets": torch.empty((28,), dtype=torch.int32, device=self.device),
+                   "rule_in": torch.empty((pairs,), dtype=torch.int32, device=self.device),
+                   "rule_out": torch.empty((pairs,), dtype=torch.int32, device=self.device)}
+        pairs = int(out["rule_in"].shape[0])
+        _check(out["offsets"], torch.int32, (28,), "offsets", self.device)
+        _check(out["rule_out"], torch.int32, (pairs,), "rule_out", self.device)
+        nv = vox["num_voxels"]
+        rc = self.lib.emc2_rulebook(self._h, int(scale), cap, coords.data_ptr(), nv.data_ptr() + 4 * scale,
+                                    out["offsets"].data_ptr(), out["rule_in"].data_ptr(),
+                                    out["rule_out"].data_ptr(), pairs, self._stream())
+        self._raise(rc, "emc2_rulebook")
         return out
 
     def occlusion(self, points: torch.Tensor, proj: torch.Tensor, vis_mask: torch.Tensor, cell: int,

@@ -11,7 +11,7 @@ static const char* const kKernelNames[K_KINDS] = {
     "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
     "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features",
     "vif_scan", "vif_fill", "vif_mean", "occl_fill", "occl_splat", "occl_test",
-    "channels_last"};
+    "channels_last", "rb_mark", "rb_count", "rb_scan", "rb_fill", "rb_clear"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
     if (e == cudaSuccess) return EMC2_OK;
@@ -175,6 +175,10 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     const size_t o_vif_cursor = plan.take(maxpts * sizeof(int));
     const size_t o_vif_list = plan.take(maxpts * sizeof(int));
     const size_t o_vif_part = plan.take((size_t)h->vif_scan_blocks * sizeof(int));
+    const size_t rb_tiles = (maxpts + kTile - 1) / kTile;
+    const size_t o_rb_bits = plan.take(maxpts * sizeof(uint32_t));
+    const size_t o_rb_counts = plan.take(27 * rb_tiles * sizeof(int));
+    const size_t o_rb_base = plan.take((27 * rb_tiles + 27) * sizeof(int));
     const size_t o_wofs = plan.take((size_t)h->scan_blocks * (kThreads / 32) * 3 * sizeof(int));
     h->max_tiles = (c.max_points + kTile - 1) / kTile;
     const size_t tile_ints = (size_t)c.max_batch * h->max_tiles * c.num_experts;
@@ -207,6 +211,9 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     h->d_vif_cursor = reinterpret_cast<int*>(base + o_vif_cursor);
     h->d_vif_list = reinterpret_cast<int*>(base + o_vif_list);
     h->d_vif_part = reinterpret_cast<int*>(base + o_vif_part);
+    h->d_rb_bits = reinterpret_cast<uint32_t*>(base + o_rb_bits);
+    h->d_rb_counts = reinterpret_cast<int*>(base + o_rb_counts);
+    h->d_rb_base = reinterpret_cast<int*>(base + o_rb_base);
     h->d_scan_warp_ofs = reinterpret_cast<int*>(base + o_wofs);
     h->d_tile_counts = reinterpret_cast<int*>(base + o_tc);
     h->d_tile_base = reinterpret_cast<int*>(base + o_tb);
@@ -355,6 +362,22 @@ int emc2_voxel_image(emc2_bridge_t* h, int32_t B, int32_t N, int32_t capacity, c
                               d_vox_img, d_vox_img_count, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int emc2_rulebook(emc2_bridge_t* h, int32_t scale, int32_t capacity, const int32_t* d_coords,
+                  const int32_t* d_num_voxels, int32_t* d_rule_offsets, int32_t* d_rule_in, int32_t* d_rule_out,
+                  int64_t pair_capacity, void* cuda_stream) {
+    if (!h || scale < 0 || scale > 1 || capacity < 0 || pair_capacity < 0) return EMC2_ERR_INVALID_ARG;
+    if ((int64_t)capacity > (int64_t)h->cfg.max_batch * h->cfg.max_points) return EMC2_ERR_INVALID_ARG;
+    if (!d_num_voxels || !d_rule_offsets) return EMC2_ERR_INVALID_ARG;
+    if (capacity > 0 && (!d_coords || !aligned16(d_coords))) return EMC2_ERR_INVALID_ARG;
+    if (pair_capacity > 0 && (!d_rule_in || !d_rule_out)) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (capacity == 0) return check_cuda(h, cudaMemsetAsync(d_rule_offsets, 0, 28 * sizeof(int32_t), st));
+    return launch_rulebook(h, scale, capacity, d_coords, d_num_voxels, d_rule_offsets, d_rule_in, d_rule_out,
+                           pair_capacity, st);
+}
+
 int emc2_occlusion(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points, const float* d_proj,
                    const uint8_t* d_vis_mask, int32_t cell, float margin, float* d_zbuf, uint8_t* d_occ_mask,
                    uint8_t* d_clear_mask, void* cuda_stream) {
@@ -421,6 +444,7 @@ int emc2_bridge_status(emc2_bridge_t* h, void* cuda_stream) {
     if (e != cudaSuccess) return check_cuda(h, e);
     if (word & 2) return EMC2_ERR_TIMEOUT;
     if (word & 1) return EMC2_ERR_CAPACITY;
+    if (word & 4) return EMC2_ERR_INVALID_ARG;
     return EMC2_OK;
 }
 

@@ -39,6 +39,11 @@ enum KernelKind {
     K_OCCL_SPLAT,
     K_OCCL_TEST,
     K_CHANNELS_LAST,
+    K_RB_MARK,
+    K_RB_COUNT,
+    K_RB_SCAN,
+    K_RB_FILL,
+    K_RB_CLEAR,
     K_KINDS
 };
 
@@ -126,6 +131,9 @@ struct emc2_bridge {
     int* d_vif_list = nullptr;
     int* d_vif_part = nullptr;     // [vif_scan_blocks]
     int vif_scan_blocks = 0;
+    uint32_t* d_rb_bits = nullptr;  // emc2_rulebook: [max points] neighbour bits per voxel
+    int* d_rb_counts = nullptr;    // [27][voxel tiles] pairs per (offset, tile), and their prefix sums
+    int* d_rb_base = nullptr;
     int max_tiles = 0;
     bool overlap = true;           // emc2_bridge_run puts stage 1 on `side`
     cudaStream_t side = nullptr;   // stream of stage 1 inside emc2_bridge_run
@@ -180,6 +188,9 @@ int voxel_image_scan_max_blocks();
 int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t* d_point_voxel,
                        const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
                        const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st);
+int launch_rulebook(emc2_bridge* h, int scale, int capacity, const int32_t* d_coords, const int32_t* d_num_voxels,
+                    int32_t* d_rule_offsets, int32_t* d_rule_in, int32_t* d_rule_out, long long pair_capacity,
+                    cudaStream_t st);
 int launch_channels_last(emc2_bridge* h, int B, const float* d_planar, float* d_feat, cudaStream_t st);
 int launch_pool_features(emc2_bridge* h, int B, int p, const float* d_feat, float* d_pooled, cudaStream_t st);
 int launch_scene_route(emc2_bridge* h, int B, const int32_t* d_offsets, const uint8_t* priority, int min_points,

@@ -149,6 +149,66 @@ def test_image_features_per_voxel(b200, oracle, cid, B, N):
     br.close()
 
 
+@pytest.mark.parametrize("cid,B,N", [(2, 2, 60_000), (1, 3, 33_333), (3, 1, 150_000), (0, 1, 16_384), (2, 1, 1)])
+def test_sparse_convolution_rulebook(b200, oracle, cid, B, N):
+    w = gen.workload(cid).with_shape(B, N)
+    batch = gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    for s in range(2):                             # the two scales use the two kinds of cell store
+        M = ref[f"vox{s}"]["num_voxels"]
+        off, rin, rout = oracle.rulebook(ref[f"vox{s}"]["coords"][:M])
+        for rep in range(2):                       # twice: the store must be clean again after a call
+            out = br.rulebook(bufs["vox"], s)
+            br.status()
+            assert np.array_equal(np_(out["offsets"]), off), s
+            assert np.array_equal(np_(out["rule_in"])[:off[27]], rin), s
+            assert np.array_equal(np_(out["rule_out"])[:off[27]], rout), s
+    # and the voxelizer still finds its store all zero
+    bufs = br.run(d["points"], d["proj"], d["feat"], bufs)
+    br.status()
+    compare_bridge(w, ref, bufs)
+    br.close()
+
+
+def test_rulebook_errors_only_the_device_sees(b200, oracle):
+    w = gen.KITTI.with_shape(1, 20_000)
+    batch = gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    br.status()
+    M = ref["vox0"]["num_voxels"]
+    off, rin, rout = oracle.rulebook(ref["vox0"]["coords"][:M])
+    total = int(off[27])
+    # too few pair slots: the true count is reported, nothing is written past the end
+    small = total // 2
+    guard = 64
+    out = {"offsets": torch.empty(28, dtype=torch.int32, device="cuda"),
+           "rule_in": torch.full((small + guard,), -7, dtype=torch.int32, device="cuda"),
+           "rule_out": torch.full((small + guard,), -7, dtype=torch.int32, device="cuda")}
+    view = {"offsets": out["offsets"], "rule_in": out["rule_in"][:small], "rule_out": out["rule_out"][:small]}
+    br.rulebook(bufs["vox"], 0, out=view)
+    assert br.status(raise_on_error=False) == b200.bridge.EMC2_ERR_CAPACITY
+    assert np.array_equal(np_(out["offsets"]), off)
+    assert (np_(out["rule_in"])[small:] == -7).all() and (np_(out["rule_out"])[small:] == -7).all()
+    # every pair slot below the end that belongs to a written position holds the right pair
+    got_in, got_out = np_(out["rule_in"])[:small], np_(out["rule_out"])[:small]
+    assert np.array_equal(got_in, rin[:small]) and np.array_equal(got_out, rout[:small])
+    # a list that is not in ascending order is reported, and the store is clean afterwards
+    bad = {"coords": [bufs["vox"]["coords"][0].clone(), bufs["vox"]["coords"][1]], "num_voxels": bufs["vox"]["num_voxels"]}
+    bad["coords"][0][[5, 9]] = bad["coords"][0][[9, 5]]
+    br.rulebook(bad, 0)
+    assert br.status(raise_on_error=False) == b200.bridge.EMC2_ERR_INVALID_ARG
+    out = br.rulebook(bufs["vox"], 0)
+    br.status()
+    assert np.array_equal(np_(out["rule_in"])[:total], rin) and np.array_equal(np_(out["rule_out"])[:total], rout)
+    br.close()
+
+
 @pytest.mark.parametrize("cid,B,N,cell,margin", [(2, 2, 120_000, 8, 0.5), (1, 3, 40_001, 4, 0.25),
                                                  (3, 1, 300_000, 16, 1.0), (2, 1, 5000, 64, 0.0)])
 def test_occlusion_and_routing_of_occluded_points(b200, oracle, cid, B, N, cell, margin):
