@@ -134,6 +134,27 @@ __device__ __forceinline__ void neighbours3(const ScaleDev& g, const Site& s, in
     }
 }
 
+// Which of the three x-neighbours at (dz, dy) exist (bit dx + 1), for a valid site.
+__device__ __forceinline__ uint32_t exist3(const ScaleDev& g, const Site& s, int j) {
+    const int dz = j / 3 - 1, dy = j % 3 - 1;
+    if (!s.okz[dz + 1] || !s.oky[dy + 1]) return 0u;
+    const uint32_t mid = s.cell + (uint32_t)dz * s.sz + (uint32_t)dy * s.sy;
+    const uint32_t inside = (s.okx[0] ? 1u : 0u) | 2u | (s.okx[2] ? 4u : 0u);
+    if (g.mode == MODE_BITMAP) {
+        const uint32_t w = mid >> 5, pos = mid & 31u;
+        // 34-bit window: the word's 32 cells with one cell of the words before and after it
+        unsigned long long window = (unsigned long long)g.store[2 * (size_t)w] << 1;
+        if (pos == 0 && s.okx[0]) window |= g.store[2 * (size_t)(w - 1)] >> 31;
+        if (pos == 31 && s.okx[2]) window |= (unsigned long long)(g.store[2 * (size_t)(w + 1)] & 1u) << 33;
+        return (uint32_t)(window >> pos) & inside;
+    }
+    uint32_t three = 0;
+#pragma unroll
+    for (int i = 0; i < 3; ++i)
+        if (s.okx[i] && g.store[4 * (size_t)(mid + i - 1)]) three |= 1u << i;
+    return three;
+}
+
 __global__ void __launch_bounds__(kThreads) rb_count_kernel(const __grid_constant__ RbArgs a) {
     __shared__ int wcount[kThreads / 32][kOffsets];
     const int M = voxels_in_list(a);
@@ -145,12 +166,7 @@ __global__ void __launch_bounds__(kThreads) rb_count_kernel(const __grid_constan
         const Site s = site_of(a, c);
         if (s.cell != 0xFFFFFFFFu) {
 #pragma unroll
-            for (int j = 0; j < 9; ++j) {
-                int r[3];
-                neighbours3(a.g, s, j, 7u, r);
-#pragma unroll
-                for (int i = 0; i < 3; ++i) bits |= (r[i] >= 0 ? 1u : 0u) << (3 * j + i);
-            }
+            for (int j = 0; j < 9; ++j) bits |= exist3(a.g, s, j) << (3 * j);
         }
     }
     if (m < a.capacity) a.nbr_bits[m] = bits;
