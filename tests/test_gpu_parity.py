@@ -173,6 +173,41 @@ def test_sparse_convolution_rulebook(b200, oracle, cid, B, N):
     br.close()
 
 
+def test_rulebook_at_full_size(b200, oracle):
+    """The benchmark's batch: properties that hold at any size, and the first frame pair by pair."""
+    w = gen.NUSCENES
+    batch = gen.make_batch(w, feature_frames=1)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    vox = br.voxelize(d["points"])
+    out = br.rulebook(vox, 0)
+    br.status()
+    M = int(vox["num_voxels"][0].item())
+    coords = np_(vox["coords"][0])[:M].astype(np.int64)
+    off = np_(out["offsets"]).astype(np.int64)
+    total = int(off[27])
+    rin, rout = np_(out["rule_in"])[:total].astype(np.int64), np_(out["rule_out"])[:total].astype(np.int64)
+    assert off[0] == 0 and np.all(np.diff(off) >= 0)
+    assert rin.min() >= 0 and rin.max() < M and rout.min() >= 0 and rout.max() < M
+    for k in range(27):
+        i, o = rin[off[k]:off[k + 1]], rout[off[k]:off[k + 1]]
+        shift = np.array([0, k // 9 - 1, (k // 3) % 3 - 1, k % 3 - 1])
+        assert np.array_equal(coords[i], coords[o] + shift), k       # every listed pair is a true neighbour pair
+        assert np.all(np.diff(o) > 0), k                              # ascending, no pair twice
+        assert off[k + 1] - off[k] == off[27 - k] - off[26 - k], k    # as many as for the opposite offset
+    assert np.array_equal(rin[off[13]:off[14]], np.arange(M))
+    # frames never pair with one another, so the first frame's rows form the rulebook of its own list
+    M0 = int((coords[:, 0] == 0).sum())
+    want_off, want_in, want_out = oracle.rulebook(coords[:M0].astype(np.int32))
+    for k in range(27):
+        i, o = rin[off[k]:off[k + 1]], rout[off[k]:off[k + 1]]
+        n = int(np.searchsorted(o, M0))
+        assert n == want_off[k + 1] - want_off[k], k
+        assert np.array_equal(i[:n], want_in[want_off[k]:want_off[k + 1]]), k
+        assert np.array_equal(o[:n], want_out[want_off[k]:want_off[k + 1]]), k
+    br.close()
+
+
 def test_rulebook_errors_only_the_device_sees(b200, oracle):
     w = gen.KITTI.with_shape(1, 20_000)
     batch = gen.make_batch(w)
