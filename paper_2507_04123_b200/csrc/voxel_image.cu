@@ -98,23 +98,53 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_mean_kernel
     const int rows = (int)blockDim.x / cf4;                  // voxels a CTA handles at a time
     const int r = (int)threadIdx.x / cf4, c = (int)threadIdx.x - r * cf4;
     if (r >= rows) return;
-    for (int m = blockIdx.x * rows + r; m < M; m += gridDim.x * rows) {
-        const int s0 = a.start[m], n = a.counts[m];
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        int seen = 0;
-        for (int k = 0; k < n; ++k) {
-            const int i = a.list[s0 + k];
-            if (i < 0) continue;
-            const float4 v = __ldcs(a.gathered + (size_t)i * cf4 + c);
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-            seen += 1;
+    // Two voxels per thread and round: their loads (list start and length, first list entry, first
+    // row) do not depend on one another and are in flight together.
+    const int stride = gridDim.x * rows;
+    for (int m0 = blockIdx.x * rows + r; m0 < M; m0 += 2 * stride) {
+        int mm[2] = {m0, m0 + stride}, s0[2], n[2], first[2], seen[2] = {0, 0};
+        float4 acc[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const bool ok = mm[u] < M;
+            s0[u] = ok ? a.start[mm[u]] : 0;
+            n[u] = ok ? a.counts[mm[u]] : 0;
         }
-        if (seen > 1) {
-            const float inv = 1.0f / (float)seen;
-            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) first[u] = n[u] > 0 ? a.list[s0[u]] : -1;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (first[u] >= 0) {
+                acc[u] = __ldcs(a.gathered + (size_t)first[u] * cf4 + c);
+                seen[u] = 1;
+            }
         }
-        __stcs(a.vox_img + (size_t)m * cf4 + c, acc);
-        if (c == 0) a.vox_cnt[m] = seen;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            for (int k = 1; k < n[u]; k += 4) {            // four entries in flight; summed in list order
+                int idx[4];
+                float4 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) idx[j] = k + j < n[u] ? a.list[s0[u] + k + j] : -1;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (idx[j] >= 0) v[j] = __ldcs(a.gathered + (size_t)idx[j] * cf4 + c);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (idx[j] < 0) continue;
+                    acc[u].x += v[j].x; acc[u].y += v[j].y; acc[u].z += v[j].z; acc[u].w += v[j].w;
+                    seen[u] += 1;
+                }
+            }
+            if (mm[u] >= M) continue;
+            if (seen[u] > 1) {
+                const float inv = 1.0f / (float)seen[u];
+                acc[u].x *= inv; acc[u].y *= inv; acc[u].z *= inv; acc[u].w *= inv;
+            }
+            __stcs(a.vox_img + (size_t)mm[u] * cf4 + c, acc[u]);
+            if (c == 0) a.vox_cnt[mm[u]] = seen[u];
+        }
     }
 }
 
