@@ -287,6 +287,16 @@ def run_ours(args, w):
     for _ in range(3):
         staged_step()
     staged_secs = max_over_ranks(time_steps(staged_step, args.steps, sync, barrier))
+    graph_secs = None
+    if args.graph:
+        # The one-call step captured once into a CUDA graph and replayed (fewer launch gaps on small batches).
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        for _ in range(args.warmup):
+            graph.replay()
+        graph_secs = max_over_ranks(time_steps(graph.replay, args.steps, sync, barrier))
+        br.status()
     br.profile_read(reset=True)
 
     # End to end: pinned host inputs copied in every step, small results read back every step.
@@ -366,6 +376,7 @@ def run_ours(args, w):
                          else "working set fits in L2 (latency-bound workload, no flush)"},
         "mpoints_per_s": fps * N / 1e6,
         "staged_ms_per_step": staged_secs / args.steps * 1e3,
+        "graph_ms_per_step": graph_secs / args.steps * 1e3 if graph_secs is not None else None,
         "bridge_algorithmic_bytes_per_step": abytes,
         "one_call_bytes_per_step": one_call_bytes(w, B, N, int(nv[0]), int(nv[1]), texels),
         "bridge_gbs": total_gbs, "bridge_frac_of_8tbs": total_gbs / NOMINAL_HBM_GBS,
@@ -506,6 +517,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--occlusion", action="store_true", help="also time emc2_occlusion (depth-buffer test)")
+    ap.add_argument("--graph", action="store_true", help="also time the one-call step replayed from a CUDA graph")
     ap.add_argument("--rulebook", action="store_true", help="also time emc2_rulebook (sparse-convolution rulebook)")
     ap.add_argument("--channels-last", action="store_true", help="also time emc2_features_channels_last")
     ap.add_argument("--voxel-image", action="store_true", help="also time emc2_voxel_image (fusion by voxel)")

@@ -85,6 +85,31 @@ def test_one_call_on_a_side_stream_of_the_caller(b200, oracle):
     br.close()
 
 
+def test_one_call_replays_from_a_cuda_graph(b200, oracle):
+    # emc2_bridge_run only enqueues (kernels, a fork and a join by events), so a caller can capture
+    # it once and replay it on new frames written into the same buffers.
+    w = gen.KITTI.with_shape(2, 30000)
+    first, second = gen.make_batch(w, frames=[0, 1]), gen.make_batch(w, frames=[2, 3])
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(first)
+    bufs = br.run(d["points"], d["proj"], d["feat"])      # allocates the outputs, outside the capture
+    br.status()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        br.run(d["points"], d["proj"], d["feat"], bufs)
+    for batch in (second, first):
+        for k, v in batch.items():
+            d[k].copy_(torch.from_numpy(v))
+        bufs["pg"]["gathered"].fill_(-1.0)
+        bufs["vox"]["num_voxels"].fill_(-1)
+        graph.replay()
+        torch.cuda.synchronize()
+        br.status()
+        compare_bridge(w, oracle.bridge(w, batch), bufs)
+    del graph
+    br.close()
+
+
 def test_planar_maps_to_channels_last(b200, oracle):
     rng = np.random.default_rng(21)
     from dataclasses import replace
