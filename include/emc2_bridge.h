@@ -22,7 +22,9 @@
  *     NULL = legacy default stream) only enqueues kernels.  These calls do not
  *     allocate, do not synchronise and do not touch the host except to return.
  *     Some kernels are cooperative launches (grid-wide barrier), which the
- *     device must support; emc2_bridge_create() fails otherwise.
+ *     device must support; emc2_bridge_create() fails otherwise.  The calls
+ *     that take a handle and a stream can therefore be captured into a CUDA
+ *     graph and replayed (emc2_bridge_status synchronises and cannot).
  *   - One handle serves one device and one stream at a time; it is not
  *     thread-safe.  Calls on the same handle must be ordered on the stream.
  *   - Errors are returned as negative emc2_status_t values.  Errors the host
