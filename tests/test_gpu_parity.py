@@ -107,6 +107,36 @@ def test_one_call_replays_from_a_cuda_graph(b200, oracle):
         br.status()
         compare_bridge(w, oracle.bridge(w, batch), bufs)
     del graph
+    # the stage calls and the optional calls, one after another in a second graph
+    vi = br.voxel_image(bufs["vox"], 0, bufs["pg"]["vis_mask"], bufs["pg"]["gathered"])
+    rb = br.rulebook(bufs["vox"], 0)
+    oc = br.occlusion(d["points"], d["proj"], bufs["pg"]["vis_mask"], 8, 0.5)
+    pooled = br.pool_features(d["feat"], 2)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        br.run_staged(d["points"], d["proj"], d["feat"], bufs)
+        br.voxel_image(bufs["vox"], 0, bufs["pg"]["vis_mask"], bufs["pg"]["gathered"], vi)
+        br.rulebook(bufs["vox"], 0, out=rb)
+        br.occlusion(d["points"], d["proj"], bufs["pg"]["vis_mask"], 8, 0.5, oc)
+        br.pool_features(d["feat"], 2, out=pooled)
+    for k, v in second.items():
+        d[k].copy_(torch.from_numpy(v))
+    for t in (rb["rule_in"], oc["occ_mask"], vi["vox_img_count"]):
+        t.fill_(-1 if t.dtype != torch.uint8 else 255)
+    graph.replay()
+    torch.cuda.synchronize()
+    br.status()
+    ref = oracle.bridge(w, second)
+    compare_bridge(w, ref, bufs)
+    M = ref["vox0"]["num_voxels"]
+    off, rin, rout = oracle.rulebook(ref["vox0"]["coords"][:M])
+    assert np.array_equal(np_(rb["offsets"]), off) and np.array_equal(np_(rb["rule_in"])[:off[27]], rin)
+    _, cnt = oracle.voxel_image(ref["vox0"]["point_voxel"], M, ref["vis_mask"], ref["gathered"])
+    assert np.array_equal(np_(vi["vox_img_count"])[:M], cnt)
+    _, want_occ, _ = oracle.occlusion(second["points"], second["proj"], w.img_h, w.img_w, ref["vis_mask"], 8, 0.5)
+    assert np.array_equal(np_(oc["occ_mask"]), want_occ)
+    assert np.abs(np_(pooled).astype(np.float64) - oracle.pool(second["feat"], 2)).max() <= 1e-5
+    del graph
     br.close()
 
 
