@@ -167,6 +167,23 @@ int emc2_bridge_run(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_
                     float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
                     float* d_points_out, float* d_feat_out, void* cuda_stream);
 
+/* emc2_bridge_run for a caller whose frame lives in HOST memory (the sensor side of Sec. 3.1: LiDAR
+ * points, calibration and image features arrive on the host): enqueues, on `cuda_stream`, the copies
+ * of h_points [B, N, C], h_proj [B, K, 3, 4] and h_feat [B, K, Hf, Wf, Cf] into the caller's device
+ * buffers d_points, d_proj, d_feat, then emc2_bridge_run on them with the same outputs, then the
+ * copies of d_offsets [B, E+1] and d_num_voxels [2] into h_offsets and h_num_voxels (either may be
+ * NULL: not copied).  Nothing is synchronised: the host buffers must stay valid and unchanged until
+ * the stream has passed the call; the copies are asynchronous only for page-locked host memory.  A
+ * caller who alternates between two handles, streams and buffer sets overlaps one frame's copies with
+ * the other's kernels. */
+int emc2_bridge_run_host(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* h_points, const float* h_proj,
+                         const float* h_feat, float* d_points, float* d_proj, float* d_feat,
+                         int32_t* const d_coords[2], int32_t* const d_counts[2], float* const d_mean[2],
+                         int32_t* const d_point_voxel[2], const int32_t capacity[2], int32_t* d_num_voxels,
+                         float* d_bev, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam, float* d_gathered,
+                         uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm, float* d_points_out,
+                         float* d_feat_out, int32_t* h_offsets, int32_t* h_num_voxels, void* cuda_stream);
+
 /* Layout change for callers whose image branch (a ResNet in Sec. 3.1) emits planar maps: copies
  * d_planar float [B, K, Cf, Hf, Wf] into d_feat float [B, K, Hf, Wf, Cf], the channels-last layout
  * the gather reads (one tap = one contiguous row).  The handle's K, Hf, Wf, Cf apply; the two

@@ -33,7 +33,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_status", "emc2_bridge_destroy", "emc2_status_string", "emc2_bridge_last_cuda_error",
     "emc2_bridge_scratch_bytes", "emc2_bridge_kernel_kinds", "emc2_bridge_kernel_name",
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
-    "emc2_bridge_run", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
+    "emc2_bridge_run", "emc2_bridge_run_host", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
     "emc2_features_channels_last",
     "emc2_voxel_image", "emc2_occlusion", "emc2_rulebook",
 )
@@ -81,6 +81,8 @@ def load_library() -> ctypes.CDLL:
     lib.emc2_route_dispatch.argtypes = [vp, i32, i32] + [vp] * 9
     lib.emc2_bridge_run.argtypes = ([vp, i32, i32, vp, vp, vp, P(vp), P(vp), P(vp), P(vp), P(i32), vp, vp]
                                     + [vp] * 4 + [vp] * 5 + [vp])
+    lib.emc2_bridge_run_host.argtypes = ([vp, i32, i32] + [vp] * 6 + [P(vp), P(vp), P(vp), P(vp), P(i32), vp, vp]
+                                         + [vp] * 4 + [vp] * 5 + [vp, vp, vp])
     lib.emc2_route_dispatch_static.argtypes = [P(Emc2Config), i32, i32] + [vp] * 9
     lib.emc2_bridge_status.argtypes = [vp, vp]
     lib.emc2_occlusion.argtypes = [vp, i32, i32, vp, vp, vp, i32, ctypes.c_float, vp, vp, vp, vp]
@@ -466,6 +468,43 @@ class Bridge:
             rd["expert"].data_ptr(), rd["offsets"].data_ptr(), rd["perm"].data_ptr(),
             rd["points_out"].data_ptr(), rd["feat_out"].data_ptr(), self._stream())
         self._raise(rc, "emc2_bridge_run")
+        return bufs
+
+    def run_host(self, host: Dict[str, torch.Tensor], staging: Dict[str, torch.Tensor], bufs: Dict[str, object],
+                 h_offsets: Optional[torch.Tensor] = None, h_num_voxels: Optional[torch.Tensor] = None) -> Dict[str, object]:
+        """emc2_bridge_run_host: host tensors ``points, proj, feat`` are copied into the device tensors of
+        ``staging``, the whole bridge runs into ``bufs`` (as :meth:`run` returns them), offsets and voxel
+        counts are copied to the host tensors given.  Everything is only enqueued on the current stream."""
+        c = self.cfg
+        B, N, C = host["points"].shape
+        shapes = {"points": (B, N, c.point_floats), "proj": (B, c.num_cameras, 3, 4),
+                  "feat": (B, c.num_cameras, c.feat_h, c.feat_w, c.feat_c)}
+        for k, shp in shapes.items():
+            _check(staging[k], torch.float32, shp, "staging " + k, self.device)
+            t = host[k]
+            if t.device.type != "cpu" or t.dtype != torch.float32 or tuple(t.shape) != shp or not t.is_contiguous():
+                raise ValueError(f"host {k}: need a contiguous float32 CPU tensor of shape {shp}")
+        for t, shp, name in ((h_offsets, (B, c.num_experts + 1), "h_offsets"), (h_num_voxels, (2,), "h_num_voxels")):
+            if t is not None and (t.device.type != "cpu" or t.dtype != torch.int32 or tuple(t.shape) != shp
+                                  or not t.is_contiguous()):
+                raise ValueError(f"{name}: need a contiguous int32 CPU tensor of shape {shp}")
+        vox, pg, rd = bufs["vox"], bufs["pg"], bufs["rd"]
+        arr = ctypes.c_void_p * 2
+        pv = vox["point_voxel"]
+        cap = [int(vox["coords"][s].shape[0]) for s in range(2)]
+        rc = self.lib.emc2_bridge_run_host(
+            self._h, B, N, host["points"].data_ptr(), host["proj"].data_ptr(), host["feat"].data_ptr(),
+            staging["points"].data_ptr(), staging["proj"].data_ptr(), staging["feat"].data_ptr(),
+            arr(*[t.data_ptr() for t in vox["coords"]]), arr(*[t.data_ptr() for t in vox["counts"]]),
+            arr(*[t.data_ptr() for t in vox["mean"]]),
+            arr(*[t.data_ptr() for t in pv]) if pv is not None else None,
+            (ctypes.c_int32 * 2)(*cap), vox["num_voxels"].data_ptr(), _ptr(vox["bev"]),
+            pg["uvd"].data_ptr(), pg["vis_mask"].data_ptr(), pg["cam"].data_ptr(), pg["gathered"].data_ptr(),
+            rd["expert"].data_ptr(), rd["offsets"].data_ptr(), rd["perm"].data_ptr(),
+            rd["points_out"].data_ptr(), rd["feat_out"].data_ptr(),
+            h_offsets.data_ptr() if h_offsets is not None else None,
+            h_num_voxels.data_ptr() if h_num_voxels is not None else None, self._stream())
+        self._raise(rc, "emc2_bridge_run_host")
         return bufs
 
     # ------------------------------------------------------------------ measurement aids

@@ -393,6 +393,43 @@ int emc2_occlusion(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points
                             d_occ_mask, d_clear_mask, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int emc2_bridge_run_host(emc2_bridge_t* h, int32_t B, int32_t N, const float* h_points, const float* h_proj,
+                         const float* h_feat, float* d_points, float* d_proj, float* d_feat,
+                         int32_t* const d_coords[2], int32_t* const d_counts[2], float* const d_mean[2],
+                         int32_t* const d_point_voxel[2], const int32_t capacity[2], int32_t* d_num_voxels,
+                         float* d_bev, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam, float* d_gathered,
+                         uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm, float* d_points_out,
+                         float* d_feat_out, int32_t* h_offsets, int32_t* h_num_voxels, void* cuda_stream) {
+    int rc = check_call(h, B, N);
+    if (rc != EMC2_OK) return rc;
+    const emc2_config_t& c = h->cfg;
+    if (B > 0 && (!h_proj || !h_feat || !d_proj || !d_feat || (N > 0 && (!h_points || !d_points))))
+        return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(c.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaSuccess;
+    if (B > 0) {
+        const size_t pts = (size_t)B * N * c.point_floats * sizeof(float);
+        const size_t prj = (size_t)B * c.num_cameras * 12 * sizeof(float);
+        const size_t fts = (size_t)B * c.num_cameras * c.feat_h * c.feat_w * c.feat_c * sizeof(float);
+        if (pts) e = cudaMemcpyAsync(d_points, h_points, pts, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(d_proj, h_proj, prj, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(d_feat, h_feat, fts, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return check_cuda(h, e);
+    }
+    rc = emc2_bridge_run(h, B, N, d_points, d_proj, d_feat, d_coords, d_counts, d_mean, d_point_voxel, capacity,
+                         d_num_voxels, d_bev, d_uvd, d_vis_mask, d_cam, d_gathered, d_expert, d_offsets, d_perm,
+                         d_points_out, d_feat_out, cuda_stream);
+    if (rc != EMC2_OK) return rc;
+    if (h_offsets && d_offsets && B > 0)
+        e = cudaMemcpyAsync(h_offsets, d_offsets, (size_t)B * (c.num_experts + 1) * sizeof(int32_t),
+                            cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && h_num_voxels && d_num_voxels)
+        e = cudaMemcpyAsync(h_num_voxels, d_num_voxels, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+    return check_cuda(h, e);
+}
+
 int emc2_features_channels_last(emc2_bridge_t* h, int32_t B, const float* d_planar, float* d_feat,
                                 void* cuda_stream) {
     if (!h || B < 0 || B > h->cfg.max_batch) return EMC2_ERR_INVALID_ARG;

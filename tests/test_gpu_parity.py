@@ -85,6 +85,34 @@ def test_one_call_on_a_side_stream_of_the_caller(b200, oracle):
     br.close()
 
 
+def test_one_call_from_host_buffers(b200, oracle):
+    # pinned and pageable host memory; results come back into host tensors without a sync by the library
+    w = gen.NUSCENES.with_shape(2, 20000)
+    batch = gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])          # output buffers of the right shapes
+    for pinned in (True, False):
+        host = {k: torch.from_numpy(v.copy()) for k, v in batch.items()}
+        if pinned:
+            host = {k: v.pin_memory() for k, v in host.items()}
+        staging = {k: torch.full_like(v, float("nan")) for k, v in d.items()}
+        h_off = torch.full((w.B, w.num_experts + 1), -1, dtype=torch.int32)
+        h_nv = torch.full((2,), -1, dtype=torch.int32)
+        if pinned:
+            h_off, h_nv = h_off.pin_memory(), h_nv.pin_memory()
+        bufs["rd"]["feat_out"].fill_(-1.0)
+        br.run_host(host, staging, bufs, h_off, h_nv)
+        torch.cuda.synchronize()
+        br.status()
+        compare_bridge(w, ref, bufs)
+        assert np.array_equal(h_off.numpy(), ref["offsets"])
+        assert h_nv.tolist() == [ref["vox0"]["num_voxels"], ref["vox1"]["num_voxels"]]
+        assert torch.equal(staging["points"].cpu(), host["points"])
+    br.close()
+
+
 def test_one_call_replays_from_a_cuda_graph(b200, oracle):
     # emc2_bridge_run only enqueues (kernels, a fork and a join by events), so a caller can capture
     # it once and replay it on new frames written into the same buffers.
