@@ -238,6 +238,17 @@ int emc2_voxel_image(emc2_bridge_t* bridge, int32_t B, int32_t N, int32_t capaci
                      const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
                      const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, void* cuda_stream);
 
+/* Fusion by voxel straight from the feature maps (Fig. 5 again; this is the per-voxel form of the
+ * bridge's image branch: the per-point rows of emc2_project_gather are neither written nor read).
+ * Outputs as emc2_voxel_image.  Instead of the gathered rows and the visibility mask the call takes
+ * d_uvd float [B, N, 3] and d_cam int8 [B, N] of the projection stage and the feature maps d_feat
+ * float [B, K, Hf, Wf, Cf]; a point counts iff d_cam >= 0, and its row is the bilinear blend the
+ * gather stage would have produced.  Same scratch, same ordering rule as emc2_voxel_image. */
+int emc2_voxel_image_sampled(emc2_bridge_t* bridge, int32_t B, int32_t N, int32_t capacity,
+                             const int32_t* d_point_voxel, const int32_t* d_counts, const int32_t* d_num_voxels,
+                             const float* d_uvd, const int8_t* d_cam, const float* d_feat, float* d_vox_img,
+                             int32_t* d_vox_img_count, void* cuda_stream);
+
 /* Occlusion test for the "occluded / out-of-view" bucket of the dispatcher (Sec. 3.2 names occlusion
  * among the causes of missing LiDAR detail; the paper gives no test, this is a depth buffer).  Every
  * camera image is cut into cells of cell x cell pixels (cell a power of two).  For each camera k that

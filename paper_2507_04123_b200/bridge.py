@@ -35,7 +35,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_profile_enable", "emc2_bridge_profile_read", "emc2_route_dispatch_static",
     "emc2_bridge_run", "emc2_bridge_run_host", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
     "emc2_features_channels_last",
-    "emc2_voxel_image", "emc2_occlusion", "emc2_rulebook",
+    "emc2_voxel_image", "emc2_voxel_image_sampled", "emc2_occlusion", "emc2_rulebook",
 )
 
 
@@ -87,6 +87,7 @@ def load_library() -> ctypes.CDLL:
     lib.emc2_bridge_status.argtypes = [vp, vp]
     lib.emc2_occlusion.argtypes = [vp, i32, i32, vp, vp, vp, i32, ctypes.c_float, vp, vp, vp, vp]
     lib.emc2_voxel_image.argtypes = [vp, i32, i32, i32] + [vp] * 8
+    lib.emc2_voxel_image_sampled.argtypes = [vp, i32, i32, i32] + [vp] * 9
     lib.emc2_rulebook.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, ctypes.c_int64, vp]
     lib.emc2_pool_features.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.emc2_features_channels_last.argtypes = [vp, i32, vp, vp, vp]
@@ -316,6 +317,29 @@ class Bridge:
                                        nv.data_ptr() + 4 * scale, vis_mask.data_ptr(), gathered.data_ptr(),
                                        out["vox_img"].data_ptr(), out["vox_img_count"].data_ptr(), self._stream())
         self._raise(rc, "emc2_voxel_image")
+        return out
+
+    def voxel_image_sampled(self, vox: Dict[str, object], scale: int, uvd: torch.Tensor, cam: torch.Tensor,
+                            feat: torch.Tensor, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        """emc2_voxel_image_sampled: per-voxel image features blended straight from the feature maps."""
+        B, N = cam.shape
+        c = self.cfg
+        pv = vox["point_voxel"][scale]
+        counts = vox["counts"][scale]
+        cap = int(counts.shape[0])
+        _check(pv, torch.int32, (B, N), "point_voxel", self.device)
+        _check(uvd, torch.float32, (B, N, 3), "uvd", self.device)
+        _check(cam, torch.int8, (B, N), "cam", self.device)
+        _check(feat, torch.float32, (B, c.num_cameras, c.feat_h, c.feat_w, c.feat_c), "feat", self.device)
+        if out is None:
+            out = {"vox_img": torch.empty((cap, c.feat_c), dtype=torch.float32, device=self.device),
+                   "vox_img_count": torch.empty((cap,), dtype=torch.int32, device=self.device)}
+        nv = vox["num_voxels"]
+        rc = self.lib.emc2_voxel_image_sampled(self._h, B, N, cap, pv.data_ptr(), counts.data_ptr(),
+                                               nv.data_ptr() + 4 * scale, uvd.data_ptr(), cam.data_ptr(),
+                                               feat.data_ptr(), out["vox_img"].data_ptr(),
+                                               out["vox_img_count"].data_ptr(), self._stream())
+        self._raise(rc, "emc2_voxel_image_sampled")
         return out
 
     def rulebook(self, vox: Dict[str, object], scale: int, pair_capacity: Optional[int] = None,

@@ -10,7 +10,7 @@ namespace emc2 {
 static const char* const kKernelNames[K_KINDS] = {
     "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
     "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features",
-    "vif_scan", "vif_fill", "vif_mean", "occl_fill", "occl_splat", "occl_test",
+    "vif_scan", "vif_fill", "vif_mean", "vif_sample", "occl_fill", "occl_splat", "occl_test",
     "channels_last", "rb_mark", "rb_count", "rb_scan", "rb_fill", "rb_clear"};
 
 int check_cuda(emc2_bridge* h, cudaError_t e) {
@@ -174,6 +174,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     const size_t o_vif_start = plan.take(maxpts * sizeof(int));
     const size_t o_vif_cursor = plan.take(maxpts * sizeof(int));
     const size_t o_vif_list = plan.take(maxpts * sizeof(int));
+    const size_t o_vif_recs = plan.take(maxpts * sizeof(uint4));
     const size_t o_vif_part = plan.take((size_t)h->vif_scan_blocks * sizeof(int));
     const size_t rb_tiles = (maxpts + kTile - 1) / kTile;
     const size_t o_rb_bits = plan.take(maxpts * sizeof(uint32_t));
@@ -210,6 +211,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     h->d_vif_start = reinterpret_cast<int*>(base + o_vif_start);
     h->d_vif_cursor = reinterpret_cast<int*>(base + o_vif_cursor);
     h->d_vif_list = reinterpret_cast<int*>(base + o_vif_list);
+    h->d_vif_recs = reinterpret_cast<uint4*>(base + o_vif_recs);
     h->d_vif_part = reinterpret_cast<int*>(base + o_vif_part);
     h->d_rb_bits = reinterpret_cast<uint32_t*>(base + o_rb_bits);
     h->d_rb_counts = reinterpret_cast<int*>(base + o_rb_counts);
@@ -359,7 +361,25 @@ int emc2_voxel_image(emc2_bridge_t* h, int32_t B, int32_t N, int32_t capacity, c
     DeviceGuard guard(h->cfg.device);
     if (!guard.ok) return EMC2_ERR_CUDA;
     return launch_voxel_image(h, B, N, capacity, d_point_voxel, d_counts, d_num_voxels, d_vis_mask, d_gathered,
-                              d_vox_img, d_vox_img_count, static_cast<cudaStream_t>(cuda_stream));
+                              nullptr, nullptr, nullptr, d_vox_img, d_vox_img_count,
+                              static_cast<cudaStream_t>(cuda_stream));
+}
+
+int emc2_voxel_image_sampled(emc2_bridge_t* h, int32_t B, int32_t N, int32_t capacity, const int32_t* d_point_voxel,
+                             const int32_t* d_counts, const int32_t* d_num_voxels, const float* d_uvd,
+                             const int8_t* d_cam, const float* d_feat, float* d_vox_img, int32_t* d_vox_img_count,
+                             void* cuda_stream) {
+    int rc = check_call(h, B, N);
+    if (rc != EMC2_OK) return rc;
+    if (capacity < 0 || !d_num_voxels) return EMC2_ERR_INVALID_ARG;
+    if (B == 0 || N == 0 || capacity == 0) return EMC2_OK;
+    if (!d_point_voxel || !d_counts || !d_uvd || !d_cam || !d_feat || !d_vox_img || !d_vox_img_count)
+        return EMC2_ERR_INVALID_ARG;
+    if (!aligned16(d_feat) || !aligned16(d_vox_img)) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_voxel_image(h, B, N, capacity, d_point_voxel, d_counts, d_num_voxels, nullptr, nullptr, d_uvd,
+                              d_cam, d_feat, d_vox_img, d_vox_img_count, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int emc2_rulebook(emc2_bridge_t* h, int32_t scale, int32_t capacity, const int32_t* d_coords,

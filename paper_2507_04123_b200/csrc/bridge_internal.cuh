@@ -35,6 +35,7 @@ enum KernelKind {
     K_VIF_SCAN,
     K_VIF_FILL,
     K_VIF_MEAN,
+    K_VIF_SAMPLE,
     K_OCCL_FILL,
     K_OCCL_SPLAT,
     K_OCCL_TEST,
@@ -129,6 +130,7 @@ struct emc2_bridge {
     int* d_vif_start = nullptr;    // emc2_voxel_image: [max points] list starts, cursors, lists
     int* d_vif_cursor = nullptr;
     int* d_vif_list = nullptr;
+    uint4* d_vif_recs = nullptr;   // emc2_voxel_image_sampled: [max points] tap records in list order
     int* d_vif_part = nullptr;     // [vif_scan_blocks]
     int vif_scan_blocks = 0;
     uint32_t* d_rb_bits = nullptr;  // emc2_rulebook: [max points] neighbour bits per voxel
@@ -187,7 +189,8 @@ int launch_occlusion(emc2_bridge* h, int B, int N, const float* d_points, const 
 int voxel_image_scan_max_blocks();
 int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t* d_point_voxel,
                        const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
-                       const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st);
+                       const float* d_gathered, const float* d_uvd, const int8_t* d_cam, const float* d_feat,
+                       float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st);
 int launch_rulebook(emc2_bridge* h, int scale, int capacity, const int32_t* d_coords, const int32_t* d_num_voxels,
                     int32_t* d_rule_offsets, int32_t* d_rule_in, int32_t* d_rule_out, long long pair_capacity,
                     cudaStream_t st);
@@ -235,6 +238,57 @@ __device__ __forceinline__ uint32_t cell_of(const ScaleDev& g, float x, float y,
 }
 
 __device__ __forceinline__ int warp_sum(int v) { return __reduce_add_sync(0xFFFFFFFFu, v); }
+
+// ---- bilinear sampling of the channels-last feature maps (used by every kernel that blends rows)
+constexpr uint32_t kZeroRow = 0xFFFFFFFFu;
+
+__device__ __forceinline__ float4 blend(const float4& f00, const float4& f01, const float4& f10, const float4& f11,
+                                        float wx, float wy) {
+    const float ax = 1.0f - wx, ay = 1.0f - wy;
+    float4 o;
+    o.x = ay * (ax * f00.x + wx * f01.x) + wy * (ax * f10.x + wx * f11.x);
+    o.y = ay * (ax * f00.y + wx * f01.y) + wy * (ax * f10.y + wx * f11.y);
+    o.z = ay * (ax * f00.z + wx * f01.z) + wy * (ax * f10.z + wx * f11.z);
+    o.w = ay * (ax * f00.w + wx * f01.w) + wy * (ax * f10.w + wx * f11.w);
+    return o;
+}
+
+// Tap record of a point seen by camera `cam` of frame b at pixel (u, v): {float4 index of tap
+// (y0, x0), clamp flags, wx, wy}; kZeroRow in .x for a point no camera sees.
+__device__ __forceinline__ uint4 tap_record(int b, int cam, float u, float v, int K, int Hf, int Wf, int cf4,
+                                            float inv_stride, float offset) {
+    uint4 rec = make_uint4(kZeroRow, 0u, 0u, 0u);
+    if (cam >= 0) {
+        // Texel coordinates: one fp32 subtraction, then an exact scaling (the stride is a power of
+        // two).  Taps are clamped to the map on every side.
+        const float fx = __fsub_rn(u, offset) * inv_stride, fy = __fsub_rn(v, offset) * inv_stride;
+        const float flx = floorf(fx), fly = floorf(fy);
+        int x0 = (int)flx, y0 = (int)fly;
+        const int x1 = max(min(x0 + 1, Wf - 1), 0), y1 = max(min(y0 + 1, Hf - 1), 0);
+        x0 = max(min(x0, Wf - 1), 0);
+        y0 = max(min(y0, Hf - 1), 0);
+        const uint32_t map = ((uint32_t)b * K + cam) * Hf;
+        rec.x = ((map + y0) * Wf + x0) * (uint32_t)cf4;
+        rec.y = (uint32_t)(x1 - x0) | ((uint32_t)(y1 - y0) << 1);
+        rec.z = __float_as_uint(fx - flx);
+        rec.w = __float_as_uint(fy - fly);
+    }
+    return rec;
+}
+
+// Blended feature column c of the row described by `rec` (zeros for kZeroRow).
+__device__ __forceinline__ float4 gather_column(const float4* __restrict__ feat, const uint4& rec, int c, uint32_t cf4,
+                                                uint32_t row_stride) {
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (rec.x != kZeroRow) {
+        const float4* p = feat + rec.x + c;
+        const uint32_t dx = (rec.y & 1u) ? cf4 : 0u, dy = (rec.y & 2u) ? row_stride : 0u;
+        const float4 f00 = __ldg(p), f01 = __ldg(p + dx), f10 = __ldg(p + dy), f11 = __ldg(p + dy + dx);
+        o = blend(f00, f01, f10, f11, __uint_as_float(rec.z), __uint_as_float(rec.w));
+    }
+    return o;
+}
+
 
 #endif  // __CUDACC__
 

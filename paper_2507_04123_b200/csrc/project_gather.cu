@@ -27,19 +27,6 @@ struct PgArgs {
     float min_depth, inv_stride, offset;
 };
 
-constexpr uint32_t kZeroRow = 0xFFFFFFFFu;
-
-__device__ __forceinline__ float4 blend(const float4& f00, const float4& f01, const float4& f10, const float4& f11,
-                                        float wx, float wy) {
-    const float ax = 1.0f - wx, ay = 1.0f - wy;
-    float4 o;
-    o.x = ay * (ax * f00.x + wx * f01.x) + wy * (ax * f10.x + wx * f11.x);
-    o.y = ay * (ax * f00.y + wx * f01.y) + wy * (ax * f10.y + wx * f11.y);
-    o.z = ay * (ax * f00.z + wx * f01.z) + wy * (ax * f10.z + wx * f11.z);
-    o.w = ay * (ax * f00.w + wx * f01.w) + wy * (ax * f10.w + wx * f11.w);
-    return o;
-}
-
 // Projection of one point into the K cameras of its frame (P: [K][3][4] row-major).
 struct Projected {
     unsigned mask;      // bit k: visible in camera k
@@ -93,42 +80,6 @@ __device__ __forceinline__ Projected project_point(const float4* P, int K, float
 __device__ __forceinline__ void load_proj(const float* __restrict__ proj, int b, int K, float4* sP) {
     const float4* src = reinterpret_cast<const float4*>(proj) + (size_t)b * K * 3;
     for (int i = threadIdx.x; i < K * 3; i += blockDim.x) sP[i] = __ldg(src + i);
-}
-
-// Tap record of a point seen by camera `cam` of frame b at pixel (u, v): {float4 index of tap
-// (y0, x0), clamp flags, wx, wy}; kZeroRow in .x for a point no camera sees.
-__device__ __forceinline__ uint4 tap_record(int b, int cam, float u, float v, int K, int Hf, int Wf, int cf4,
-                                            float inv_stride, float offset) {
-    uint4 rec = make_uint4(kZeroRow, 0u, 0u, 0u);
-    if (cam >= 0) {
-        // Texel coordinates: one fp32 subtraction, then an exact scaling (the stride is a power of
-        // two).  Taps are clamped to the map on every side.
-        const float fx = __fsub_rn(u, offset) * inv_stride, fy = __fsub_rn(v, offset) * inv_stride;
-        const float flx = floorf(fx), fly = floorf(fy);
-        int x0 = (int)flx, y0 = (int)fly;
-        const int x1 = max(min(x0 + 1, Wf - 1), 0), y1 = max(min(y0 + 1, Hf - 1), 0);
-        x0 = max(min(x0, Wf - 1), 0);
-        y0 = max(min(y0, Hf - 1), 0);
-        const uint32_t map = ((uint32_t)b * K + cam) * Hf;
-        rec.x = ((map + y0) * Wf + x0) * (uint32_t)cf4;
-        rec.y = (uint32_t)(x1 - x0) | ((uint32_t)(y1 - y0) << 1);
-        rec.z = __float_as_uint(fx - flx);
-        rec.w = __float_as_uint(fy - fly);
-    }
-    return rec;
-}
-
-// Blended feature column c of the row described by `rec` (zeros for kZeroRow).
-__device__ __forceinline__ float4 gather_column(const float4* __restrict__ feat, const uint4& rec, int c, uint32_t cf4,
-                                                uint32_t row_stride) {
-    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (rec.x != kZeroRow) {
-        const float4* p = feat + rec.x + c;
-        const uint32_t dx = (rec.y & 1u) ? cf4 : 0u, dy = (rec.y & 2u) ? row_stride : 0u;
-        const float4 f00 = __ldg(p), f01 = __ldg(p + dx), f10 = __ldg(p + dy), f11 = __ldg(p + dy + dx);
-        o = blend(f00, f01, f10, f11, __uint_as_float(rec.z), __uint_as_float(rec.w));
-    }
-    return o;
 }
 
 // CF4 > 0: Cf/4 known at compile time, blockDim.x == 16 * CF4.  CF4 == 0: any Cf, 256 threads.

@@ -10,6 +10,9 @@
 //   vif_fill   every kept point takes a ticket in its voxel's list (one atomic with return).
 //   vif_mean   16 voxels x Cf/4 columns of threads per CTA: a voxel's threads walk its list and
 //              read each visible point's row with one contiguous 128-bit load per thread.
+//   vif_sample the same, but the rows are blended from the feature maps on the spot
+//              (emc2_voxel_image_sampled: no [points, Cf] buffer at all); for it vif_fill stores
+//              each listed point's tap record (16 bytes) in place of its index.
 #include <cooperative_groups.h>
 
 #include "bridge_internal.cuh"
@@ -23,13 +26,19 @@ struct VifArgs {
     const int32_t* pv;          // [total] row of the point's voxel, -1 if none
     const int32_t* counts;      // [M] kept points per voxel
     const int32_t* num_voxels;  // device: voxels found by emc2_voxelize for this scale
-    const uint8_t* vis;         // [total]
-    const float4* gathered;     // [total, cf4]
+    const uint8_t* vis;         // [total], or null: a point is visible iff cam[i] >= 0
+    const float4* gathered;     // [total, cf4] (vif_mean)
+    const int8_t* cam;          // [total] camera of every point (vif_sample)
+    const float* uvd;           // [total, 3] pixel and depth in that camera (vif_sample)
+    const float4* feat;         // feature maps (vif_sample)
+    int N, K, Hf, Wf;
+    float inv_stride, offset;
     float4* vox_img;            // [capacity, cf4]
     int32_t* vox_cnt;           // [capacity]
     int* start;                 // [capacity] first list slot of each voxel
     int* cursor;                // [capacity]
     int* list;                  // [total] point indices; bitwise complement for points no camera sees
+    uint4* recs;                // [total] vif_sample: tap record of every listed point, in list order
     int* part;                  // [gridDim.x]
     long long total;
     int capacity, cf4;
@@ -86,7 +95,12 @@ __global__ void __launch_bounds__(kThreads) vif_fill_kernel(VifArgs a) {
         const int m = a.pv[i];
         if (m < 0 || m >= M) continue;
         const int pos = a.start[m] + atomicAdd(&a.cursor[m], 1);
-        a.list[pos] = a.vis[i] ? (int)i : ~(int)i;
+        if (a.vis) {
+            a.list[pos] = a.vis[i] ? (int)i : ~(int)i;
+        } else {                                        // rows will be blended from the maps: keep the taps
+            a.recs[pos] = tap_record((int)(i / a.N), (int)a.cam[i], a.uvd[3 * i], a.uvd[3 * i + 1], a.K, a.Hf, a.Wf,
+                                     a.cf4, a.inv_stride, a.offset);
+        }
     }
 }
 
@@ -148,6 +162,70 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_mean_kernel
     }
 }
 
+// vif_mean without the per-point rows: every listed point's row is blended from its four taps of
+// the feature maps here (the blend of the gather stage, from the point's pixel and camera), so the
+// [points, Cf] buffer is neither written nor read.  Same thread layout as vif_mean.
+template <int CF4>
+__global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_sample_kernel(VifArgs a) {
+    const int M = voxels_in_use(a);
+    const int cf4 = CF4 > 0 ? CF4 : a.cf4;
+    const int rows = (int)blockDim.x / cf4;
+    const int r = (int)threadIdx.x / cf4, c = (int)threadIdx.x - r * cf4;
+    if (r >= rows) return;
+    const uint32_t row_stride = (uint32_t)a.Wf * cf4;
+    const int stride = gridDim.x * rows;
+    for (int m0 = blockIdx.x * rows + r; m0 < M; m0 += 2 * stride) {
+        int mm[2] = {m0, m0 + stride}, s0[2], n[2], seen[2] = {0, 0};
+        float4 acc[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const bool ok = mm[u] < M;
+            s0[u] = ok ? a.start[mm[u]] : 0;
+            n[u] = ok ? a.counts[mm[u]] : 0;
+            acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        // The first entries of the two voxels together, then the rest of each list, two at a time;
+        // every voxel's rows are added in list order.
+        {
+            uint4 rec[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) rec[u] = n[u] > 0 ? a.recs[s0[u]] : make_uint4(kZeroRow, 0u, 0u, 0u);
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                acc[u] = gather_column(a.feat, rec[u], c, (uint32_t)cf4, row_stride);
+                seen[u] = rec[u].x != kZeroRow ? 1 : 0;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            for (int k = 1; k < n[u]; k += 2) {
+                uint4 rec[2];
+                float4 v[2];
+#pragma unroll
+                for (int j = 0; j < 2; ++j) rec[j] = k + j < n[u] ? a.recs[s0[u] + k + j] : make_uint4(kZeroRow, 0u, 0u, 0u);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) v[j] = gather_column(a.feat, rec[j], c, (uint32_t)cf4, row_stride);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    if (rec[j].x == kZeroRow) continue;
+                    acc[u].x += v[j].x; acc[u].y += v[j].y; acc[u].z += v[j].z; acc[u].w += v[j].w;
+                    seen[u] += 1;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (mm[u] >= M) continue;
+            if (seen[u] > 1) {
+                const float inv = 1.0f / (float)seen[u];
+                acc[u].x *= inv; acc[u].y *= inv; acc[u].z *= inv; acc[u].w *= inv;
+            }
+            __stcs(a.vox_img + (size_t)mm[u] * cf4 + c, acc[u]);
+            if (c == 0) a.vox_cnt[mm[u]] = seen[u];
+        }
+    }
+}
+
 }  // namespace
 
 int voxel_image_scan_max_blocks() {
@@ -158,17 +236,25 @@ int voxel_image_scan_max_blocks() {
     return sms * min(per_sm, 2);
 }
 
+// d_gathered != null: rows are read from it and d_vis_mask says which points count; else rows are
+// sampled from d_feat at d_uvd in camera d_cam, and a point counts iff its camera is >= 0.
 int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t* d_point_voxel,
                        const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
-                       const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st) {
+                       const float* d_gathered, const float* d_uvd, const int8_t* d_cam, const float* d_feat,
+                       float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st) {
+    const emc2_config_t& cfg = h->cfg;
     VifArgs a;
     a.pv = d_point_voxel; a.counts = d_counts; a.num_voxels = d_num_voxels; a.vis = d_vis_mask;
     a.gathered = reinterpret_cast<const float4*>(d_gathered);
+    a.cam = d_cam; a.uvd = d_uvd; a.feat = reinterpret_cast<const float4*>(d_feat);
+    a.N = N; a.K = cfg.num_cameras; a.Hf = cfg.feat_h; a.Wf = cfg.feat_w;
+    a.inv_stride = 1.0f / (float)cfg.feat_stride; a.offset = cfg.feat_offset;
     a.vox_img = reinterpret_cast<float4*>(d_vox_img); a.vox_cnt = d_vox_img_count;
     a.start = h->d_vif_start; a.cursor = h->d_vif_cursor; a.list = h->d_vif_list; a.part = h->d_vif_part;
+    a.recs = h->d_vif_recs;
     a.total = (long long)B * N;
     a.capacity = (int)min((long long)capacity, a.total);   // a voxel holds at least one point
-    a.cf4 = h->cfg.feat_c / 4;
+    a.cf4 = cfg.feat_c / 4;
     if (a.total == 0 || a.capacity == 0) return EMC2_OK;
     if (a.cf4 > kThreads) return EMC2_ERR_INVALID_ARG;      // a feature row must fit one CTA
     {
@@ -183,13 +269,20 @@ int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t
         const int blocks = (int)min((long long)148 * 16, (a.total + kThreads - 1) / kThreads);
         vif_fill_kernel<<<blocks, kThreads, 0, st>>>(a);
     }
-    {
+    const int blocks = (int)min((long long)148 * 16, ((long long)a.capacity + 15) / 16);
+    if (d_gathered) {
         LaunchScope ls(h, K_VIF_MEAN, st);
-        const int blocks = (int)min((long long)148 * 16, ((long long)a.capacity + 15) / 16);
         switch (a.cf4) {
             case 16: vif_mean_kernel<16><<<blocks, 16 * 16, 0, st>>>(a); break;
             case 20: vif_mean_kernel<20><<<blocks, 16 * 20, 0, st>>>(a); break;
             default: vif_mean_kernel<0><<<blocks, kThreads, 0, st>>>(a); break;
+        }
+    } else {
+        LaunchScope ls(h, K_VIF_SAMPLE, st);
+        switch (a.cf4) {
+            case 16: vif_sample_kernel<16><<<blocks, 16 * 16, 0, st>>>(a); break;
+            case 20: vif_sample_kernel<20><<<blocks, 16 * 20, 0, st>>>(a); break;
+            default: vif_sample_kernel<0><<<blocks, kThreads, 0, st>>>(a); break;
         }
     }
     return check_cuda(h, cudaGetLastError());

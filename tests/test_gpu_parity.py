@@ -229,6 +229,13 @@ def test_image_features_per_voxel(b200, oracle, cid, B, N):
             ok, mx, nbad = close(np_(out["vox_img"])[:M], want)
             assert ok, f"scale {s}: max abs err {mx}, {nbad} outside tolerance"
             assert not np_(out["vox_img"])[:M][cnt == 0].any()
+            # the same rows without the per-point buffer: blended from the maps voxel by voxel
+            out = br.voxel_image_sampled(bufs["vox"], s, bufs["pg"]["uvd"], bufs["pg"]["cam"], d["feat"])
+            br.status()
+            assert np.array_equal(np_(out["vox_img_count"])[:M], cnt), s
+            ok, mx, nbad = close(np_(out["vox_img"])[:M], want)
+            assert ok, f"sampled, scale {s}: max abs err {mx}, {nbad} outside tolerance"
+            assert not np_(out["vox_img"])[:M][cnt == 0].any()
     br.close()
 
 
