@@ -287,6 +287,17 @@ def run_ours(args, w):
     for _ in range(3):
         staged_step()
     staged_secs = max_over_ranks(time_steps(staged_step, args.steps, sync, barrier))
+    dispatch_only_secs = None
+    if args.dispatch_only:
+        # The same call for a consumer of the dispatched rows only: the rows in point order are not stored.
+        kept = bufs["pg"]["gathered"]
+        bufs["pg"]["gathered"] = None
+        for _ in range(args.warmup):
+            step()
+        dispatch_only_secs = max_over_ranks(time_steps(step, args.steps, sync, barrier))
+        br.status()
+        bufs["pg"]["gathered"] = kept
+        step()
     graph_secs = None
     if args.graph:
         # The one-call step captured once into a CUDA graph and replayed (fewer launch gaps on small batches).
@@ -408,6 +419,7 @@ def run_ours(args, w):
                          else "working set fits in L2 (latency-bound workload, no flush)"},
         "mpoints_per_s": fps * N / 1e6,
         "staged_ms_per_step": staged_secs / args.steps * 1e3,
+        "dispatch_only_ms_per_step": dispatch_only_secs / args.steps * 1e3 if dispatch_only_secs is not None else None,
         "graph_ms_per_step": graph_secs / args.steps * 1e3 if graph_secs is not None else None,
         "bridge_algorithmic_bytes_per_step": abytes,
         "one_call_bytes_per_step": one_call_bytes(w, B, N, int(nv[0]), int(nv[1]), texels),
@@ -563,6 +575,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--occlusion", action="store_true", help="also time emc2_occlusion (depth-buffer test)")
+    ap.add_argument("--dispatch-only", action="store_true",
+                    help="also time the one-call step without the feature rows in point order (d_gathered = NULL)")
     ap.add_argument("--graph", action="store_true", help="also time the one-call step replayed from a CUDA graph")
     ap.add_argument("--rulebook", action="store_true", help="also time emc2_rulebook (sparse-convolution rulebook)")
     ap.add_argument("--channels-last", action="store_true", help="also time emc2_features_channels_last")

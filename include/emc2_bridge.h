@@ -159,7 +159,9 @@ int emc2_route_dispatch(emc2_bridge_t* bridge, int32_t B, int32_t N, const float
  * priority) beside them: it starts once the work already queued on `cuda_stream` has finished,
  * and `cuda_stream` waits for it before the call's work counts as complete.  Seen from
  * `cuda_stream` the call therefore behaves like the three calls, only shorter.  No allocation,
- * no host synchronisation. */
+ * no host synchronisation.  d_gathered may be NULL for a caller who consumes only the dispatched
+ * rows (d_feat_out with d_perm): the rows in point order are then not stored, which saves their
+ * 4 * Cf bytes per point of memory traffic. */
 int emc2_bridge_run(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_points, const float* d_proj,
                     const float* d_feat, int32_t* const d_coords[2], int32_t* const d_counts[2],
                     float* const d_mean[2], int32_t* const d_point_voxel[2], const int32_t capacity[2],

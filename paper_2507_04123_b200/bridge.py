@@ -460,7 +460,8 @@ class Bridge:
 
     def run(self, points: torch.Tensor, proj: torch.Tensor, feat: torch.Tensor,
             bufs: Optional[Dict[str, object]] = None) -> Dict[str, object]:
-        """emc2_bridge_run: all stages in one call; same outputs as :meth:`run_staged`."""
+        """emc2_bridge_run: all stages in one call; same outputs as :meth:`run_staged`.  With
+        ``bufs["pg"]["gathered"] = None`` the rows in point order are not stored."""
         B, N, C = points.shape
         c = self.cfg
         _check(points, torch.float32, (B, N, c.point_floats), "points", self.device)
@@ -488,7 +489,7 @@ class Bridge:
             arr(*[t.data_ptr() for t in vox["mean"]]),
             arr(*[t.data_ptr() for t in pv]) if pv is not None else None,
             (ctypes.c_int32 * 2)(*cap), vox["num_voxels"].data_ptr(), _ptr(vox["bev"]),
-            pg["uvd"].data_ptr(), pg["vis_mask"].data_ptr(), pg["cam"].data_ptr(), pg["gathered"].data_ptr(),
+            pg["uvd"].data_ptr(), pg["vis_mask"].data_ptr(), pg["cam"].data_ptr(), _ptr(pg.get("gathered")),
             rd["expert"].data_ptr(), rd["offsets"].data_ptr(), rd["perm"].data_ptr(),
             rd["points_out"].data_ptr(), rd["feat_out"].data_ptr(), self._stream())
         self._raise(rc, "emc2_bridge_run")
@@ -523,7 +524,7 @@ class Bridge:
             arr(*[t.data_ptr() for t in vox["mean"]]),
             arr(*[t.data_ptr() for t in pv]) if pv is not None else None,
             (ctypes.c_int32 * 2)(*cap), vox["num_voxels"].data_ptr(), _ptr(vox["bev"]),
-            pg["uvd"].data_ptr(), pg["vis_mask"].data_ptr(), pg["cam"].data_ptr(), pg["gathered"].data_ptr(),
+            pg["uvd"].data_ptr(), pg["vis_mask"].data_ptr(), pg["cam"].data_ptr(), _ptr(pg.get("gathered")),
             rd["expert"].data_ptr(), rd["offsets"].data_ptr(), rd["perm"].data_ptr(),
             rd["points_out"].data_ptr(), rd["feat_out"].data_ptr(),
             h_offsets.data_ptr() if h_offsets is not None else None,

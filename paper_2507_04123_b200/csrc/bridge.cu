@@ -325,8 +325,8 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
     if (rc == EMC2_OK && B > 0) {
         // The checks of emc2_project_gather and emc2_route_dispatch, then one pass over the rows.
         if (!d_offsets) rc2 = EMC2_ERR_INVALID_ARG;
-        else if (N > 0 && (!d_points || !d_proj || !d_feat || !d_uvd || !d_vis_mask || !d_cam || !d_gathered ||
-                           !d_expert || !d_perm || !d_points_out || !d_feat_out))
+        else if (N > 0 && (!d_points || !d_proj || !d_feat || !d_uvd || !d_vis_mask || !d_cam ||
+                           !d_expert || !d_perm || !d_points_out || !d_feat_out))   // d_gathered may be null
             rc2 = EMC2_ERR_INVALID_ARG;
         else if (!aligned16(d_points) || !aligned16(d_proj) || !aligned16(d_feat) || !aligned16(d_gathered) ||
                  !aligned16(d_feat_out))

@@ -264,7 +264,9 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) gather_scatter_
         const int r = i / C, c = i - r * C;
         pdst[(size_t)sdest[r] * C + c] = __ldg(psrc + i);
     }
-    // Feature rows: 16 rows x Cf/4 columns of threads; blended once, stored at both places.
+    // Feature rows: 16 rows x Cf/4 columns of threads; blended once, stored at both places (the
+    // rows in point order only if the caller wants them).
+    const bool keep = a.gathered != nullptr;
     float4* out = a.gathered + g0 * cf4;
     float4* fdst = a.feat_out + f0 * cf4;
     const uint32_t dyv = (uint32_t)a.Wf * cf4;
@@ -275,7 +277,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) gather_scatter_
             const int r = r0 + 16 * j;
             if (r >= npts) break;
             const float4 o = gather_column(a.feat, srow[r], c, (uint32_t)CF4, dyv);
-            __stcs(out + r * CF4 + c, o);
+            if (keep) __stcs(out + r * CF4 + c, o);
             __stcs(fdst + (size_t)sdest[r] * CF4 + c, o);
         }
     } else {
@@ -283,7 +285,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) gather_scatter_
         for (int i = t; i < items; i += blockDim.x) {
             const int r = i / cf4, c = i - r * cf4;
             const float4 o = gather_column(a.feat, srow[r], c, (uint32_t)cf4, dyv);
-            __stcs(out + i, o);
+            if (keep) __stcs(out + i, o);
             __stcs(fdst + (size_t)sdest[r] * cf4 + c, o);
         }
     }

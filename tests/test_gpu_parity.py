@@ -85,6 +85,25 @@ def test_one_call_on_a_side_stream_of_the_caller(b200, oracle):
     br.close()
 
 
+def test_one_call_without_the_rows_in_point_order(b200, oracle):
+    w = gen.NUSCENES.with_shape(2, 30001)
+    batch = gen.make_batch(w)
+    ref = oracle.bridge(w, batch)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    kept = bufs["pg"]["gathered"]
+    kept.fill_(7.0)
+    bufs["rd"]["feat_out"].fill_(-1.0)
+    bufs["pg"]["gathered"] = None
+    br.run(d["points"], d["proj"], d["feat"], bufs)
+    br.status()
+    assert bool((kept == 7.0).all())                 # not written
+    bufs["pg"]["gathered"] = torch.from_numpy(ref["gathered"]).cuda()   # everything else as always
+    compare_bridge(w, ref, bufs)
+    br.close()
+
+
 def test_one_call_from_host_buffers(b200, oracle):
     # pinned and pageable host memory; results come back into host tensors without a sync by the library
     w = gen.NUSCENES.with_shape(2, 20000)
