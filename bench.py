@@ -237,6 +237,13 @@ def run_ours(args, w):
     B, N = w.B, w.N
     frames = sharding.frames_for_rank(rank, world, B)      # every rank owns its own frames
     batch = gen.make_batch(w, frames=frames, feature_frames=args.feature_frames)
+    if args.point_order == "azimuth":
+        # Context only: the generators shuffle the points of a frame; a spinning LiDAR delivers them in
+        # firing order.  Sorting by azimuth (then range) stands in for that.
+        pts = batch["points"]
+        for b in range(pts.shape[0]):
+            key = np.lexsort((np.hypot(pts[b, :, 0], pts[b, :, 1]), np.arctan2(pts[b, :, 1], pts[b, :, 0])))
+            pts[b] = pts[b][key]
     host = {k: torch.from_numpy(v).pin_memory() for k, v in batch.items()}
     d = {k: v.to(dev, non_blocking=True) for k, v in host.items()}
     sync = lambda: torch.cuda.synchronize(dev)
@@ -414,7 +421,8 @@ def run_ours(args, w):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "frames_per_step_per_gpu": B, "points_per_frame": N, "point_floats": w.C,
-                   "cameras": w.K, "feat_c": w.feat_c, "parallelism": f"replicas x{world} (frames sharded, no collective)",
+                   "cameras": w.K, "feat_c": w.feat_c, "point_order": args.point_order,
+                   "parallelism": f"replicas x{world} (frames sharded, no collective)",
                    "l2": "inputs and outputs of a step exceed L2 (no flush)" if abytes["total"] > 2 * L2_BYTES
                          else "working set fits in L2 (latency-bound workload, no flush)"},
         "mpoints_per_s": fps * N / 1e6,
@@ -575,6 +583,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--occlusion", action="store_true", help="also time emc2_occlusion (depth-buffer test)")
+    ap.add_argument("--point-order", choices=["shuffled", "azimuth"], default="shuffled",
+                    help="order of the points inside a frame (default: the generators' shuffled order)")
     ap.add_argument("--dispatch-only", action="store_true",
                     help="also time the one-call step without the feature rows in point order (d_gathered = NULL)")
     ap.add_argument("--graph", action="store_true", help="also time the one-call step replayed from a CUDA graph")
