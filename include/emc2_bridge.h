@@ -175,7 +175,8 @@ int emc2_bridge_run(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_
  * buffers d_points, d_proj, d_feat, then emc2_bridge_run on them with the same outputs, then the
  * copies of d_offsets [B, E+1] and d_num_voxels [2] into h_offsets and h_num_voxels (either may be
  * NULL: not copied).  Nothing is synchronised: the host buffers must stay valid and unchanged until
- * the stream has passed the call; the copies are asynchronous only for page-locked host memory.  A
+ * the stream has passed the call; the copies are asynchronous only for page-locked host memory
+ * (which stream capture requires).  A
  * caller who alternates between two handles, streams and buffer sets overlaps one frame's copies with
  * the other's kernels. */
 int emc2_bridge_run_host(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* h_points, const float* h_proj,
