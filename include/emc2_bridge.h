@@ -54,7 +54,9 @@ typedef enum {
     EMC2_ERR_TIMEOUT = -5,     /* reserved: a bounded device-side wait gave up.  No kernel of this library
                                   spins on another CTA (the only grid-wide waits are the barriers of
                                   cooperative launches), so it is never returned at present */
-    EMC2_ERR_INTERNAL = -6,
+    EMC2_ERR_INTERNAL = -6,    /* from emc2_bridge_status: a call found the handle's scratch in use (two
+                                  calls on one handle at once); that call's voxel outputs are void and the
+                                  handle should be destroyed */
     EMC2_ERR_TOO_LARGE = -7    /* the call needs more scratch than a fixed-size scratch area holds */
 } emc2_status_t;
 

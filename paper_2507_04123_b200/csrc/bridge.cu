@@ -161,6 +161,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         const uint64_t per_group = d.mode == MODE_BITMAP ? kBitmapGroupCells : kTableGroupCells;
         d.ngroups = (uint32_t)((total_cells + per_group - 1) / per_group);
         d.max_ovf = d.cap > 0 ? (uint32_t)(maxpts / ((size_t)d.cap + 1) + 1) : 0;
+        d.max_list = (uint32_t)maxpts;
         o_store[s] = plan.take((size_t)d.ngroups * 1024);
         o_flag[s] = plan.take((size_t)d.ngroups * sizeof(int4));
         o_acc[s] = plan.take(maxpts * 2 * sizeof(float4));
@@ -502,6 +503,7 @@ int emc2_bridge_status(emc2_bridge_t* h, void* cuda_stream) {
     if (word & 2) return EMC2_ERR_TIMEOUT;
     if (word & 1) return EMC2_ERR_CAPACITY;
     if (word & 4) return EMC2_ERR_INVALID_ARG;
+    if (word & 8) return EMC2_ERR_INTERNAL;
     return EMC2_OK;
 }
 

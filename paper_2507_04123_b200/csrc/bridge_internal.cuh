@@ -86,6 +86,7 @@ struct ScaleDev {
     uint32_t cells;         // cells per frame
     uint32_t ngroups;       // 1 KB groups of `store` for the largest batch
     uint32_t max_ovf;       // most cells that can exceed the cap
+    uint32_t max_list;      // entries of acc / cell_list / ovf_list: the most points of a call
     uint32_t* store;        // bitmap: {bits, rank} per 32 cells; table: {count, rank, over-cap rank, -} per cell;
                             // bits / counts are zero between calls
     int4* group_info;       // [ngroups] {voxels, cells over the cap, their points} before the group in its

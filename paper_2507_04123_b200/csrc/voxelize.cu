@@ -38,6 +38,7 @@ namespace emc2 {
 namespace {
 
 constexpr int kStatusCapacity = 1;
+constexpr int kStatusDirtyStore = 8;   // the cell store held more than one call's points can set
 constexpr int kPtsPerThread = 2;                      // independent points per thread (memory-level parallelism)
 constexpr int kBigTile = kThreads * kPtsPerThread;    // points per CTA in the two per-point passes
 constexpr int kOvfBlocks = 296;                       // CTAs of vox_finalize that serve cells over the cap
@@ -165,7 +166,7 @@ __device__ __forceinline__ void sector_stats(const ScaleDev& g, const Sector& s,
 // any group's first cell computable from three small records.  Phase 2 then hands the groups out
 // round-robin, so that densely occupied regions are spread over all warps, writes the ranks into
 // the store and lists the occupied cell ids in rank order.  The loops have no CTA barrier.
-__global__ void __launch_bounds__(kThreads) vox_scan_kernel(ScanArgs a) {
+__global__ void __launch_bounds__(kThreads, 6) vox_scan_kernel(ScanArgs a) {
     constexpr int kWarps = kThreads / 32;
     __shared__ int sm[kWarps][3];
     __shared__ int wtot[kWarps][3];
@@ -237,11 +238,17 @@ __global__ void __launch_bounds__(kThreads) vox_scan_kernel(ScanArgs a) {
     }
     __syncthreads();
     const int tot0 = sm[0][0];
+    // More voxels, cells over the cap or points in them than a call's points allow: the store was not
+    // all zero when the call began (two calls on one handle at once).  Nothing is ranked or listed
+    // then; the scale reports no voxels and the handle's status becomes an internal error.
+    const bool dirty = (uint32_t)tot0 > g.max_list || (uint32_t)sm[0][1] > g.max_ovf || (uint32_t)sm[0][2] > g.max_list;
     if (cta == 0 && t == 0) {
-        g.totals[0] = sm[0][0]; g.totals[1] = sm[0][1]; g.totals[2] = sm[0][2];
-        a.num_voxels[sc] = tot0;
-        if (tot0 > a.capacity[sc]) atomicOr(a.status, kStatusCapacity);
+        g.totals[0] = dirty ? 0 : sm[0][0]; g.totals[1] = dirty ? 0 : sm[0][1]; g.totals[2] = dirty ? 0 : sm[0][2];
+        a.num_voxels[sc] = dirty ? 0 : tot0;
+        if (dirty) atomicOr(a.status, kStatusDirtyStore);
+        else if (tot0 > a.capacity[sc]) atomicOr(a.status, kStatusCapacity);
     }
+    if (dirty) return;
     // Clear the accumulators of the voxels found (two 16-byte halves per voxel).
     {
         const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -365,8 +372,11 @@ vox_accum_kernel(const float* __restrict__ pts, long long total, int N, AccumArg
             if (s.j >= 0) {
                 // Which of this cell's points survive the cap is decided per cell in
                 // vox_finalize_kernel, which also writes their point_voxel entries.
-                const int tk = atomicAdd(&g.ovf_cursor[(size_t)s.j * kCursorStride], 1);
-                g.ovf_list[g.ovf_off[s.j] + tk] = (int)(g0 + t);
+                if ((uint32_t)s.j < g.max_ovf) {      // always, unless the store was dirty
+                    const int tk = atomicAdd(&g.ovf_cursor[(size_t)s.j * kCursorStride], 1);
+                    const uint32_t pos = (uint32_t)(g.ovf_off[s.j] + tk);
+                    if (pos < g.max_list) g.ovf_list[pos] = (int)(g0 + t);
+                }
                 continue;
             }
             if (pv) pv[g0 + t] = s.m;
