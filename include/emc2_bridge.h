@@ -238,7 +238,8 @@ int emc2_rulebook(emc2_bridge_t* bridge, int32_t scale, int32_t capacity, const 
  * d_gathered [B, N, Cf].  Rows past min(*d_num_voxels, capacity) are left untouched.  Concatenating
  * [d_mean row | d_vox_img row] gives the fused voxel feature; the library leaves that to the consumer.
  * Enqueues three kernels on `cuda_stream`; uses handle scratch, so calls on one handle must be
- * ordered. */
+ * ordered.  d_counts that add up to more than B * N (not this batch's counts) make
+ * EMC2_ERR_INVALID_ARG sticky and nothing is written. */
 int emc2_voxel_image(emc2_bridge_t* bridge, int32_t B, int32_t N, int32_t capacity, const int32_t* d_point_voxel,
                      const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
                      const float* d_gathered, float* d_vox_img, int32_t* d_vox_img_count, void* cuda_stream);

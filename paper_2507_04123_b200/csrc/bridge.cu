@@ -176,7 +176,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     const size_t o_vif_cursor = plan.take(maxpts * sizeof(int));
     const size_t o_vif_list = plan.take(maxpts * sizeof(int));
     const size_t o_vif_recs = plan.take(maxpts * sizeof(uint4));
-    const size_t o_vif_part = plan.take((size_t)h->vif_scan_blocks * sizeof(int));
+    const size_t o_vif_part = plan.take(((size_t)h->vif_scan_blocks + 1) * sizeof(int));
     const size_t rb_tiles = (maxpts + kTile - 1) / kTile;
     const size_t o_rb_bits = plan.take(maxpts * sizeof(uint32_t));
     const size_t o_rb_counts = plan.take(27 * rb_tiles * sizeof(int));

@@ -40,6 +40,8 @@ struct VifArgs {
     int* list;                  // [total] point indices; bitwise complement for points no camera sees
     uint4* recs;                // [total] vif_sample: tap record of every listed point, in list order
     int* part;                  // [gridDim.x]
+    int* bad;                   // set by vif_scan when counts[] add up to more than there are points
+    int* status;
     long long total;
     int capacity, cf4;
 };
@@ -57,56 +59,77 @@ __global__ void __launch_bounds__(kThreads) vif_scan_kernel(VifArgs a) {
     const int per = (int)((M + nthreads - 1) / nthreads);
     const long long lo64 = ((long long)blockIdx.x * kThreads + t) * per;
     const int lo = (int)min((long long)M, lo64), hi = (int)min((long long)M, lo64 + per);
+    // Sums saturate at one more than the points of the call (at most 2^24 + 1): they cannot wrap, and
+    // counts[] that add up to more than the points are still seen as such.
+    const int limit = (int)min(a.total, (long long)1 << 24) + 1;
+    auto count_of = [&](int m) { return min(max(a.counts[m], 0), limit); };
     int sum = 0;
-    for (int m = lo; m < hi; ++m) sum += a.counts[m];
+    for (int m = lo; m < hi; ++m) sum = min(sum + count_of(m), limit);
     int inc = sum;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
         const int y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-        if (lane >= d) inc += y;
+        if (lane >= d) inc = min(inc + y, limit);
     }
     if (lane == 31) wsum[warp] = inc;
     __syncthreads();
     int before = 0, cta_total = 0;
     for (int w = 0; w < kThreads / 32; ++w) {
-        if (w < warp) before += wsum[w];
-        cta_total += wsum[w];
+        if (w < warp) before = min(before + wsum[w], limit);
+        cta_total = min(cta_total + wsum[w], limit);
     }
     if (t == 0) a.part[blockIdx.x] = cta_total;
     grid.sync();
     if (warp == 0) {
         int v = 0;
-        for (int c = lane; c < (int)blockIdx.x; c += 32) v += a.part[c];
-        v = warp_sum(v);
+        for (int c = lane; c < (int)blockIdx.x; c += 32) v = min(v + a.part[c], limit);
+        v = min(warp_sum(v), limit);                      // 32 terms of at most 2^24 + 1
         if (lane == 0) s_base = v;
     }
     __syncthreads();
-    int run = s_base + before + inc - sum;
+    // counts[] that add up to more than the points of the call are not the voxelizer's counts for this
+    // batch: the lists would not fit the list array, so the later kernels do nothing.
+    if (blockIdx.x == gridDim.x - 1 && t == 0) {
+        const int inconsistent = (long long)s_base + cta_total > a.total ? 1 : 0;
+        *a.bad = inconsistent;
+        if (inconsistent) atomicOr(a.status, 4);
+    }
+    int run = min(s_base + before, limit) + inc - sum;      // exact whenever the counts are consistent
     for (int m = lo; m < hi; ++m) {
         a.start[m] = run;
         a.cursor[m] = 0;
-        run += a.counts[m];
+        run = min(run + count_of(m), limit);
     }
 }
 
 __global__ void __launch_bounds__(kThreads) vif_fill_kernel(VifArgs a) {
+    if (*a.bad) return;
     const int M = voxels_in_use(a);
     for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < a.total; i += (long long)gridDim.x * kThreads) {
         const int m = a.pv[i];
         if (m < 0 || m >= M) continue;
-        const int pos = a.start[m] + atomicAdd(&a.cursor[m], 1);
+        // What goes into the list first (its loads do not wait for the ticket), then the ticket.
+        int entry = 0;
+        uint4 rec = make_uint4(kZeroRow, 0u, 0u, 0u);
         if (a.vis) {
-            a.list[pos] = a.vis[i] ? (int)i : ~(int)i;
+            entry = a.vis[i] ? (int)i : ~(int)i;
         } else {                                        // rows will be blended from the maps: keep the taps
-            a.recs[pos] = tap_record((int)(i / a.N), (int)a.cam[i], a.uvd[3 * i], a.uvd[3 * i + 1], a.K, a.Hf, a.Wf,
-                                     a.cf4, a.inv_stride, a.offset);
+            rec = tap_record((int)(i / a.N), (int)a.cam[i], a.uvd[3 * i], a.uvd[3 * i + 1], a.K, a.Hf, a.Wf, a.cf4,
+                             a.inv_stride, a.offset);
         }
+        const int pos = a.start[m] + atomicAdd(&a.cursor[m], 1);
+        // Inside the list whenever counts[] are the kept-point counts of pv[] (the voxelizer's outputs
+        // for this batch); anything else must not index out of range.
+        if ((unsigned)pos >= (unsigned)a.total) continue;
+        if (a.vis) a.list[pos] = entry;
+        else a.recs[pos] = rec;
     }
 }
 
 // CF4 > 0: Cf/4 known at compile time, blockDim.x == 16 * CF4.  CF4 == 0: any Cf, 256 threads.
 template <int CF4>
 __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_mean_kernel(VifArgs a) {
+    if (*a.bad) return;
     const int M = voxels_in_use(a);
     const int cf4 = CF4 > 0 ? CF4 : a.cf4;
     const int rows = (int)blockDim.x / cf4;                  // voxels a CTA handles at a time
@@ -167,6 +190,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_mean_kernel
 // [points, Cf] buffer is neither written nor read.  Same thread layout as vif_mean.
 template <int CF4>
 __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_sample_kernel(VifArgs a) {
+    if (*a.bad) return;
     const int M = voxels_in_use(a);
     const int cf4 = CF4 > 0 ? CF4 : a.cf4;
     const int rows = (int)blockDim.x / cf4;
@@ -252,6 +276,8 @@ int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t
     a.vox_img = reinterpret_cast<float4*>(d_vox_img); a.vox_cnt = d_vox_img_count;
     a.start = h->d_vif_start; a.cursor = h->d_vif_cursor; a.list = h->d_vif_list; a.part = h->d_vif_part;
     a.recs = h->d_vif_recs;
+    a.bad = h->d_vif_part + h->vif_scan_blocks;
+    a.status = h->d_status;
     a.total = (long long)B * N;
     a.capacity = (int)min((long long)capacity, a.total);   // a voxel holds at least one point
     a.cf4 = cfg.feat_c / 4;

@@ -258,6 +258,33 @@ def test_image_features_per_voxel(b200, oracle, cid, B, N):
     br.close()
 
 
+def test_per_voxel_fusion_rejects_counts_of_another_batch(b200, oracle):
+    # counts that add up to more than the points would make the per-voxel lists overrun their array:
+    # the scan sees it, nothing is written and the status says so
+    w = gen.KITTI.with_shape(1, 20_000)
+    batch = gen.make_batch(w)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    br.status()
+    good = br.voxel_image(bufs["vox"], 0, bufs["pg"]["vis_mask"], bufs["pg"]["gathered"])
+    br.status()
+    wrong = {k: v for k, v in bufs["vox"].items()}
+    wrong["counts"] = [torch.full_like(bufs["vox"]["counts"][0], 1 << 30), bufs["vox"]["counts"][1]]
+    out = {"vox_img": torch.full_like(good["vox_img"], 3.0), "vox_img_count": torch.full_like(good["vox_img_count"], -5)}
+    br.voxel_image(wrong, 0, bufs["pg"]["vis_mask"], bufs["pg"]["gathered"], out)
+    assert br.status(raise_on_error=False) == b200.bridge.EMC2_ERR_INVALID_ARG
+    assert bool((out["vox_img"] == 3.0).all()) and bool((out["vox_img_count"] == -5).all())
+    br.voxel_image_sampled(wrong, 0, bufs["pg"]["uvd"], bufs["pg"]["cam"], d["feat"], out)
+    assert br.status(raise_on_error=False) == b200.bridge.EMC2_ERR_INVALID_ARG
+    assert bool((out["vox_img"] == 3.0).all())
+    again = br.voxel_image(bufs["vox"], 0, bufs["pg"]["vis_mask"], bufs["pg"]["gathered"])   # and it recovers
+    br.status()
+    M = int(bufs["vox"]["num_voxels"][0].item())             # rows past the voxels found are not written
+    assert torch.equal(again["vox_img_count"][:M], good["vox_img_count"][:M])
+    br.close()
+
+
 @pytest.mark.parametrize("cid,B,N", [(2, 2, 60_000), (1, 3, 33_333), (3, 1, 150_000), (0, 1, 16_384), (2, 1, 1)])
 def test_sparse_convolution_rulebook(b200, oracle, cid, B, N):
     w = gen.workload(cid).with_shape(B, N)
