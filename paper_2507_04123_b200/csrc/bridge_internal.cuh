@@ -259,7 +259,7 @@ __device__ __forceinline__ float4 blend(const float4& f00, const float4& f01, co
 __device__ __forceinline__ uint4 tap_record(int b, int cam, float u, float v, int K, int Hf, int Wf, int cf4,
                                             float inv_stride, float offset) {
     uint4 rec = make_uint4(kZeroRow, 0u, 0u, 0u);
-    if (cam >= 0) {
+    if (cam >= 0 && cam < K) {
         // Texel coordinates: one fp32 subtraction, then an exact scaling (the stride is a power of
         // two).  Taps are clamped to the map on every side.
         const float fx = __fsub_rn(u, offset) * inv_stride, fy = __fsub_rn(v, offset) * inv_stride;

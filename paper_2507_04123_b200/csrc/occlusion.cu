@@ -31,7 +31,9 @@ __device__ __forceinline__ size_t cell_and_depth(const OcclArgs& a, const float4
     const float t1 = __fmaf_rn(p1.x, x, __fmaf_rn(p1.y, y, __fmaf_rn(p1.z, z, p1.w)));
     const float u = __fdiv_rn(t0, t2), v = __fdiv_rn(t1, t2);
     // The cell size is a power of two, so the scaling is exact.
-    const int cx = min((int)floorf(u * a.inv_cell), a.Wz - 1), cy = min((int)floorf(v * a.inv_cell), a.Hz - 1);
+    // Inside the buffer for every pixel of the image; clamped, so that a mask that is not this batch's
+    // cannot index outside it.
+    const int cx = max(min((int)floorf(u * a.inv_cell), a.Wz - 1), 0), cy = max(min((int)floorf(v * a.inv_cell), a.Hz - 1), 0);
     depth = t2;
     return (((size_t)b * a.K + k) * a.Hz + cy) * a.Wz + cx;
 }
@@ -40,7 +42,7 @@ template <int C, bool TEST>
 __global__ void __launch_bounds__(kThreads) occl_kernel(const __grid_constant__ OcclArgs a) {
     const long long i = (long long)blockIdx.x * kThreads + threadIdx.x;
     if (i >= a.total) return;
-    unsigned m = a.vis[i];
+    unsigned m = a.vis[i] & ((1u << a.K) - 1u);            // cameras the handle has
     unsigned occ = 0;
     if (m) {
         const int b = (int)(i / a.N);
