@@ -81,16 +81,17 @@ def distinct_texels(w, pg):
     uvd, cam = pg["uvd"], pg["cam"]
     B, N = cam.shape
     vis = cam >= 0
-    fx = (uvd[..., 0] / w.feat_stride)[vis]
-    fy = (uvd[..., 1] / w.feat_stride)[vis]
+    off = float(getattr(w, "feat_offset", 0.0))
+    fx = ((uvd[..., 0] - off) / w.feat_stride)[vis]
+    fy = ((uvd[..., 1] - off) / w.feat_stride)[vis]
     b = torch.arange(B, device=cam.device)[:, None].expand(B, N)[vis].long()
     k = cam[vis].long()
     x0, y0 = fx.floor().long(), fy.floor().long()
     keys = []
     for dy in (0, 1):
         for dx in (0, 1):
-            x = (x0 + dx).clamp(max=w.feat_w - 1)
-            y = (y0 + dy).clamp(max=w.feat_h - 1)
+            x = (x0 + dx).clamp(min=0, max=w.feat_w - 1)
+            y = (y0 + dy).clamp(min=0, max=w.feat_h - 1)
             keys.append(((b * w.K + k) * w.feat_h + y) * w.feat_w + x)
     return int(torch.unique(torch.cat(keys)).numel())
 
