@@ -347,6 +347,27 @@ const char* emc2_bridge_kernel_name(int kind);
 int emc2_bridge_profile_enable(emc2_bridge_t* bridge, int enable);
 int emc2_bridge_profile_read(emc2_bridge_t* bridge, int64_t* launches, double* ms, int reset);
 
+/* With profiling enabled: the launches recorded since the last profile_read / profile_timeline, in
+ * the order they were enqueued, each with the device time at which it began and ended, in
+ * milliseconds after the first of them began (events on the launching streams, so launches on
+ * the side stream of emc2_bridge_run show where they ran beside the others).  Fills at most
+ * `capacity` entries of the HOST arrays kinds / start_ms / end_ms, returns the number filled (or a
+ * negative status) and consumes the records like emc2_bridge_profile_read. */
+int emc2_bridge_profile_timeline(emc2_bridge_t* bridge, int32_t* kinds, float* start_ms, float* end_ms,
+                                 int32_t capacity);
+
+/* Choice between implementations that produce the same outputs (measurement aid, no paper
+ * counterpart; the defaults are the measured winners).  Returns EMC2_ERR_INVALID_ARG for an unknown
+ * knob or a value outside its range. */
+typedef enum {
+    EMC2_TUNE_ROW_STORE = 0,    /* how the one-call path stores feature rows: 0 = 128-bit stores from
+                                   registers; 1 = rows staged in shared memory, ordered by expert, and written
+                                   with bulk asynchronous copies (cp.async.bulk), both destinations; 2 = bulk
+                                   copies for the dispatched rows only */
+    EMC2_TUNE_KNOBS
+} emc2_tuning_t;
+int emc2_bridge_set_tuning(emc2_bridge_t* bridge, int32_t knob, int32_t value);
+
 #ifdef __cplusplus
 }
 #endif

@@ -36,7 +36,12 @@ ABI_SYMBOLS = (
     "emc2_bridge_run", "emc2_bridge_run_host", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
     "emc2_features_channels_last",
     "emc2_voxel_image", "emc2_voxel_image_sampled", "emc2_occlusion", "emc2_rulebook",
+    "emc2_bridge_set_tuning", "emc2_bridge_profile_timeline",
 )
+
+# emc2_tuning_t
+TUNE_ROW_STORE = 0
+TUNE_NAMES = {"row_store": TUNE_ROW_STORE}
 
 
 class Emc2Grid(ctypes.Structure):
@@ -93,6 +98,8 @@ def load_library() -> ctypes.CDLL:
     lib.emc2_features_channels_last.argtypes = [vp, i32, vp, vp, vp]
     lib.emc2_scene_route.argtypes = [vp, i32, vp, P(ctypes.c_uint8), i32, vp, vp]
     lib.emc2_bridge_set_overlap.argtypes = [vp, ctypes.c_int]
+    lib.emc2_bridge_set_tuning.argtypes = [vp, i32, i32]
+    lib.emc2_bridge_profile_timeline.argtypes = [vp, P(i32), P(ctypes.c_float), P(ctypes.c_float), i32]
     lib.emc2_bridge_destroy.argtypes = [vp]
     lib.emc2_status_string.argtypes = [ctypes.c_int]
     lib.emc2_status_string.restype = ctypes.c_char_p
@@ -427,6 +434,11 @@ class Bridge:
         """emc2_bridge_set_overlap: stage 1 of :meth:`run` beside stages 2 - 4 (default) or after them."""
         self._raise(self.lib.emc2_bridge_set_overlap(self._h, int(enable)), "emc2_bridge_set_overlap")
 
+    def set_tuning(self, knob, value: int) -> None:
+        """emc2_bridge_set_tuning: ``knob`` is an emc2_tuning_t value or its name in TUNE_NAMES."""
+        k = TUNE_NAMES[knob] if isinstance(knob, str) else int(knob)
+        self._raise(self.lib.emc2_bridge_set_tuning(self._h, k, int(value)), "emc2_bridge_set_tuning")
+
     def status(self, raise_on_error: bool = True) -> int:
         """emc2_bridge_status: waits for the current stream, returns the sticky device status."""
         rc = self.lib.emc2_bridge_status(self._h, self._stream())
@@ -547,3 +559,14 @@ class Bridge:
         self._raise(self.lib.emc2_bridge_profile_read(self._h, launches, ms, int(reset)),
                     "emc2_bridge_profile_read")
         return {name: (int(launches[k]), float(ms[k])) for k, name in enumerate(self.kernel_names())}
+
+    def profile_timeline(self, capacity: int = 4096) -> List[Tuple[str, float, float]]:
+        """emc2_bridge_profile_timeline: (kernel, start ms, end ms) of the launches recorded since the last read."""
+        kinds = (ctypes.c_int32 * capacity)()
+        t0 = (ctypes.c_float * capacity)()
+        t1 = (ctypes.c_float * capacity)()
+        n = self.lib.emc2_bridge_profile_timeline(self._h, kinds, t0, t1, capacity)
+        if n < 0:
+            self._raise(n, "emc2_bridge_profile_timeline")
+        names = self.kernel_names()
+        return [(names[kinds[i]], float(t0[i]), float(t1[i])) for i in range(n)]

@@ -8,7 +8,7 @@
 namespace emc2 {
 
 static const char* const kKernelNames[K_KINDS] = {
-    "vox_mark", "vox_scan", "vox_accum", "vox_finalize",
+    "vox_mark", "vox_count", "vox_prefix", "vox_rank", "vox_accum", "vox_finalize",
     "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features",
     "vif_scan", "vif_fill", "vif_mean", "vif_sample", "occl_fill", "occl_splat", "occl_test",
     "channels_last", "rb_mark", "rb_count", "rb_scan", "rb_fill", "rb_clear"};
@@ -139,8 +139,8 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     for (int t = 0; t < EMC2_MAX_THRESHOLDS; ++t)
         h->thr2[t] = t < c.num_thresholds ? c.thresholds[t] * c.thresholds[t] : 0.0f;
 
-    h->scan_blocks = voxel_scan_max_blocks();
-    if (h->scan_blocks < 2) { delete h; return EMC2_ERR_CUDA; }
+    if (cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, config->device) != cudaSuccess ||
+        h->num_sms < 1) { delete h; return EMC2_ERR_CUDA; }
     h->vif_scan_blocks = voxel_image_scan_max_blocks();
     if (h->vif_scan_blocks < 1) { delete h; return EMC2_ERR_CUDA; }
 
@@ -171,7 +171,10 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         o_ovf[s][4] = d.cap > 0 ? plan.take((size_t)d.max_ovf * kCursorStride * sizeof(int)) : 0;
         o_tot[s] = plan.take(4 * sizeof(int));
     }
-    const size_t o_part = plan.take((size_t)h->scan_blocks * 3 * sizeof(int));
+    // The rank scan gives a CTA 32 groups of one scale.
+    const size_t scan_ctas = (size_t)(h->scale[0].ngroups + 31) / 32 + (size_t)(h->scale[1].ngroups + 31) / 32;
+    const size_t o_part = plan.take(scan_ctas * 3 * sizeof(int));
+    const size_t o_pbase = plan.take(scan_ctas * 3 * sizeof(int));
     const size_t o_vif_start = plan.take(maxpts * sizeof(int));
     const size_t o_vif_cursor = plan.take(maxpts * sizeof(int));
     const size_t o_vif_list = plan.take(maxpts * sizeof(int));
@@ -181,7 +184,6 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     const size_t o_rb_bits = plan.take(maxpts * sizeof(uint32_t));
     const size_t o_rb_counts = plan.take(27 * rb_tiles * sizeof(int));
     const size_t o_rb_base = plan.take((27 * rb_tiles + 27) * sizeof(int));
-    const size_t o_wofs = plan.take((size_t)h->scan_blocks * (kThreads / 32) * 3 * sizeof(int));
     h->max_tiles = (c.max_points + kTile - 1) / kTile;
     const size_t tile_ints = (size_t)c.max_batch * h->max_tiles * c.num_experts;
     const size_t o_tc = plan.take(tile_ints * sizeof(int));
@@ -208,7 +210,8 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
         d.ovf_cursor = d.cap > 0 ? reinterpret_cast<int*>(base + o_ovf[s][4]) : nullptr;
         d.totals = reinterpret_cast<int*>(base + o_tot[s]);
     }
-    h->d_scan_part = reinterpret_cast<int*>(base + o_part);
+    h->d_scan_tot = reinterpret_cast<int*>(base + o_part);
+    h->d_scan_base = reinterpret_cast<int*>(base + o_pbase);
     h->d_vif_start = reinterpret_cast<int*>(base + o_vif_start);
     h->d_vif_cursor = reinterpret_cast<int*>(base + o_vif_cursor);
     h->d_vif_list = reinterpret_cast<int*>(base + o_vif_list);
@@ -217,7 +220,6 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     h->d_rb_bits = reinterpret_cast<uint32_t*>(base + o_rb_bits);
     h->d_rb_counts = reinterpret_cast<int*>(base + o_rb_counts);
     h->d_rb_base = reinterpret_cast<int*>(base + o_rb_base);
-    h->d_scan_warp_ofs = reinterpret_cast<int*>(base + o_wofs);
     h->d_tile_counts = reinterpret_cast<int*>(base + o_tc);
     h->d_tile_base = reinterpret_cast<int*>(base + o_tb);
     h->d_status = reinterpret_cast<int*>(base + o_status);
@@ -311,17 +313,8 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
         if (e == cudaSuccess) e = cudaStreamWaitEvent(h->side, h->ev_fork, 0);
         if (e != cudaSuccess) return check_cuda(h, e);
     }
-    // A thinner rank scan leaves stages 2 - 4 more of each SM; it pays while the scan's streaming
-    // read of the cell stores is small beside the feature rows those stages move.
-    {
-        double store_bytes = 0.0;
-        for (int s = 0; s < 2; ++s)
-            store_bytes += (double)B * h->scale[s].cells * (h->scale[s].mode == MODE_BITMAP ? 0.25 : 16.0);
-        h->thin_scan = h->overlap && 2.0 * store_bytes < (double)B * N * h->cfg.feat_c * 4.0;
-    }
     int rc = emc2_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity, d_num_voxels,
                            d_bev, vox_st);
-    h->thin_scan = false;
     int rc2 = EMC2_OK;
     if (rc == EMC2_OK && B > 0) {
         // The checks of emc2_project_gather and emc2_route_dispatch, then one pass over the rows.
@@ -490,6 +483,14 @@ int emc2_bridge_set_overlap(emc2_bridge_t* h, int enable) {
     return EMC2_OK;
 }
 
+int emc2_bridge_set_tuning(emc2_bridge_t* h, int32_t knob, int32_t value) {
+    if (!h || knob < 0 || knob >= EMC2_TUNE_KNOBS) return EMC2_ERR_INVALID_ARG;
+    static const int kMaxValue[EMC2_TUNE_KNOBS] = {2};
+    if (value < 0 || value > kMaxValue[knob]) return EMC2_ERR_INVALID_ARG;
+    h->tune[knob] = value;
+    return EMC2_OK;
+}
+
 int emc2_bridge_status(emc2_bridge_t* h, void* cuda_stream) {
     if (!h) return EMC2_ERR_INVALID_ARG;
     DeviceGuard guard(h->cfg.device);
@@ -566,6 +567,25 @@ int emc2_bridge_profile_read(emc2_bridge_t* h, int64_t* launches, double* ms, in
         if (reset) { h->launches[k] = 0; h->ms[k] = 0.0; }
     }
     return rc;
+}
+
+int emc2_bridge_profile_timeline(emc2_bridge_t* h, int32_t* kinds, float* start_ms, float* end_ms,
+                                 int32_t capacity) {
+    if (!h || capacity < 0 || (capacity > 0 && (!kinds || !start_ms || !end_ms))) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    int n = 0, rc = EMC2_OK;
+    cudaEvent_t origin = h->recs.empty() ? nullptr : h->recs.front().a;
+    for (ProfRec& r : h->recs) {
+        float t0 = 0.f, t1 = 0.f;
+        cudaError_t e = cudaEventSynchronize(r.b);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&t0, origin, r.a);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&t1, origin, r.b);
+        if (e != cudaSuccess) rc = check_cuda(h, e);
+        else if (n < capacity) { kinds[n] = r.kind; start_ms[n] = t0; end_ms[n] = t1; ++n; }
+    }
+    for (ProfRec& r : h->recs) { h->event_pool.push_back(r.a); h->event_pool.push_back(r.b); }
+    h->recs.clear();
+    return rc != EMC2_OK ? rc : n;
 }
 
 }  // extern "C"

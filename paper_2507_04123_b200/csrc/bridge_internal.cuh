@@ -15,13 +15,14 @@ constexpr int kThreads = 256;
 constexpr int kBitmapGroupCells = 32 * 4 * 32;  // a 1 KB bitmap group: 32 sectors of four {bits, rank} pairs
 constexpr int kTableGroupCells = 32 * 2;         // a 1 KB table group: 32 sectors of two cell records
 constexpr int kMaxTableCells = 1 << 24;  // per-cell records up to 16 Mi cells per batch (256 MB)
-constexpr int kMaxScanBlocks = 1024;     // CTAs of the cooperative rank scan, at most
 constexpr int kCursorStride = 8;         // ints between list cursors: one 32-byte sector each
 
 // Kernel kinds, for the launch counters and the optional event timing.
 enum KernelKind {
     K_VOX_MARK = 0,
-    K_VOX_SCAN,
+    K_VOX_COUNT,
+    K_VOX_PREFIX,
+    K_VOX_RANK,
     K_VOX_ACCUM,
     K_VOX_FINALIZE,
     K_PROJECT_GATHER,
@@ -89,8 +90,8 @@ struct ScaleDev {
     uint32_t max_list;      // entries of acc / cell_list / ovf_list: the most points of a call
     uint32_t* store;        // bitmap: {bits, rank} per 32 cells; table: {count, rank, over-cap rank, -} per cell;
                             // bits / counts are zero between calls
-    int4* group_info;       // [ngroups] {voxels, cells over the cap, their points} before the group in its
-                            // warp's range of the rank scan, and the group's voxels (rewritten by every call)
+    int4* group_info;       // [ngroups] {voxels, cells over the cap, their points} of the group (rewritten by
+                            // every call)
     float4* acc;            // [max voxels][2] per-voxel accumulators
     uint32_t* cell_list;    // [max voxels] cell id of each unique voxel (table stores: bit 31 = over the cap)
     int* ovf_off;           // per cell over the cap j: start of its points in ovf_list
@@ -98,7 +99,7 @@ struct ScaleDev {
     uint32_t* ovf_cell;     // per cell over the cap j: its cell id
     int* ovf_vox;           // per cell over the cap j: its row m in the unique list
     int* ovf_list;          // global point indices of the points in cells over the cap
-    int* totals;            // [0] voxels, [1] cells over the cap, [2] points in cells over the cap
+    int* totals;            // [0] voxels, [1] cells over the cap, [2] points in cells over the cap, [3] store found dirty
 };
 
 // Routing tables as the kernels take them (Sec. 3.2 distance rule, per point with visibility).
@@ -124,10 +125,8 @@ struct emc2_bridge {
     int* d_status = nullptr;       // sticky device status word
     int* d_tile_counts = nullptr;  // [B, tiles per frame, E]
     int* d_tile_base = nullptr;    // same shape, exclusive bases
-    int* d_scan_part = nullptr;    // [scan_blocks][3] per-CTA totals of the voxel rank scan
-    int* d_scan_warp_ofs = nullptr;  // [scan_blocks * 8][3] per-warp offsets inside their CTA
-    int scan_blocks = 0;           // CTAs of the cooperative rank scan (all co-resident)
-    bool thin_scan = false;        // set while emc2_bridge_run enqueues stage 1 beside stages 2 - 4
+    int* d_scan_tot = nullptr;     // [CTAs of the voxel rank scan, both scales][3] per-CTA totals
+    int* d_scan_base = nullptr;    // same shape: their exclusive prefix sums inside each scale
     int* d_vif_start = nullptr;    // emc2_voxel_image: [max points] list starts, cursors, lists
     int* d_vif_cursor = nullptr;
     int* d_vif_list = nullptr;
@@ -138,6 +137,8 @@ struct emc2_bridge {
     int* d_rb_counts = nullptr;    // [27][voxel tiles] pairs per (offset, tile), and their prefix sums
     int* d_rb_base = nullptr;
     int max_tiles = 0;
+    int tune[EMC2_TUNE_KNOBS] = {0};   // emc2_bridge_set_tuning
+    int num_sms = 0;               // multiprocessors of the handle's device
     bool overlap = true;           // emc2_bridge_run puts stage 1 on `side`
     cudaStream_t side = nullptr;   // stream of stage 1 inside emc2_bridge_run
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
@@ -163,8 +164,6 @@ struct LaunchScope {
 
 int check_cuda(emc2_bridge* h, cudaError_t e);
 
-// Largest cooperative grid of the voxel rank scan on the current device (0: unsupported).
-int voxel_scan_max_blocks();
 int launch_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* const d_coords[2],
                     int32_t* const d_counts[2], float* const d_mean[2], int32_t* const d_point_voxel[2],
                     const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st);

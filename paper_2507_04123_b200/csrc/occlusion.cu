@@ -86,7 +86,7 @@ int launch_occlusion(emc2_bridge* h, int B, int N, const float* d_points, const 
     const size_t nz = (size_t)B * a.K * a.Hz * a.Wz;
     {
         LaunchScope ls(h, K_OCCL_FILL, st);
-        occl_fill_kernel<<<(unsigned)min((size_t)148 * 8, (nz + kThreads - 1) / kThreads), kThreads, 0, st>>>(d_zbuf, nz);
+        occl_fill_kernel<<<(unsigned)min((size_t)h->num_sms * 8, (nz + kThreads - 1) / kThreads), kThreads, 0, st>>>(d_zbuf, nz);
     }
     if (a.total > 0) {
         const unsigned blocks = (unsigned)((a.total + kThreads - 1) / kThreads);

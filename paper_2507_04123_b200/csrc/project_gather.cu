@@ -291,9 +291,136 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) gather_scatter_
     }
 }
 
+// ---- the same pass with the rows staged in shared memory and written by bulk asynchronous copies
+// A thread of gather_scatter_kernel issues, per 16 bytes of output, four 128-bit tap loads and two
+// 128-bit global stores; the load/store path of the SM is its busiest unit.  Here the blended
+// values go to shared memory instead, a sub-tile of 32 rows at a time (the rows of one warp of the
+// ranking phase), once in point order and once ordered by expert.  The first copy is one contiguous
+// block of `gathered`; in the second, the rows of one expert are one contiguous run of `feat_out`
+// (ranks inside a tile are stable and tile bases are prefix sums), so a sub-tile leaves as at most
+// 1 + E bulk copies (cp.async.bulk shared -> global) issued by one warp, and the global stores no
+// longer pass through the threads' load/store instructions.  Two stage buffers: the copies of one
+// sub-tile run while the next is blended.
+__device__ __forceinline__ void bulk_store(void* gdst, const void* ssrc, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 :: "l"(gdst), "r"((uint32_t)__cvta_generic_to_shared(ssrc)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Waits until at most `kPending` of this thread's bulk groups still read their shared-memory source.
+template <int kPending>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(kPending) : "memory");
+}
+// Makes this thread's earlier shared-memory writes visible to the asynchronous copy engine.
+__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// kBoth: also stage and bulk-copy the rows in point order; otherwise those are stored from registers.
+template <int C, int CF4, bool kBoth>
+__global__ void __launch_bounds__(16 * CF4) gather_scatter_bulk_kernel(const __grid_constant__ GsArgs a) {
+    constexpr int kSub = 32, kBufs = 2, kWarpsTile = kTile / 32;
+    __shared__ __align__(128) float4 stage[kBufs][kBoth ? 2 : 1][kSub * CF4];   // [buffer][expert order, point order]
+    __shared__ uint4 srow[kTile];
+    __shared__ int sdest[kTile];
+    __shared__ uint8_t spos[kTile];                       // row's place in its sub-tile when ordered by expert
+    __shared__ int wcnt[kWarpsTile][EMC2_MAX_EXPERTS];    // rows of expert k in sub-tile w
+    __shared__ int wrow[kWarpsTile][EMC2_MAX_EXPERTS];    // first feat_out row (in the frame) of that run
+    const int b = blockIdx.y, tile = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int i0 = tile * kTile;
+    const int npts = min(kTile, a.N - i0);
+    const size_t f0 = (size_t)b * a.N;
+    const size_t g0 = f0 + i0;
+
+    int e = -1, rank = 0;
+    if (t < kTile) {
+        if (t < npts) {
+            e = (int)a.expert[g0 + t];
+            const float u = a.uvd[(g0 + t) * 3], v = a.uvd[(g0 + t) * 3 + 1];
+            srow[t] = tap_record(b, (int)a.cam[g0 + t], u, v, a.K, a.Hf, a.Wf, CF4, a.inv_stride, a.offset);
+        }
+        for (int k = 0; k < a.E; ++k) {
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
+            if (e == k) rank = __popc(m & ((1u << lane) - 1u));
+            if (lane == 0) wcnt[warp][k] = __popc(m);
+        }
+    }
+    __syncthreads();
+    if (t < npts) {
+        int before = 0, below = 0;
+        for (int w = 0; w < warp; ++w) before += wcnt[w][e];
+        for (int k = 0; k < e; ++k) below += wcnt[warp][k];
+        const int d = a.tile_base[((size_t)b * a.tiles + tile) * a.E + e] + before + rank;
+        sdest[t] = d;
+        spos[t] = (uint8_t)(below + rank);
+        a.perm[f0 + d] = i0 + t;
+    }
+    if (t < kWarpsTile * a.E) {
+        const int w = t / a.E, k = t - w * a.E;
+        int before = 0;
+        for (int w2 = 0; w2 < w; ++w2) before += wcnt[w2][k];
+        wrow[w][k] = a.tile_base[((size_t)b * a.tiles + tile) * a.E + k] + before;
+    }
+    __syncthreads();
+
+    const float* psrc = a.pts + g0 * C;
+    float* pdst = a.pts_out + f0 * C;
+    for (int i = t; i < npts * C; i += blockDim.x) {
+        const int r = i / C, c = i - r * C;
+        pdst[(size_t)sdest[r] * C + c] = __ldg(psrc + i);
+    }
+
+    const bool keep = a.gathered != nullptr;
+    float4* out = a.gathered + g0 * CF4;
+    float4* fdst = a.feat_out + f0 * CF4;
+    const uint32_t dyv = (uint32_t)a.Wf * CF4;
+    const int c = t % CF4, r0 = t / CF4;
+    const int nsub = (npts + kSub - 1) / kSub;
+    for (int s = 0; s < nsub; ++s) {
+        const int buf = s & 1;
+        if (s >= kBufs) {                                 // the copies that read this buffer must have read it
+            if (warp == 0) bulk_wait_read<kBufs - 1>();
+            __syncthreads();
+        }
+        const int nr = min(kSub, npts - s * kSub);
+#pragma unroll
+        for (int jj = 0; jj < kSub / 16; ++jj) {
+            const int rl = r0 + 16 * jj;
+            if (rl < nr) {
+                const int r = s * kSub + rl;
+                const float4 o = gather_column(a.feat, srow[r], c, (uint32_t)CF4, dyv);
+                stage[buf][0][(int)spos[r] * CF4 + c] = o;
+                if (kBoth) { if (keep) stage[buf][kBoth ? 1 : 0][rl * CF4 + c] = o; }
+                else if (keep) __stcs(out + r * CF4 + c, o);
+            }
+        }
+        fence_async_shared();
+        __syncthreads();
+        if (warp == 0) {
+            if (lane < a.E) {
+                const int cnt = wcnt[s][lane];
+                int start = 0;
+                for (int k = 0; k < lane; ++k) start += wcnt[s][k];
+                if (cnt > 0)
+                    bulk_store(fdst + (size_t)wrow[s][lane] * CF4, &stage[buf][0][start * CF4], (uint32_t)cnt * CF4 * 16u);
+            } else if (kBoth && lane == 31 && keep) {
+                bulk_store(out + (size_t)s * kSub * CF4, &stage[buf][kBoth ? 1 : 0][0], (uint32_t)nr * CF4 * 16u);
+            }
+            bulk_commit();
+        }
+    }
+    if (warp == 0) bulk_wait_read<0>();                   // shared memory must outlive the copies that read it
+}
+
 template <int C>
 void launch_gs(emc2_bridge* h, const GsArgs& a, dim3 grid, cudaStream_t st) {
     LaunchScope ls(h, K_GATHER_SCATTER, st);
+    const int mode = h->tune[EMC2_TUNE_ROW_STORE];
+    if (mode == 1 && a.E < 31) {
+        if (a.cf4 == 16) { gather_scatter_bulk_kernel<C, 16, true><<<grid, 16 * 16, 0, st>>>(a); return; }
+        if (a.cf4 == 20) { gather_scatter_bulk_kernel<C, 20, true><<<grid, 16 * 20, 0, st>>>(a); return; }
+    } else if (mode == 2) {
+        if (a.cf4 == 16) { gather_scatter_bulk_kernel<C, 16, false><<<grid, 16 * 16, 0, st>>>(a); return; }
+        if (a.cf4 == 20) { gather_scatter_bulk_kernel<C, 20, false><<<grid, 16 * 20, 0, st>>>(a); return; }
+    }
     switch (a.cf4) {
         case 16: gather_scatter_kernel<C, 16><<<grid, 16 * 16, 0, st>>>(a); break;
         case 20: gather_scatter_kernel<C, 20><<<grid, 16 * 20, 0, st>>>(a); break;

@@ -292,10 +292,10 @@ int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t
     }
     {
         LaunchScope ls(h, K_VIF_FILL, st);
-        const int blocks = (int)min((long long)148 * 16, (a.total + kThreads - 1) / kThreads);
+        const int blocks = (int)min((long long)h->num_sms * 16, (a.total + kThreads - 1) / kThreads);
         vif_fill_kernel<<<blocks, kThreads, 0, st>>>(a);
     }
-    const int blocks = (int)min((long long)148 * 16, ((long long)a.capacity + 15) / 16);
+    const int blocks = (int)min((long long)h->num_sms * 16, ((long long)a.capacity + 15) / 16);
     if (d_gathered) {
         LaunchScope ls(h, K_VIF_MEAN, st);
         switch (a.cf4) {

@@ -10,11 +10,11 @@
 //
 //   vox_mark      every point marks its two cells with one fire-and-forget reduction each;
 //                 the same launch zeroes the BEV image.
-//   vox_scan      one cooperative launch: counts per 1 KB group of the store, grid barrier,
-//                 then the exclusive prefix sums (the parallel prefix-sum index search of
-//                 Sec. 3.6) are written into the rank fields and the occupied cell ids listed
-//                 in that order; accumulators are cleared and the bookkeeping of cells over the
-//                 cap is laid out.
+//   vox_count,    the rank scan, three launches: counts per 1 KB group of the store, prefix sums
+//   vox_prefix,   of the per-CTA totals, then the exclusive prefix sums (the parallel prefix-sum
+//   vox_rank      index search of Sec. 3.6) are written into the rank fields and the occupied
+//                 cell ids listed in that order; accumulators are cleared and the bookkeeping of
+//                 cells over the cap is laid out.
 //   vox_accum     every point looks its rank up, writes point_voxel and adds itself to its
 //                 voxels' accumulators with two fp32 vector reductions (offsets from the cell
 //                 corner, the other channels, the count).
@@ -28,11 +28,7 @@
 // L2 (about 10 ns each on B200), so nothing here funnels many points into a shared flag or
 // counter: the only contended words are the cells themselves.  The cost of a call follows the
 // occupied groups, not the grid volume, except for one streaming read of the store.
-#include <cooperative_groups.h>
-
 #include "bridge_internal.cuh"
-
-namespace cg = cooperative_groups;
 
 namespace emc2 {
 namespace {
@@ -41,7 +37,6 @@ constexpr int kStatusCapacity = 1;
 constexpr int kStatusDirtyStore = 8;   // the cell store held more than one call's points can set
 constexpr int kPtsPerThread = 2;                      // independent points per thread (memory-level parallelism)
 constexpr int kBigTile = kThreads * kPtsPerThread;    // points per CTA in the two per-point passes
-constexpr int kOvfBlocks = 296;                       // CTAs of vox_finalize that serve cells over the cap
 
 // Where a point's cell sits in the unique list.
 struct Slot {
@@ -127,9 +122,9 @@ struct ScanArgs {
     int capacity[2];
     int32_t* num_voxels;
     int* status;
-    int* part;                  // [gridDim.x][3] per-CTA totals
-    int* warp_ofs;              // [gridDim.x * warps][3] totals of the warps before a warp in its CTA
-    int g0;                     // CTAs [0, g0) serve scale 0, the rest scale 1
+    int* cta_tot;               // [ctas0 + ctas1][3] voxels, cells over the cap and their points per CTA
+    int* cta_base;              // same shape: exclusive prefix sums inside each scale
+    int ctas0, ctas1;           // CTAs of vox_count / vox_rank serving scale 0 and scale 1
 };
 
 // One lane owns one 32-byte sector of the store: four {bits, rank} pairs or two cell records;
@@ -160,49 +155,96 @@ __device__ __forceinline__ void sector_stats(const ScaleDev& g, const Sector& s,
     }
 }
 
-// Cooperative launch.  Phase 1: every warp owns a contiguous range of groups of one scale, CTA
-// after CTA, counts them and records, per group, its count and the running total inside the
-// warp's range.  After the grid barrier every CTA scans the CTA totals, which makes the rank of
-// any group's first cell computable from three small records.  Phase 2 then hands the groups out
-// round-robin, so that densely occupied regions are spread over all warps, writes the ranks into
-// the store and lists the occupied cell ids in rank order.  The loops have no CTA barrier.
-__global__ void __launch_bounds__(kThreads, 6) vox_scan_kernel(ScanArgs a) {
+// Writes the ranks of one group into its sector and lists its occupied cells in rank order.
+// base[] = voxels, cells over the cap and points in such cells before the group.
+__device__ __forceinline__ void rank_group(const ScaleDev& g, uint32_t grp, Sector x, const int base[3], int lane) {
+    int run[3] = {0, 0, 0}, gtot[3];
+    sector_stats(g, x, run);
+    const bool mine = run[0] > 0;
+    warp_excl_scan3(run, gtot);                   // run[] = exclusive offsets inside the group
+    if (!mine) return;
+    int m = base[0] + run[0];
+    if (g.mode == MODE_BITMAP) {
+        const uint32_t word0 = (grp * 32u + lane) * 4u;
+        const uint32_t bw[4] = {x.a.x, x.a.z, x.b.x, x.b.z};
+        uint32_t rk[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            rk[i] = (uint32_t)m;
+            uint32_t bits = bw[i];
+            while (bits) {                        // plain stores: nothing here waits on memory
+                const int bit = __ffs(bits) - 1;
+                bits &= bits - 1;
+                g.cell_list[m++] = (word0 + i) * 32u + bit;
+            }
+        }
+        x.a.y = rk[0]; x.a.w = rk[1]; x.b.y = rk[2]; x.b.w = rk[3];
+    } else {
+        int j = base[1] + run[1], off = base[2] + run[2];
+        const uint32_t cell0 = (grp * 32u + lane) * 2u;
+        x.a.y = (uint32_t)m; x.a.z = (uint32_t)j;
+        const int n0 = (int)x.a.x, n1 = (int)x.b.x;
+        const bool o0 = g.cap > 0 && n0 > g.cap, o1 = g.cap > 0 && n1 > g.cap;
+        if (o0) {
+            g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+            j += 1; off += n0;
+        }
+        if (n0 > 0) g.cell_list[m++] = cell0 | (o0 ? 0x80000000u : 0u);
+        x.b.y = (uint32_t)m; x.b.z = (uint32_t)j;
+        if (o1) {
+            g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0 + 1u; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+        }
+        if (n1 > 0) g.cell_list[m] = (cell0 + 1u) | (o1 ? 0x80000000u : 0u);
+    }
+    uint4* p = reinterpret_cast<uint4*>(g.store) + ((size_t)grp * 32 + lane) * 2;
+    p[0] = x.a;
+    p[1] = x.b;
+}
+
+// The rank scan is three plain launches, each a few memory round trips deep, so that it keeps its
+// pace when it runs beside kernels that saturate the memory system (a deep chain of dependent loads
+// stretches with the latency of every hop).  A CTA owns 32 consecutive groups of one scale, a warp
+// four of them.
+//   vox_count   streams the store once: per-group counts into group_info, per-CTA totals.
+//   vox_prefix  one CTA per scale: exclusive prefix sums of the CTA totals, the scale's totals, the
+//               number of voxels and the capacity / consistency checks.
+//   vox_rank    a warp turns its CTA's 32 group counts into group bases with one warp scan, loads
+//               only its occupied groups (all at once), writes their ranks and lists their cells in
+//               rank order: the parallel prefix-sum index search of Sec. 3.6.  Also clears the
+//               accumulators of the voxels found.
+constexpr int kGroupsPerWarp = 4;
+constexpr int kGroupsPerCta = kGroupsPerWarp * (kThreads / 32);
+static_assert(kGroupsPerCta == 32, "vox_rank_kernel scans one group count per lane");
+
+__global__ void __launch_bounds__(kThreads) vox_count_kernel(ScanArgs a) {
     constexpr int kWarps = kThreads / 32;
-    __shared__ int sm[kWarps][3];
     __shared__ int wtot[kWarps][3];
-    __shared__ int cta_base[kMaxScanBlocks][3];   // exclusive totals of the CTAs of this scale
-    cg::grid_group grid = cg::this_grid();
-    const int sc = (int)blockIdx.x >= a.g0 ? 1 : 0;
-    const int first = sc ? a.g0 : 0;
-    const int cta = (int)blockIdx.x - first;
-    const int ncta = sc ? (int)gridDim.x - a.g0 : a.g0;
+    const int sc = (int)blockIdx.x >= a.ctas0 ? 1 : 0;
+    const uint32_t cta = blockIdx.x - (sc ? a.ctas0 : 0);
     const ScaleDev& g = a.s[sc];
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const uint32_t ng = a.ngroups_used[sc];
-    const uint32_t per = max(1u, (ng + (uint32_t)(ncta * kWarps) - 1u) / (uint32_t)(ncta * kWarps));
-    const uint32_t lo = min(ng, (uint32_t)(cta * kWarps + warp) * per), hi = min(ng, lo + per);
-
-    int carry[3] = {0, 0, 0};
-    for (uint32_t grp = lo; grp < hi; grp += 4) {
-        Sector x[4];
+    const uint32_t g0 = cta * kGroupsPerCta + warp * kGroupsPerWarp;
+    Sector x[kGroupsPerWarp];
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (grp + u < hi) {                   // streaming: most of the store is empty, keep it out of L2
-                const uint4* p = reinterpret_cast<const uint4*>(g.store) + ((size_t)(grp + u) * 32 + lane) * 2;
-                x[u].a = __ldcs(p);
-                x[u].b = __ldcs(p + 1);
-            }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (grp + u >= hi) break;
-            int s[3] = {0, 0, 0};
-            sector_stats(g, x[u], s);
-#pragma unroll
-            for (int k = 0; k < 3; ++k) s[k] = warp_sum(s[k]);
-            if (lane == 0) g.group_info[grp + u] = make_int4(carry[0], carry[1], carry[2], s[0]);
-#pragma unroll
-            for (int k = 0; k < 3; ++k) carry[k] += s[k];
+    for (int u = 0; u < kGroupsPerWarp; ++u) {
+        x[u].a = x[u].b = make_uint4(0u, 0u, 0u, 0u);
+        if (g0 + u < ng) {                        // streaming: most of the store is empty, keep it out of L2
+            const uint4* p = reinterpret_cast<const uint4*>(g.store) + ((size_t)(g0 + u) * 32 + lane) * 2;
+            x[u].a = __ldcs(p);
+            x[u].b = __ldcs(p + 1);
         }
+    }
+    int carry[3] = {0, 0, 0};
+#pragma unroll
+    for (int u = 0; u < kGroupsPerWarp; ++u) {
+        int s[3] = {0, 0, 0};
+        sector_stats(g, x[u], s);
+#pragma unroll
+        for (int k = 0; k < 3; ++k) s[k] = warp_sum(s[k]);
+        if (lane == 0 && g0 + u < ng) g.group_info[g0 + u] = make_int4(s[0], s[1], s[2], 0);
+#pragma unroll
+        for (int k = 0; k < 3; ++k) carry[k] += s[k];
     }
     if (lane == 0) {
 #pragma unroll
@@ -211,101 +253,110 @@ __global__ void __launch_bounds__(kThreads, 6) vox_scan_kernel(ScanArgs a) {
     __syncthreads();
     if (t < 3) {
         int v = 0;
-        for (int w = 0; w < kWarps; ++w) {
-            a.warp_ofs[((size_t)blockIdx.x * kWarps + w) * 3 + t] = v;   // warp's offset inside its CTA
-            v += wtot[w][t];
-        }
-        a.part[blockIdx.x * 3 + t] = v;
+        for (int w = 0; w < kWarps; ++w) v += wtot[w][t];
+        a.cta_tot[(size_t)blockIdx.x * 3 + t] = v;
     }
-    grid.sync();
+}
 
-    // Exclusive scan of the CTA totals of this scale, by warp 0: each lane sums a run of CTAs.
-    if (warp == 0) {
-        const int run = (ncta + 31) / 32;
-        const int c_lo = min(ncta, lane * run), c_hi = min(ncta, c_lo + run);
-        int v[3] = {0, 0, 0}, tt[3];
-        for (int c = c_lo; c < c_hi; ++c) {
-            const int* p = a.part + (size_t)(first + c) * 3;
-            v[0] += p[0]; v[1] += p[1]; v[2] += p[2];
-        }
-        warp_excl_scan3(v, tt);
-        for (int c = c_lo; c < c_hi; ++c) {
-            const int* p = a.part + (size_t)(first + c) * 3;
-            cta_base[c][0] = v[0]; cta_base[c][1] = v[1]; cta_base[c][2] = v[2];
-            v[0] += p[0]; v[1] += p[1]; v[2] += p[2];
-        }
-        if (lane == 0) { sm[0][0] = tt[0]; sm[0][1] = tt[1]; sm[0][2] = tt[2]; }
+constexpr int kPrefixThreads = 1024;
+
+// grid = 2: CTA sc scans the CTA totals of scale sc.
+__global__ void __launch_bounds__(kPrefixThreads) vox_prefix_kernel(ScanArgs a) {
+    constexpr int kWarps = kPrefixThreads / 32;
+    __shared__ int wsum[3][kWarps];
+    __shared__ int tot[3];
+    const int sc = blockIdx.x;
+    const ScaleDev& g = a.s[sc];
+    const int first = sc ? a.ctas0 : 0, n = sc ? a.ctas1 : a.ctas0;
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int per = (n + kPrefixThreads - 1) / kPrefixThreads;
+    const int lo = min(n, t * per), hi = min(n, lo + per);
+    const int* src = a.cta_tot + (size_t)first * 3;
+    int* dst = a.cta_base + (size_t)first * 3;
+    int run[3] = {0, 0, 0}, wt[3];
+    for (int i = lo; i < hi; ++i) {
+#pragma unroll
+        for (int k = 0; k < 3; ++k) run[k] += src[(size_t)i * 3 + k];
+    }
+    warp_excl_scan3(run, wt);                     // run[] = exclusive inside the warp
+    if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < 3; ++k) wsum[k][warp] = wt[k];
     }
     __syncthreads();
-    const int tot0 = sm[0][0];
-    // More voxels, cells over the cap or points in them than a call's points allow: the store was not
-    // all zero when the call began (two calls on one handle at once).  Nothing is ranked or listed
-    // then; the scale reports no voxels and the handle's status becomes an internal error.
-    const bool dirty = (uint32_t)tot0 > g.max_list || (uint32_t)sm[0][1] > g.max_ovf || (uint32_t)sm[0][2] > g.max_list;
-    if (cta == 0 && t == 0) {
-        g.totals[0] = dirty ? 0 : sm[0][0]; g.totals[1] = dirty ? 0 : sm[0][1]; g.totals[2] = dirty ? 0 : sm[0][2];
-        a.num_voxels[sc] = dirty ? 0 : tot0;
-        if (dirty) atomicOr(a.status, kStatusDirtyStore);
-        else if (tot0 > a.capacity[sc]) atomicOr(a.status, kStatusCapacity);
+    if (warp < 3) {                               // warp k scans the warp totals of counter k
+        int x = wsum[warp][lane];
+        const int v = x;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
+            if (lane >= d) x += y;
+        }
+        wsum[warp][lane] = x - v;
+        if (lane == 31) tot[warp] = x;
     }
-    if (dirty) return;
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 3; ++k) run[k] += wsum[k][warp];
+    for (int i = lo; i < hi; ++i) {
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+            dst[(size_t)i * 3 + k] = run[k];
+            run[k] += src[(size_t)i * 3 + k];
+        }
+    }
+    if (t == 0) {
+        // More voxels, cells over the cap or points in them than a call's points allow: the store was
+        // not all zero when the call began (two calls on one handle at once).  Nothing is ranked or
+        // listed then; the scale reports no voxels and the handle's status becomes an internal error.
+        const bool dirty = (uint32_t)tot[0] > g.max_list || (uint32_t)tot[1] > g.max_ovf || (uint32_t)tot[2] > g.max_list;
+        g.totals[0] = dirty ? 0 : tot[0]; g.totals[1] = dirty ? 0 : tot[1]; g.totals[2] = dirty ? 0 : tot[2];
+        g.totals[3] = dirty ? 1 : 0;
+        a.num_voxels[sc] = dirty ? 0 : tot[0];
+        if (dirty) atomicOr(a.status, kStatusDirtyStore);
+        else if (tot[0] > a.capacity[sc]) atomicOr(a.status, kStatusCapacity);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 5) vox_rank_kernel(ScanArgs a) {
+    const int sc = (int)blockIdx.x >= a.ctas0 ? 1 : 0;
+    const uint32_t cta = blockIdx.x - (sc ? a.ctas0 : 0);
+    const uint32_t ncta = sc ? a.ctas1 : a.ctas0;
+    const ScaleDev& g = a.s[sc];
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const uint32_t ng = a.ngroups_used[sc];
+    // Everything that does not depend on another load is requested first: the scale's totals, the
+    // CTA's base and its 32 group counts.
+    const int dirty = g.totals[3], tot0 = g.totals[0];
+    const uint32_t gc = cta * kGroupsPerCta;
+    int pre[3] = {0, 0, 0}, ctot[3];
+    if (gc + lane < ng) {
+        const int4 info = g.group_info[gc + lane];
+        pre[0] = info.x; pre[1] = info.y; pre[2] = info.z;
+    }
+    int base[3];
+#pragma unroll
+    for (int k = 0; k < 3; ++k) base[k] = a.cta_base[(size_t)blockIdx.x * 3 + k];
+    if (dirty) return;                            // dirty store: see vox_prefix_kernel
+    const unsigned occupied = __ballot_sync(0xFFFFFFFFu, pre[0] > 0);
+    Sector x[kGroupsPerWarp];
+#pragma unroll
+    for (int u = 0; u < kGroupsPerWarp; ++u)
+        if ((occupied >> (warp * kGroupsPerWarp + u)) & 1u) x[u] = load_sector(g.store, gc + warp * kGroupsPerWarp + u, lane);
     // Clear the accumulators of the voxels found (two 16-byte halves per voxel).
     {
         const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
         const size_t n = 2 * (size_t)tot0;
         for (size_t i = (size_t)cta * kThreads + t; i < n; i += (size_t)ncta * kThreads) g.acc[i] = z;
     }
-
-    const uint32_t nw = (uint32_t)(ncta * kWarps);
-    for (uint32_t grp = (uint32_t)(cta * kWarps + warp); grp < ng; grp += nw) {
-        const int4 info = g.group_info[grp];      // same for all lanes
-        if (info.w == 0) continue;
-        const uint32_t owner = grp / per;         // warp that counted this group, within the scale
-        const int* wo = a.warp_ofs + ((size_t)first * kWarps + owner) * 3;
-        const int* cb = cta_base[owner / kWarps];
-        const int base0 = cb[0] + wo[0] + info.x;
-        Sector x = load_sector(g.store, grp, lane);
-        int run[3] = {0, 0, 0}, gtot[3];
-        sector_stats(g, x, run);
-        const bool mine = run[0] > 0;
-        warp_excl_scan3(run, gtot);               // run[] = exclusive offsets inside the group
-        if (!mine) continue;
-        int m = base0 + run[0];
-        if (g.mode == MODE_BITMAP) {
-            const uint32_t word0 = (grp * 32u + lane) * 4u;
-            const uint32_t bw[4] = {x.a.x, x.a.z, x.b.x, x.b.z};
-            uint32_t rk[4];
+    warp_excl_scan3(pre, ctot);                   // pre[] = what the CTA's groups before this lane's group hold
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                rk[i] = (uint32_t)m;
-                uint32_t bits = bw[i];
-                while (bits) {                    // plain stores: nothing here waits on memory
-                    const int bit = __ffs(bits) - 1;
-                    bits &= bits - 1;
-                    g.cell_list[m++] = (word0 + i) * 32u + bit;
-                }
-            }
-            x.a.y = rk[0]; x.a.w = rk[1]; x.b.y = rk[2]; x.b.w = rk[3];
-        } else {
-            int j = cb[1] + wo[1] + info.y + run[1], off = cb[2] + wo[2] + info.z + run[2];
-            const uint32_t cell0 = (grp * 32u + lane) * 2u;
-            x.a.y = (uint32_t)m; x.a.z = (uint32_t)j;
-            const int n0 = (int)x.a.x, n1 = (int)x.b.x;
-            const bool o0 = g.cap > 0 && n0 > g.cap, o1 = g.cap > 0 && n1 > g.cap;
-            if (o0) {
-                g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
-                j += 1; off += n0;
-            }
-            if (n0 > 0) g.cell_list[m++] = cell0 | (o0 ? 0x80000000u : 0u);
-            x.b.y = (uint32_t)m; x.b.z = (uint32_t)j;
-            if (o1) {
-                g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0 + 1u; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
-            }
-            if (n1 > 0) g.cell_list[m] = (cell0 + 1u) | (o1 ? 0x80000000u : 0u);
-        }
-        uint4* p = reinterpret_cast<uint4*>(g.store) + ((size_t)grp * 32 + lane) * 2;
-        p[0] = x.a;
-        p[1] = x.b;
+    for (int u = 0; u < kGroupsPerWarp; ++u) {
+        const int gi = warp * kGroupsPerWarp + u;
+        int gb[3];
+#pragma unroll
+        for (int k = 0; k < 3; ++k) gb[k] = base[k] + __shfl_sync(0xFFFFFFFFu, pre[k], gi);
+        if ((occupied >> gi) & 1u) rank_group(g, gc + gi, x[u], gb, lane);
     }
 }
 
@@ -517,7 +568,8 @@ vox_finalize_kernel(const float* __restrict__ pts, long long total, AccumArgs a,
     }
     // Voxel rows: a warp takes 32 consecutive rows of one scale at a time, reads their cell ids
     // from the list the rank scan wrote, writes the rows and puts the cells' store words back to
-    // zero.  Every warp has its own batch, so the batches' memory latencies overlap.
+    // zero (whole 32-byte sectors of a bitmap store: a partial write would first fetch the sector).
+    // Every warp has its own batch, so the batches' memory latencies overlap.
     __shared__ float4 s_stage[kWarps][64];
     float4* stage = s_stage[threadIdx.x >> 5];
     const int tot0 = a.s[0].totals[0], tot1 = a.s[1].totals[0];
@@ -530,8 +582,13 @@ vox_finalize_kernel(const float* __restrict__ pts, long long total, AccumArgs a,
         const int n = min(32, (sc ? tot1 : tot0) - mb);
         const uint32_t entry = lane < n ? g.cell_list[mb + lane] : 0u;
         if (lane < n) {
-            if (g.mode == MODE_BITMAP) *reinterpret_cast<uint2*>(g.store + 2 * (size_t)(entry >> 5)) = make_uint2(0u, 0u);
-            else *reinterpret_cast<uint4*>(g.store + 4 * (size_t)(entry & 0x7FFFFFFFu)) = make_uint4(0u, 0u, 0u, 0u);
+            if (g.mode == MODE_BITMAP) {
+                uint4* sp = reinterpret_cast<uint4*>(g.store + 8 * (size_t)(entry >> 7));
+                sp[0] = make_uint4(0u, 0u, 0u, 0u);
+                sp[1] = make_uint4(0u, 0u, 0u, 0u);
+            } else {
+                *reinterpret_cast<uint4*>(g.store + 4 * (size_t)(entry & 0x7FFFFFFFu)) = make_uint4(0u, 0u, 0u, 0u);
+            }
         }
         write_batch<C>(a, sc, mb, n, entry, stage);
     }
@@ -561,22 +618,18 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     }
     sa.num_voxels = d_num_voxels;
     sa.status = h->d_status;
-    sa.part = h->d_scan_part;
-    sa.warp_ofs = h->d_scan_warp_ofs;
+    sa.cta_tot = h->d_scan_tot;
+    sa.cta_base = h->d_scan_base;
+    sa.ctas0 = (int)((sa.ngroups_used[0] + kGroupsPerCta - 1) / kGroupsPerCta);
+    sa.ctas1 = (int)((sa.ngroups_used[1] + kGroupsPerCta - 1) / kGroupsPerCta);
     aa.bev = d_bev;
-    // Split the cooperative grid between the scales in proportion to their group counts.
-    // Beside stages 2 - 4 (emc2_bridge_run) a thinner grid leaves them more of each SM and the
-    // step as a whole is shorter, although this kernel alone takes longer.
-    const int G = h->thin_scan ? max(2, h->scan_blocks / 2) : h->scan_blocks;
-    const double share = (double)sa.ngroups_used[0] / (double)((uint64_t)sa.ngroups_used[0] + sa.ngroups_used[1] + 1);
-    sa.g0 = min(G - 1, max(1, (int)(share * G)));
 
     const size_t bev_n = d_bev ? (size_t)B * C * h->scale[1].dims[1] * h->scale[1].dims[0] : 0;
     const bool bev_vec = (bev_n & 3) == 0;
     if (bev_n && !bev_vec) cudaMemsetAsync(d_bev, 0, bev_n * sizeof(float), st);
     {
         // Also zeroes the BEV image; with no points it still runs for that.
-        const int blocks = max(ptiles, (bev_n && bev_vec) ? 148 : 0);
+        const int blocks = max(ptiles, (bev_n && bev_vec) ? h->num_sms : 0);
         if (blocks > 0) {
             LaunchScope ls(h, K_VOX_MARK, st);
             vox_mark_kernel<C><<<blocks, kThreads, 0, st>>>(d_points, total, N, sa.s[0], sa.s[1],
@@ -584,39 +637,33 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
                                                            bev_vec ? bev_n >> 2 : 0);
         }
     }
+    if (sa.ctas0 + sa.ctas1 > 0) {
+        LaunchScope ls(h, K_VOX_COUNT, st);
+        vox_count_kernel<<<sa.ctas0 + sa.ctas1, kThreads, 0, st>>>(sa);
+    }
     {
-        LaunchScope ls(h, K_VOX_SCAN, st);
-        void* args[] = {&sa};
-        cudaError_t e = cudaLaunchCooperativeKernel((const void*)vox_scan_kernel, dim3(G), dim3(kThreads), args, 0, st);
-        if (e != cudaSuccess) return check_cuda(h, e);
+        LaunchScope ls(h, K_VOX_PREFIX, st);      // with no frames it still reports zero voxels
+        vox_prefix_kernel<<<2, kPrefixThreads, 0, st>>>(sa);
+    }
+    if (sa.ctas0 + sa.ctas1 > 0) {
+        LaunchScope ls(h, K_VOX_RANK, st);
+        vox_rank_kernel<<<sa.ctas0 + sa.ctas1, kThreads, 0, st>>>(sa);
     }
     if (total > 0) {
-        {
-            LaunchScope ls(h, K_VOX_ACCUM, st);
-            vox_accum_kernel<C><<<ptiles, kThreads, 0, st>>>(d_points, total, N, aa);
-        }
-        {
-            // The number of voxels is only known on the device: a fixed grid strides over them.
-            const int ovf_blocks = any_cap ? kOvfBlocks : 0;
-            const int vox_blocks = (int)min((long long)148 * 8, (2 * total + 32 * 8 - 1) / (32 * 8) + 1);
-            LaunchScope ls(h, K_VOX_FINALIZE, st);
-            vox_finalize_kernel<C><<<ovf_blocks + vox_blocks, kThreads, 0, st>>>(d_points, total, aa, ovf_blocks);
-        }
+        LaunchScope ls(h, K_VOX_ACCUM, st);
+        vox_accum_kernel<C><<<ptiles, kThreads, 0, st>>>(d_points, total, N, aa);
+    }
+    if (total > 0) {
+        // The number of voxels is only known on the device: a fixed grid strides over them.
+        const int ovf_blocks = any_cap ? 2 * h->num_sms : 0;    // CTAs that serve cells over the cap
+        const int vox_blocks = (int)min((long long)h->num_sms * 8, (2 * total + 32 * 8 - 1) / (32 * 8) + 1);
+        LaunchScope ls(h, K_VOX_FINALIZE, st);
+        vox_finalize_kernel<C><<<ovf_blocks + vox_blocks, kThreads, 0, st>>>(d_points, total, aa, ovf_blocks);
     }
     return check_cuda(h, cudaGetLastError());
 }
 
 }  // namespace
-
-int voxel_scan_max_blocks() {
-    int dev = 0, sms = 0, per_sm = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, vox_scan_kernel, kThreads, 0) != cudaSuccess) return 0;
-    int coop = 0;
-    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return 0;
-    return min(sms * min(per_sm, 4), kMaxScanBlocks);
-}
 
 int launch_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* const d_coords[2],
                     int32_t* const d_counts[2], float* const d_mean[2], int32_t* const d_point_voxel[2],

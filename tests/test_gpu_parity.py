@@ -18,10 +18,12 @@ def b200():
     return pkg
 
 
-def run_case(pkg, oracle, w, batch=None, repeat=1, staged=False):
+def run_case(pkg, oracle, w, batch=None, repeat=1, staged=False, tune=()):
     batch = batch if batch is not None else gen.make_batch(w)
     ref = oracle.bridge(w, batch)
     br = pkg.Bridge(pkg.config_from_workload(w))
+    for knob, value in tune:
+        br.set_tuning(knob, value)
     d = to_dev(batch)
     bufs = None
     step = br.run_staged if staged else br.run   # three calls, or emc2_bridge_run
@@ -43,6 +45,23 @@ def test_benchmark_configs_match_the_oracle(b200, oracle, cid, staged):
 def test_ragged_shapes(b200, oracle, B, N):
     for base in (gen.KITTI, gen.NUSCENES):
         run_case(b200, oracle, base.with_shape(B, N), repeat=2, staged=(N % 2 == 0))
+
+
+TUNINGS = [(("row_store", 0),), (("row_store", 1),), (("row_store", 2),)]
+
+
+@pytest.mark.parametrize("tune", TUNINGS, ids=lambda t: "-".join(f"{k}{v}" for k, v in t))
+def test_every_implementation_choice_matches_the_oracle(b200, oracle, tune):
+    """The alternatives behind emc2_bridge_set_tuning produce the same outputs: full tiles, ragged tiles,
+    both feature widths, the dense frame (cap binds), and a frame with an expert that owns nothing."""
+    for w in (gen.NUSCENES.with_shape(2, 20000), gen.KITTI.with_shape(3, 4099), gen.NUSCENES.with_shape(1, 31),
+              gen.DENSE.with_shape(1, 50000)):
+        run_case(b200, oracle, w, repeat=2, tune=tune)
+    w = gen.KITTI.with_shape(1, 3000)
+    batch = gen.make_batch(w)
+    batch["points"][..., 0] = np.abs(batch["points"][..., 0]) % 15.0     # everything nearer than 20 m
+    batch["points"][..., 1] = batch["points"][..., 1] % 10.0
+    run_case(b200, oracle, w, batch=batch, repeat=2, tune=tune)
 
 
 def test_one_call_without_the_side_stream(b200, oracle):
