@@ -364,6 +364,9 @@ typedef enum {
                                    registers; 1 = rows staged in shared memory, ordered by expert, and written
                                    with bulk asynchronous copies (cp.async.bulk), both destinations; 2 = bulk
                                    copies for the dispatched rows only */
+    EMC2_TUNE_MARK_IN_PROJECTION = 1, /* emc2_bridge_run: 1 (default) = the projection kernel also marks the
+                                   voxel cells of both scales (one pass over the points fewer in stage 1);
+                                   0 = stage 1 marks them in a pass of its own, beside the projection */
     EMC2_TUNE_KNOBS
 } emc2_tuning_t;
 int emc2_bridge_set_tuning(emc2_bridge_t* bridge, int32_t knob, int32_t value);

@@ -41,7 +41,8 @@ ABI_SYMBOLS = (
 
 # emc2_tuning_t
 TUNE_ROW_STORE = 0
-TUNE_NAMES = {"row_store": TUNE_ROW_STORE}
+TUNE_MARK_IN_PROJECTION = 1
+TUNE_NAMES = {"row_store": TUNE_ROW_STORE, "mark_in_projection": TUNE_MARK_IN_PROJECTION}
 
 
 class Emc2Grid(ctypes.Structure):

@@ -175,6 +175,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     const size_t scan_ctas = (size_t)(h->scale[0].ngroups + 31) / 32 + (size_t)(h->scale[1].ngroups + 31) / 32;
     const size_t o_part = plan.take(scan_ctas * 3 * sizeof(int));
     const size_t o_pbase = plan.take(scan_ctas * 3 * sizeof(int));
+    const size_t o_units = plan.take(scan_ctas * sizeof(int));
     const size_t o_vif_start = plan.take(maxpts * sizeof(int));
     const size_t o_vif_cursor = plan.take(maxpts * sizeof(int));
     const size_t o_vif_list = plan.take(maxpts * sizeof(int));
@@ -212,6 +213,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     }
     h->d_scan_tot = reinterpret_cast<int*>(base + o_part);
     h->d_scan_base = reinterpret_cast<int*>(base + o_pbase);
+    h->d_scan_units = reinterpret_cast<int*>(base + o_units);
     h->d_vif_start = reinterpret_cast<int*>(base + o_vif_start);
     h->d_vif_cursor = reinterpret_cast<int*>(base + o_vif_cursor);
     h->d_vif_list = reinterpret_cast<int*>(base + o_vif_list);
@@ -239,10 +241,9 @@ static int check_call(emc2_bridge* h, int32_t B, int32_t N) {
     return EMC2_OK;
 }
 
-int emc2_voxelize(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points,
-                  int32_t* const d_coords[2], int32_t* const d_counts[2], float* const d_mean[2],
-                  int32_t* const d_point_voxel[2], const int32_t capacity[2], int32_t* d_num_voxels,
-                  float* d_bev, void* cuda_stream) {
+static int check_voxelize_args(emc2_bridge* h, int32_t B, int32_t N, const float* d_points,
+                               int32_t* const d_coords[2], int32_t* const d_counts[2], float* const d_mean[2],
+                               const int32_t capacity[2], const int32_t* d_num_voxels, const float* d_bev) {
     int rc = check_call(h, B, N);
     if (rc != EMC2_OK) return rc;
     const bool empty = B == 0 || N == 0;   // zero-sized buffers may be null
@@ -253,6 +254,15 @@ int emc2_voxelize(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points,
         if (!d_coords[s] || !d_counts[s] || !d_mean[s] || capacity[s] < 0) return EMC2_ERR_INVALID_ARG;
         if (!aligned16(d_coords[s])) return EMC2_ERR_INVALID_ARG;
     }
+    return EMC2_OK;
+}
+
+int emc2_voxelize(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_points,
+                  int32_t* const d_coords[2], int32_t* const d_counts[2], float* const d_mean[2],
+                  int32_t* const d_point_voxel[2], const int32_t capacity[2], int32_t* d_num_voxels,
+                  float* d_bev, void* cuda_stream) {
+    int rc = check_voxelize_args(h, B, N, d_points, d_coords, d_counts, d_mean, capacity, d_num_voxels, d_bev);
+    if (rc != EMC2_OK) return rc;
     DeviceGuard guard(h->cfg.device);
     if (!guard.ok) return EMC2_ERR_CUDA;
     return launch_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity,
@@ -303,21 +313,11 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
     // The stage calls validate before they enqueue anything; a host-detected error in stage 2 or
     // 3 - 4 leaves stage 1 enqueued, exactly as three separate calls would.
     if (!h) return EMC2_ERR_INVALID_ARG;
-    DeviceGuard guard(h->cfg.device);
-    if (!guard.ok) return EMC2_ERR_CUDA;
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    cudaStream_t vox_st = h->overlap ? h->side : st;
-    cudaError_t e = cudaSuccess;
-    if (h->overlap) {
-        e = cudaEventRecord(h->ev_fork, st);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->side, h->ev_fork, 0);
-        if (e != cudaSuccess) return check_cuda(h, e);
-    }
-    int rc = emc2_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity, d_num_voxels,
-                           d_bev, vox_st);
+    int rc = check_voxelize_args(h, B, N, d_points, d_coords, d_counts, d_mean, capacity, d_num_voxels, d_bev);
+    if (rc != EMC2_OK) return rc;
+    // The checks of emc2_project_gather and emc2_route_dispatch.
     int rc2 = EMC2_OK;
-    if (rc == EMC2_OK && B > 0) {
-        // The checks of emc2_project_gather and emc2_route_dispatch, then one pass over the rows.
+    if (B > 0) {
         if (!d_offsets) rc2 = EMC2_ERR_INVALID_ARG;
         else if (N > 0 && (!d_points || !d_proj || !d_feat || !d_uvd || !d_vis_mask || !d_cam ||
                            !d_expert || !d_perm || !d_points_out || !d_feat_out))   // d_gathered may be null
@@ -327,10 +327,31 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
             rc2 = EMC2_ERR_INVALID_ARG;
         else if (N > 0 && (d_points_out == d_points || d_feat_out == d_gathered))
             rc2 = EMC2_ERR_INVALID_ARG;
-        else
-            rc2 = launch_project_route_gather_dispatch(h, B, N, d_points, d_proj, d_feat, d_uvd, d_vis_mask, d_cam,
-                                                       d_gathered, d_expert, d_offsets, d_perm, d_points_out,
-                                                       d_feat_out, st);
+    }
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaStream_t vox_st = h->overlap ? h->side : st;
+    cudaError_t e = cudaSuccess;
+    // One pass over the points serves the projection, the routing and the voxelizer's marking; the
+    // rest of stage 1 then runs on the side stream beside the row traffic of stages 2 - 4.
+    const bool fused_mark = rc2 == EMC2_OK && B > 0 && N > 0 && h->tune[EMC2_TUNE_MARK_IN_PROJECTION] != 0;
+    if (fused_mark)
+        rc = launch_project_route(h, B, N, d_points, d_proj, d_uvd, d_vis_mask, d_cam, d_expert, true, d_bev, st);
+    if (rc == EMC2_OK && h->overlap) {
+        e = cudaEventRecord(h->ev_fork, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->side, h->ev_fork, 0);
+        if (e != cudaSuccess) return check_cuda(h, e);
+    }
+    if (rc == EMC2_OK)
+        rc = launch_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity, d_num_voxels,
+                             d_bev, vox_st, fused_mark);
+    if (rc == EMC2_OK && rc2 == EMC2_OK && B > 0) {
+        if (!fused_mark)
+            rc2 = launch_project_route(h, B, N, d_points, d_proj, d_uvd, d_vis_mask, d_cam, d_expert, false, nullptr, st);
+        if (rc2 == EMC2_OK)
+            rc2 = launch_scan_gather_scatter(h, B, N, d_points, d_feat, d_uvd, d_cam, d_gathered, d_expert, d_offsets,
+                                             d_perm, d_points_out, d_feat_out, st);
     }
     // Join even after an error, so that `cuda_stream` never runs ahead of stage 1.
     if (h->overlap) {
@@ -485,7 +506,7 @@ int emc2_bridge_set_overlap(emc2_bridge_t* h, int enable) {
 
 int emc2_bridge_set_tuning(emc2_bridge_t* h, int32_t knob, int32_t value) {
     if (!h || knob < 0 || knob >= EMC2_TUNE_KNOBS) return EMC2_ERR_INVALID_ARG;
-    static const int kMaxValue[EMC2_TUNE_KNOBS] = {2};
+    static const int kMaxValue[EMC2_TUNE_KNOBS] = {2, 1};
     if (value < 0 || value > kMaxValue[knob]) return EMC2_ERR_INVALID_ARG;
     h->tune[knob] = value;
     return EMC2_OK;

@@ -99,7 +99,7 @@ struct ScaleDev {
     uint32_t* ovf_cell;     // per cell over the cap j: its cell id
     int* ovf_vox;           // per cell over the cap j: its row m in the unique list
     int* ovf_list;          // global point indices of the points in cells over the cap
-    int* totals;            // [0] voxels, [1] cells over the cap, [2] points in cells over the cap, [3] store found dirty
+    int* totals;            // [0] voxels, [1] cells over the cap, [2] points in cells over the cap, [3] CTAs of the rank scan that found voxels
 };
 
 // Routing tables as the kernels take them (Sec. 3.2 distance rule, per point with visibility).
@@ -127,6 +127,7 @@ struct emc2_bridge {
     int* d_tile_base = nullptr;    // same shape, exclusive bases
     int* d_scan_tot = nullptr;     // [CTAs of the voxel rank scan, both scales][3] per-CTA totals
     int* d_scan_base = nullptr;    // same shape: their exclusive prefix sums inside each scale
+    int* d_scan_units = nullptr;   // per scale the CTAs that found voxels
     int* d_vif_start = nullptr;    // emc2_voxel_image: [max points] list starts, cursors, lists
     int* d_vif_cursor = nullptr;
     int* d_vif_list = nullptr;
@@ -137,7 +138,7 @@ struct emc2_bridge {
     int* d_rb_counts = nullptr;    // [27][voxel tiles] pairs per (offset, tile), and their prefix sums
     int* d_rb_base = nullptr;
     int max_tiles = 0;
-    int tune[EMC2_TUNE_KNOBS] = {0};   // emc2_bridge_set_tuning
+    int tune[EMC2_TUNE_KNOBS] = {0, 1};   // emc2_bridge_set_tuning
     int num_sms = 0;               // multiprocessors of the handle's device
     bool overlap = true;           // emc2_bridge_run puts stage 1 on `side`
     cudaStream_t side = nullptr;   // stream of stage 1 inside emc2_bridge_run
@@ -164,9 +165,12 @@ struct LaunchScope {
 
 int check_cuda(emc2_bridge* h, cudaError_t e);
 
+// `marked`: the cells of this batch are already marked and the BEV image zeroed (by the projection
+// kernel of the one-call path); the marking pass is then skipped.
 int launch_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* const d_coords[2],
                     int32_t* const d_counts[2], float* const d_mean[2], int32_t* const d_point_voxel[2],
-                    const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st);
+                    const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st,
+                    bool marked = false);
 int launch_project_gather(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj,
                           const float* d_feat, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
                           float* d_gathered, cudaStream_t st);
@@ -200,11 +204,16 @@ int launch_scene_route(emc2_bridge* h, int B, const int32_t* d_offsets, const ui
                        int32_t* d_scene_expert, cudaStream_t st);
 // Tile histograms (handle scratch) -> d_offsets and tile bases (handle scratch).
 void launch_route_scan(emc2_bridge* h, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st);
-// Stages 2 - 4 in one pass over the feature rows (the one-call path).
-int launch_project_route_gather_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj,
-                                         const float* d_feat, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
-                                         float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
-                                         float* d_points_out, float* d_feat_out, cudaStream_t st);
+// Stages 2 - 4 in one pass over the feature rows (the one-call path), in two parts: projection +
+// routing per point (which, with `d_bev_to_zero`/`mark`, also marks the voxel cells of both scales
+// and zeroes the BEV image, so that stage 1 reads the points once less), then offsets + rows.
+int launch_project_route(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj, float* d_uvd,
+                         uint8_t* d_vis_mask, int8_t* d_cam, uint8_t* d_expert, bool mark, float* d_bev_to_zero,
+                         cudaStream_t st);
+int launch_scan_gather_scatter(emc2_bridge* h, int B, int N, const float* d_points, const float* d_feat,
+                               const float* d_uvd, const int8_t* d_cam, float* d_gathered, const uint8_t* d_expert,
+                               int32_t* d_offsets, int32_t* d_perm, float* d_points_out, float* d_feat_out,
+                               cudaStream_t st);
 
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
@@ -235,6 +244,20 @@ __device__ __forceinline__ uint32_t cell_of(const ScaleDev& g, float x, float y,
     int iz = axis_cell(z, g.mn[2], g.vs[2], g.dims[2]);
     if ((ix | iy | iz) < 0) return 0xFFFFFFFFu;
     return (((uint32_t)b * g.dims[2] + iz) * g.dims[1] + iy) * g.dims[0] + ix;
+}
+
+// Marks the cells of one point in both scales' stores: one fire-and-forget reduction each (OR into
+// the bit word, ADD into the cell's point count).
+__device__ __forceinline__ void mark_point(const ScaleDev& s0, const ScaleDev& s1, float x, float y, float z, int b) {
+#pragma unroll
+    for (int sc = 0; sc < 2; ++sc) {
+        const ScaleDev& g = sc ? s1 : s0;
+        const uint32_t cell = cell_of(g, x, y, z, b);
+        if (cell == 0xFFFFFFFFu) continue;
+        // Results unused: these compile to reductions, which the thread does not wait for.
+        if (g.mode == MODE_BITMAP) atomicOr(&g.store[2 * (size_t)(cell >> 5)], 1u << (cell & 31u));
+        else atomicAdd(&g.store[4 * (size_t)cell], 1u);
+    }
 }
 
 __device__ __forceinline__ int warp_sum(int v) { return __reduce_add_sync(0xFFFFFFFFu, v); }

@@ -160,10 +160,16 @@ struct PrArgs {
     int N, tiles, K, H, W;
     float min_depth;
     RouteParams rp;
+    ScaleDev s0, s1;      // kMark: the voxel grids whose cells the points mark
+    float4* bev;          // kMark: BEV image to zero (bev_n4 float4), or null
+    size_t bev_n4;
 };
 
-// grid = (tiles per frame, B); tiles never straddle frames.
-template <int C>
+// grid = (tiles per frame, B); tiles never straddle frames.  kMark: the kernel also does the
+// voxelizer's marking pass (every point marks its cell in both scales' stores, and the BEV image
+// is zeroed, spread over the grid), so that stage 1 starts from marked stores and reads the
+// points once less; the reductions are fire-and-forget and land while the projection computes.
+template <int C, bool kMark>
 __global__ void __launch_bounds__(kThreads) project_route_kernel(const __grid_constant__ PrArgs a) {
     __shared__ float suvd[kTile * 3];
     __shared__ int hist[EMC2_MAX_EXPERTS];
@@ -185,6 +191,7 @@ __global__ void __launch_bounds__(kThreads) project_route_kernel(const __grid_co
         } else {
             x = __ldg(p); y = __ldg(p + 1); z = __ldg(p + 2);
         }
+        if (kMark) mark_point(a.s0, a.s1, x, y, z, b);
         const Projected pr = project_point(sP, a.K, x, y, z, a.W, a.H, a.min_depth);
         suvd[t * 3] = pr.u; suvd[t * 3 + 1] = pr.v; suvd[t * 3 + 2] = pr.d;
         a.vis[g0 + t] = (uint8_t)pr.mask;
@@ -203,6 +210,11 @@ __global__ void __launch_bounds__(kThreads) project_route_kernel(const __grid_co
     }
     __syncthreads();
     if (t < a.rp.E) a.tile_counts[((size_t)b * a.tiles + tile) * a.rp.E + t] = hist[t];
+    if (kMark && a.bev) {
+        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        const size_t cta = (size_t)blockIdx.y * gridDim.x + blockIdx.x, nthreads = (size_t)gridDim.x * gridDim.y * kThreads;
+        for (size_t i = cta * kThreads + t; i < a.bev_n4; i += nthreads) __stcs(a.bev + i, z);
+    }
 }
 
 struct GsArgs {
@@ -522,25 +534,51 @@ int launch_project_gather(emc2_bridge* h, int B, int N, const float* d_points, c
     return check_cuda(h, cudaGetLastError());
 }
 
-int launch_project_route_gather_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj,
-                                         const float* d_feat, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
-                                         float* d_gathered, uint8_t* d_expert, int32_t* d_offsets, int32_t* d_perm,
-                                         float* d_points_out, float* d_feat_out, cudaStream_t st) {
+int launch_project_route(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj, float* d_uvd,
+                         uint8_t* d_vis_mask, int8_t* d_cam, uint8_t* d_expert, bool mark, float* d_bev_to_zero,
+                         cudaStream_t st) {
+    const emc2_config_t& c = h->cfg;
+    const int tiles = (N + kTile - 1) / kTile;
+    if (B == 0 || tiles == 0) return EMC2_OK;
+    const dim3 grid(tiles, B);
+    PrArgs pa;
+    pa.pts = d_points; pa.proj = d_proj; pa.uvd = d_uvd; pa.vis = d_vis_mask; pa.cam = d_cam;
+    pa.expert = d_expert; pa.tile_counts = h->d_tile_counts;
+    pa.N = N; pa.tiles = tiles; pa.K = c.num_cameras; pa.H = c.img_h; pa.W = c.img_w;
+    pa.min_depth = c.min_depth;
+    pa.rp = route_params(h);
+    pa.s0 = h->scale[0]; pa.s1 = h->scale[1];
+    pa.bev = nullptr; pa.bev_n4 = 0;
+    if (mark && d_bev_to_zero) {
+        const size_t bev_n = (size_t)B * c.point_floats * h->scale[1].dims[1] * h->scale[1].dims[0];
+        if (bev_n & 3) {
+            cudaMemsetAsync(d_bev_to_zero, 0, bev_n * sizeof(float), st);
+        } else {
+            pa.bev = reinterpret_cast<float4*>(d_bev_to_zero);
+            pa.bev_n4 = bev_n >> 2;
+        }
+    }
+    {
+        LaunchScope ls(h, K_PROJECT_ROUTE, st);
+        if (c.point_floats == 4) {
+            if (mark) project_route_kernel<4, true><<<grid, kThreads, 0, st>>>(pa);
+            else project_route_kernel<4, false><<<grid, kThreads, 0, st>>>(pa);
+        } else {
+            if (mark) project_route_kernel<5, true><<<grid, kThreads, 0, st>>>(pa);
+            else project_route_kernel<5, false><<<grid, kThreads, 0, st>>>(pa);
+        }
+    }
+    return check_cuda(h, cudaGetLastError());
+}
+
+int launch_scan_gather_scatter(emc2_bridge* h, int B, int N, const float* d_points, const float* d_feat,
+                               const float* d_uvd, const int8_t* d_cam, float* d_gathered, const uint8_t* d_expert,
+                               int32_t* d_offsets, int32_t* d_perm, float* d_points_out, float* d_feat_out,
+                               cudaStream_t st) {
     const emc2_config_t& c = h->cfg;
     if (B == 0) return EMC2_OK;
     const int tiles = (N + kTile - 1) / kTile;
     const dim3 grid(tiles > 0 ? tiles : 1, B);
-    if (tiles > 0) {
-        PrArgs pa;
-        pa.pts = d_points; pa.proj = d_proj; pa.uvd = d_uvd; pa.vis = d_vis_mask; pa.cam = d_cam;
-        pa.expert = d_expert; pa.tile_counts = h->d_tile_counts;
-        pa.N = N; pa.tiles = tiles; pa.K = c.num_cameras; pa.H = c.img_h; pa.W = c.img_w;
-        pa.min_depth = c.min_depth;
-        pa.rp = route_params(h);
-        LaunchScope ls(h, K_PROJECT_ROUTE, st);
-        if (c.point_floats == 4) project_route_kernel<4><<<grid, kThreads, 0, st>>>(pa);
-        else project_route_kernel<5><<<grid, kThreads, 0, st>>>(pa);
-    }
     launch_route_scan(h, B, tiles, N, d_offsets, st);
     if (tiles > 0) {
         GsArgs ga;

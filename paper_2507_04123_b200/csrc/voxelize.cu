@@ -102,16 +102,7 @@ vox_mark_kernel(const float* __restrict__ pts, long long total, int N, ScaleDev 
         const int t = threadIdx.x + i * kThreads;
         if (t >= npts) continue;
         const float x = sp[t * C], y = sp[t * C + 1], z = sp[t * C + 2];
-        const int b = b0 + (i0 + t) / N;
-#pragma unroll
-        for (int sc = 0; sc < 2; ++sc) {
-            const ScaleDev& g = sc ? s1 : s0;
-            const uint32_t cell = cell_of(g, x, y, z, b);
-            if (cell == 0xFFFFFFFFu) continue;
-            // Results unused: these compile to reductions, which the thread does not wait for.
-            if (g.mode == MODE_BITMAP) atomicOr(&g.store[2 * (size_t)(cell >> 5)], 1u << (cell & 31u));
-            else atomicAdd(&g.store[4 * (size_t)cell], 1u);
-        }
+        mark_point(s0, s1, x, y, z, b0 + (i0 + t) / N);
     }
 }
 
@@ -124,6 +115,7 @@ struct ScanArgs {
     int* status;
     int* cta_tot;               // [ctas0 + ctas1][3] voxels, cells over the cap and their points per CTA
     int* cta_base;              // same shape: exclusive prefix sums inside each scale
+    int* unit_list;             // [ctas0 + ctas1] per scale: the CTAs of vox_count that found voxels, ascending
     int ctas0, ctas1;           // CTAs of vox_count / vox_rank serving scale 0 and scale 1
 };
 
@@ -155,47 +147,63 @@ __device__ __forceinline__ void sector_stats(const ScaleDev& g, const Sector& s,
     }
 }
 
-// Writes the ranks of one group into its sector and lists its occupied cells in rank order.
-// base[] = voxels, cells over the cap and points in such cells before the group.
-__device__ __forceinline__ void rank_group(const ScaleDev& g, uint32_t grp, Sector x, const int base[3], int lane) {
+// Ranks and cell list of one group of a BITMAP store: a lane owns one 32-byte sector, i.e. four
+// {bits, rank} words = 128 consecutive cells.  One warp scan of the lanes' popcounts places every
+// word; each lane then lists its own cells (a handful in all but the densest groups) with plain
+// stores that nothing waits for.  base0 = voxels before the group.
+__device__ __forceinline__ void rank_group_bitmap(const ScaleDev& g, uint32_t grp, Sector x, int base0, int lane) {
+    const uint32_t bw[4] = {x.a.x, x.a.z, x.b.x, x.b.z};
+    const int c = __popc(bw[0]) + __popc(bw[1]) + __popc(bw[2]) + __popc(bw[3]);
+    int inc = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += y;
+    }
+    if (c == 0) return;
+    int m = base0 + inc - c;
+    const uint32_t word0 = (grp * 32u + lane) * 4u;
+    uint32_t rk[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        rk[i] = (uint32_t)m;
+        uint32_t bits = bw[i];
+        while (bits) {
+            const int bit = __ffs(bits) - 1;
+            bits &= bits - 1;
+            g.cell_list[m++] = (word0 + i) * 32u + bit;
+        }
+    }
+    x.a.y = rk[0]; x.a.w = rk[1]; x.b.y = rk[2]; x.b.w = rk[3];
+    uint4* p = reinterpret_cast<uint4*>(g.store) + ((size_t)grp * 32 + lane) * 2;
+    p[0] = x.a;
+    p[1] = x.b;
+}
+
+// Ranks, cell list and over-cap bookkeeping of one group of a TABLE store (two cell records per
+// lane).  base[] = voxels, cells over the cap and points in such cells before the group.
+__device__ __forceinline__ void rank_group_table(const ScaleDev& g, uint32_t grp, Sector x, const int base[3], int lane) {
     int run[3] = {0, 0, 0}, gtot[3];
     sector_stats(g, x, run);
     const bool mine = run[0] > 0;
     warp_excl_scan3(run, gtot);                   // run[] = exclusive offsets inside the group
     if (!mine) return;
     int m = base[0] + run[0];
-    if (g.mode == MODE_BITMAP) {
-        const uint32_t word0 = (grp * 32u + lane) * 4u;
-        const uint32_t bw[4] = {x.a.x, x.a.z, x.b.x, x.b.z};
-        uint32_t rk[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            rk[i] = (uint32_t)m;
-            uint32_t bits = bw[i];
-            while (bits) {                        // plain stores: nothing here waits on memory
-                const int bit = __ffs(bits) - 1;
-                bits &= bits - 1;
-                g.cell_list[m++] = (word0 + i) * 32u + bit;
-            }
-        }
-        x.a.y = rk[0]; x.a.w = rk[1]; x.b.y = rk[2]; x.b.w = rk[3];
-    } else {
-        int j = base[1] + run[1], off = base[2] + run[2];
-        const uint32_t cell0 = (grp * 32u + lane) * 2u;
-        x.a.y = (uint32_t)m; x.a.z = (uint32_t)j;
-        const int n0 = (int)x.a.x, n1 = (int)x.b.x;
-        const bool o0 = g.cap > 0 && n0 > g.cap, o1 = g.cap > 0 && n1 > g.cap;
-        if (o0) {
-            g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
-            j += 1; off += n0;
-        }
-        if (n0 > 0) g.cell_list[m++] = cell0 | (o0 ? 0x80000000u : 0u);
-        x.b.y = (uint32_t)m; x.b.z = (uint32_t)j;
-        if (o1) {
-            g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0 + 1u; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
-        }
-        if (n1 > 0) g.cell_list[m] = (cell0 + 1u) | (o1 ? 0x80000000u : 0u);
+    int j = base[1] + run[1], off = base[2] + run[2];
+    const uint32_t cell0 = (grp * 32u + lane) * 2u;
+    x.a.y = (uint32_t)m; x.a.z = (uint32_t)j;
+    const int n0 = (int)x.a.x, n1 = (int)x.b.x;
+    const bool o0 = g.cap > 0 && n0 > g.cap, o1 = g.cap > 0 && n1 > g.cap;
+    if (o0) {
+        g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+        j += 1; off += n0;
     }
+    if (n0 > 0) g.cell_list[m++] = cell0 | (o0 ? 0x80000000u : 0u);
+    x.b.y = (uint32_t)m; x.b.z = (uint32_t)j;
+    if (o1) {
+        g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = cell0 + 1u; g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+    }
+    if (n1 > 0) g.cell_list[m] = (cell0 + 1u) | (o1 ? 0x80000000u : 0u);
     uint4* p = reinterpret_cast<uint4*>(g.store) + ((size_t)grp * 32 + lane) * 2;
     p[0] = x.a;
     p[1] = x.b;
@@ -229,9 +237,9 @@ __global__ void __launch_bounds__(kThreads) vox_count_kernel(ScanArgs a) {
 #pragma unroll
     for (int u = 0; u < kGroupsPerWarp; ++u) {
         x[u].a = x[u].b = make_uint4(0u, 0u, 0u, 0u);
-        if (g0 + u < ng) {                        // streaming: most of the store is empty, keep it out of L2
+        if (g0 + u < ng) {
             const uint4* p = reinterpret_cast<const uint4*>(g.store) + ((size_t)(g0 + u) * 32 + lane) * 2;
-            x[u].a = __ldcs(p);
+            x[u].a = __ldcs(p);                   // streaming: most of the store is empty, keep it out of L2
             x[u].b = __ldcs(p + 1);
         }
     }
@@ -260,11 +268,12 @@ __global__ void __launch_bounds__(kThreads) vox_count_kernel(ScanArgs a) {
 
 constexpr int kPrefixThreads = 1024;
 
-// grid = 2: CTA sc scans the CTA totals of scale sc.
+// grid = 2: CTA sc scans the CTA totals of scale sc.  It also lists the CTAs that found any voxel
+// (most of a fine grid is empty space), so that the ranking pass only visits those.
 __global__ void __launch_bounds__(kPrefixThreads) vox_prefix_kernel(ScanArgs a) {
     constexpr int kWarps = kPrefixThreads / 32;
-    __shared__ int wsum[3][kWarps];
-    __shared__ int tot[3];
+    __shared__ int wsum[4][kWarps];
+    __shared__ int tot[4];
     const int sc = blockIdx.x;
     const ScaleDev& g = a.s[sc];
     const int first = sc ? a.ctas0 : 0, n = sc ? a.ctas1 : a.ctas0;
@@ -273,18 +282,25 @@ __global__ void __launch_bounds__(kPrefixThreads) vox_prefix_kernel(ScanArgs a) 
     const int lo = min(n, t * per), hi = min(n, lo + per);
     const int* src = a.cta_tot + (size_t)first * 3;
     int* dst = a.cta_base + (size_t)first * 3;
-    int run[3] = {0, 0, 0}, wt[3];
+    int run[4] = {0, 0, 0, 0};                    // voxels, cells over the cap, their points, CTAs with voxels
     for (int i = lo; i < hi; ++i) {
 #pragma unroll
         for (int k = 0; k < 3; ++k) run[k] += src[(size_t)i * 3 + k];
+        run[3] += src[(size_t)i * 3] > 0;
     }
-    warp_excl_scan3(run, wt);                     // run[] = exclusive inside the warp
-    if (lane == 0) {
 #pragma unroll
-        for (int k = 0; k < 3; ++k) wsum[k][warp] = wt[k];
+    for (int k = 0; k < 4; ++k) {                 // run[] becomes exclusive inside the warp
+        int x = run[k];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
+            if (lane >= d) x += y;
+        }
+        if (lane == 31) wsum[k][warp] = x;
+        run[k] = x - run[k];
     }
     __syncthreads();
-    if (warp < 3) {                               // warp k scans the warp totals of counter k
+    if (warp < 4) {                               // warp k scans the warp totals of counter k
         int x = wsum[warp][lane];
         const int v = x;
 #pragma unroll
@@ -297,13 +313,14 @@ __global__ void __launch_bounds__(kPrefixThreads) vox_prefix_kernel(ScanArgs a) 
     }
     __syncthreads();
 #pragma unroll
-    for (int k = 0; k < 3; ++k) run[k] += wsum[k][warp];
+    for (int k = 0; k < 4; ++k) run[k] += wsum[k][warp];
     for (int i = lo; i < hi; ++i) {
 #pragma unroll
-        for (int k = 0; k < 3; ++k) {
-            dst[(size_t)i * 3 + k] = run[k];
-            run[k] += src[(size_t)i * 3 + k];
-        }
+        for (int k = 0; k < 3; ++k) dst[(size_t)i * 3 + k] = run[k];
+        const int v0 = src[(size_t)i * 3];
+        if (v0 > 0) a.unit_list[first + run[3]++] = i;
+#pragma unroll
+        for (int k = 0; k < 3; ++k) run[k] += src[(size_t)i * 3 + k];
     }
     if (t == 0) {
         // More voxels, cells over the cap or points in them than a call's points allow: the store was
@@ -311,52 +328,64 @@ __global__ void __launch_bounds__(kPrefixThreads) vox_prefix_kernel(ScanArgs a) 
         // listed then; the scale reports no voxels and the handle's status becomes an internal error.
         const bool dirty = (uint32_t)tot[0] > g.max_list || (uint32_t)tot[1] > g.max_ovf || (uint32_t)tot[2] > g.max_list;
         g.totals[0] = dirty ? 0 : tot[0]; g.totals[1] = dirty ? 0 : tot[1]; g.totals[2] = dirty ? 0 : tot[2];
-        g.totals[3] = dirty ? 1 : 0;
+        g.totals[3] = dirty ? 0 : tot[3];         // CTAs the ranking pass has to visit
         a.num_voxels[sc] = dirty ? 0 : tot[0];
         if (dirty) atomicOr(a.status, kStatusDirtyStore);
         else if (tot[0] > a.capacity[sc]) atomicOr(a.status, kStatusCapacity);
     }
 }
 
+// A fixed grid: every CTA first clears its share of the accumulators of the voxels found (two
+// 16-byte halves per voxel), then takes the listed units (32 groups of one scale) in turn.
 __global__ void __launch_bounds__(kThreads, 5) vox_rank_kernel(ScanArgs a) {
-    const int sc = (int)blockIdx.x >= a.ctas0 ? 1 : 0;
-    const uint32_t cta = blockIdx.x - (sc ? a.ctas0 : 0);
-    const uint32_t ncta = sc ? a.ctas1 : a.ctas0;
-    const ScaleDev& g = a.s[sc];
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const uint32_t ng = a.ngroups_used[sc];
-    // Everything that does not depend on another load is requested first: the scale's totals, the
-    // CTA's base and its 32 group counts.
-    const int dirty = g.totals[3], tot0 = g.totals[0];
-    const uint32_t gc = cta * kGroupsPerCta;
-    int pre[3] = {0, 0, 0}, ctot[3];
-    if (gc + lane < ng) {
-        const int4 info = g.group_info[gc + lane];
-        pre[0] = info.x; pre[1] = info.y; pre[2] = info.z;
-    }
-    int base[3];
-#pragma unroll
-    for (int k = 0; k < 3; ++k) base[k] = a.cta_base[(size_t)blockIdx.x * 3 + k];
-    if (dirty) return;                            // dirty store: see vox_prefix_kernel
-    const unsigned occupied = __ballot_sync(0xFFFFFFFFu, pre[0] > 0);
-    Sector x[kGroupsPerWarp];
-#pragma unroll
-    for (int u = 0; u < kGroupsPerWarp; ++u)
-        if ((occupied >> (warp * kGroupsPerWarp + u)) & 1u) x[u] = load_sector(g.store, gc + warp * kGroupsPerWarp + u, lane);
-    // Clear the accumulators of the voxels found (two 16-byte halves per voxel).
+    const int n0 = a.s[0].totals[3], n1 = a.s[1].totals[3];
+    const int v0 = a.s[0].totals[0], v1 = a.s[1].totals[0];
     {
         const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-        const size_t n = 2 * (size_t)tot0;
-        for (size_t i = (size_t)cta * kThreads + t; i < n; i += (size_t)ncta * kThreads) g.acc[i] = z;
+        const size_t c0 = 2 * (size_t)v0, c1 = 2 * (size_t)v1;
+        for (size_t i = (size_t)blockIdx.x * kThreads + t; i < c0 + c1; i += (size_t)gridDim.x * kThreads) {
+            if (i < c0) a.s[0].acc[i] = z; else a.s[1].acc[i - c0] = z;
+        }
     }
-    warp_excl_scan3(pre, ctot);                   // pre[] = what the CTA's groups before this lane's group hold
+    for (int u = blockIdx.x; u < n0 + n1; u += gridDim.x) {
+        const int sc = u >= n0 ? 1 : 0;
+        const ScaleDev& g = a.s[sc];
+        const int first = sc ? a.ctas0 : 0;
+        const uint32_t cta = (uint32_t)a.unit_list[first + (sc ? u - n0 : u)];
+        const uint32_t ng = a.ngroups_used[sc];
+        const uint32_t gc = cta * kGroupsPerCta;
+        int pre[3] = {0, 0, 0}, ctot[3];
+        if (gc + lane < ng) {
+            const int4 info = g.group_info[gc + lane];
+            pre[0] = info.x; pre[1] = info.y; pre[2] = info.z;
+        }
+        int base[3];
 #pragma unroll
-    for (int u = 0; u < kGroupsPerWarp; ++u) {
-        const int gi = warp * kGroupsPerWarp + u;
-        int gb[3];
+        for (int k = 0; k < 3; ++k) base[k] = a.cta_base[(size_t)(first + cta) * 3 + k];
+        const unsigned occupied = __ballot_sync(0xFFFFFFFFu, pre[0] > 0);
+        const bool bitmap = g.mode == MODE_BITMAP;
+        // The unit's occupied groups are dealt to the warps round-robin (a unit in open space has a few,
+        // one on the ground plane all 32); a warp requests all of its groups before it ranks any.
+        const int nocc = __popc(occupied);
+        int gidx[kGroupsPerWarp];
+        Sector x[kGroupsPerWarp];
 #pragma unroll
-        for (int k = 0; k < 3; ++k) gb[k] = base[k] + __shfl_sync(0xFFFFFFFFu, pre[k], gi);
-        if ((occupied >> gi) & 1u) rank_group(g, gc + gi, x[u], gb, lane);
+        for (int i = 0; i < kGroupsPerWarp; ++i) {
+            const int k = warp + i * (kThreads / 32);
+            gidx[i] = k < nocc ? (int)__fns(occupied, 0, k + 1) : -1;
+            if (gidx[i] >= 0) x[i] = load_sector(g.store, gc + gidx[i], lane);
+        }
+        warp_excl_scan3(pre, ctot);               // pre[] = what the unit's groups before this lane's group hold
+#pragma unroll
+        for (int i = 0; i < kGroupsPerWarp; ++i) {
+            if (gidx[i] < 0) break;
+            int gb[3];
+#pragma unroll
+            for (int k = 0; k < 3; ++k) gb[k] = base[k] + __shfl_sync(0xFFFFFFFFu, pre[k], gidx[i]);
+            if (bitmap) rank_group_bitmap(g, gc + gidx[i], x[i], gb[0], lane);
+            else rank_group_table(g, gc + gidx[i], x[i], gb, lane);
+        }
     }
 }
 
@@ -597,7 +626,7 @@ vox_finalize_kernel(const float* __restrict__ pts, long long total, AccumArgs a,
 template <int C>
 int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* const d_coords[2],
                  int32_t* const d_counts[2], float* const d_mean[2], int32_t* const d_point_voxel[2],
-                 const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st) {
+                 const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st, bool marked) {
     const long long total = (long long)B * N;
     const int ptiles = (int)((total + kBigTile - 1) / kBigTile);
     ScanArgs sa;
@@ -620,14 +649,15 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     sa.status = h->d_status;
     sa.cta_tot = h->d_scan_tot;
     sa.cta_base = h->d_scan_base;
+    sa.unit_list = h->d_scan_units;
     sa.ctas0 = (int)((sa.ngroups_used[0] + kGroupsPerCta - 1) / kGroupsPerCta);
     sa.ctas1 = (int)((sa.ngroups_used[1] + kGroupsPerCta - 1) / kGroupsPerCta);
     aa.bev = d_bev;
 
     const size_t bev_n = d_bev ? (size_t)B * C * h->scale[1].dims[1] * h->scale[1].dims[0] : 0;
     const bool bev_vec = (bev_n & 3) == 0;
-    if (bev_n && !bev_vec) cudaMemsetAsync(d_bev, 0, bev_n * sizeof(float), st);
-    {
+    if (!marked && bev_n && !bev_vec) cudaMemsetAsync(d_bev, 0, bev_n * sizeof(float), st);
+    if (!marked) {
         // Also zeroes the BEV image; with no points it still runs for that.
         const int blocks = max(ptiles, (bev_n && bev_vec) ? h->num_sms : 0);
         if (blocks > 0) {
@@ -647,7 +677,7 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     }
     if (sa.ctas0 + sa.ctas1 > 0) {
         LaunchScope ls(h, K_VOX_RANK, st);
-        vox_rank_kernel<<<sa.ctas0 + sa.ctas1, kThreads, 0, st>>>(sa);
+        vox_rank_kernel<<<min(sa.ctas0 + sa.ctas1, 5 * h->num_sms), kThreads, 0, st>>>(sa);
     }
     if (total > 0) {
         LaunchScope ls(h, K_VOX_ACCUM, st);
@@ -667,12 +697,12 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
 
 int launch_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* const d_coords[2],
                     int32_t* const d_counts[2], float* const d_mean[2], int32_t* const d_point_voxel[2],
-                    const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st) {
+                    const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st, bool marked) {
     if (h->cfg.point_floats == 4)
         return run_voxelize<4>(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity,
-                               d_num_voxels, d_bev, st);
+                               d_num_voxels, d_bev, st, marked);
     return run_voxelize<5>(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity,
-                           d_num_voxels, d_bev, st);
+                           d_num_voxels, d_bev, st, marked);
 }
 
 }  // namespace emc2
