@@ -283,6 +283,7 @@ def run_ours(args, w):
         gbs = pbytes / (secs_pool / args.steps) / 1e9
         pool_info = {"p": args.pool, "ms_per_launch": secs_pool / args.steps * 1e3, "bytes_per_launch": pbytes,
                      "achieved_gbs": gbs, f"frac_of_{kind0}_copy": gbs / peak0}
+        unpooled = (w, d["feat"])
         w = replace(w, name=f"{w.name}_pool{args.pool}", feat_stride=w.feat_stride * args.pool,
                     feat_offset=(args.pool - 1) / 2 * w.feat_stride)
         d["feat"] = pooled
@@ -540,7 +541,21 @@ def run_ours(args, w):
             br.status()
             ms_vs = secs_vs / args.steps * 1e3
             sbytes = B * N * 4 + M * 4 + nvis * 13 + texels * 4 * w.feat_c + M * (4 * w.feat_c + 4)
-            vi[f"scale{sc}"] = {"ms_per_call": ms_vi, "voxels": M, "visible_points": nvis,
+            fused = {}
+            if args.pool > 1:
+                # Multiscale Pooling folded into the per-voxel sampling (window means taken where the taps are
+                # read, from the unpooled maps) against pooling first and sampling the pooled maps.
+                w0, feat0 = unpooled
+                br_u = make_bridge(pkg, w0, local_rank, args.tune)
+                fn3 = lambda: br_u.voxel_image_pooled(bufs["vox"], sc, pg["uvd"], pg["cam"], feat0, args.pool, out)
+                for _ in range(3):
+                    fn3()
+                secs_vp = time_steps(fn3, args.steps, sync, barrier)
+                br_u.status()
+                br_u.close()
+                fused = {"pooling_folded_into_sampling_ms_per_call": secs_vp / args.steps * 1e3,
+                         "pool_then_sample_ms": pool_info["ms_per_launch"] + ms_vs}
+            vi[f"scale{sc}"] = {**fused, "ms_per_call": ms_vi, "voxels": M, "visible_points": nvis,
                                 "algorithmic_bytes": vbytes, "achieved_gbs": vbytes / (ms_vi * 1e-3) / 1e9,
                                 "sampled_ms_per_call": ms_vs, "sampled_algorithmic_bytes": sbytes,
                                 "sampled_achieved_gbs": sbytes / (ms_vs * 1e-3) / 1e9}

@@ -101,8 +101,8 @@ typedef struct {
 
 /* Validates the configuration, selects the device and allocates all scratch memory the stage
  * calls will ever need for (max_batch, max_points).  Returns EMC2_ERR_BAD_CONFIG for an
- * unusable configuration (zero voxel size, more than 2^32 - 1 cells per batch, a cap on a grid
- * too large for a direct count table, feat_c not a multiple of 4, stride not a power of two,
+ * unusable configuration (zero voxel size, more than 2^32 - 1 cells per batch,
+ * feat_c not a multiple of 4, stride not a power of two,
  * lut entry >= num_experts, ...), EMC2_ERR_CUDA if the device or memory is unavailable. */
 int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out);
 
@@ -254,6 +254,20 @@ int emc2_voxel_image_sampled(emc2_bridge_t* bridge, int32_t B, int32_t N, int32_
                              const int32_t* d_point_voxel, const int32_t* d_counts, const int32_t* d_num_voxels,
                              const float* d_uvd, const int8_t* d_cam, const float* d_feat, float* d_vox_img,
                              int32_t* d_vox_img_count, void* cuda_stream);
+
+/* Multiscale Pooling folded into the fusion by voxel (Sec. 3.5 pools the image features before they
+ * are fused, to relieve memory; Fig. 5 fuses by voxel): the result of emc2_pool_features(p) followed by
+ * emc2_voxel_image_sampled on the pooled maps, without the pooled maps ever being written or read.
+ * d_feat are the handle's UNPOOLED maps [B, K, Hf, Wf, Cf]; p is the pooling size, a power of two
+ * (1 = emc2_voxel_image_sampled).  Every tap of the bilinear blend is the mean of the p x p window of
+ * texels that the pooled texel stands for (ragged windows at the right / bottom edge average over the
+ * texels they hold); the pooled texels sit at the centres of their windows, as in emc2_pool_features.
+ * d_uvd and d_cam come from a projection with the same images (they do not depend on the maps).
+ * Other arguments, outputs, scratch and ordering rule as emc2_voxel_image_sampled. */
+int emc2_voxel_image_pooled(emc2_bridge_t* bridge, int32_t B, int32_t N, int32_t capacity,
+                            const int32_t* d_point_voxel, const int32_t* d_counts, const int32_t* d_num_voxels,
+                            const float* d_uvd, const int8_t* d_cam, const float* d_feat, int32_t p,
+                            float* d_vox_img, int32_t* d_vox_img_count, void* cuda_stream);
 
 /* Occlusion test for the "occluded / out-of-view" bucket of the dispatcher (Sec. 3.2 names occlusion
  * among the causes of missing LiDAR detail; the paper gives no test, this is a depth buffer).  Every

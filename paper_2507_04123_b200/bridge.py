@@ -36,7 +36,7 @@ ABI_SYMBOLS = (
     "emc2_bridge_run", "emc2_bridge_run_host", "emc2_bridge_set_overlap", "emc2_scene_route", "emc2_pool_features",
     "emc2_features_channels_last",
     "emc2_voxel_image", "emc2_voxel_image_sampled", "emc2_occlusion", "emc2_rulebook",
-    "emc2_bridge_set_tuning", "emc2_bridge_profile_timeline",
+    "emc2_bridge_set_tuning", "emc2_bridge_profile_timeline", "emc2_voxel_image_pooled",
 )
 
 # emc2_tuning_t
@@ -94,6 +94,7 @@ def load_library() -> ctypes.CDLL:
     lib.emc2_occlusion.argtypes = [vp, i32, i32, vp, vp, vp, i32, ctypes.c_float, vp, vp, vp, vp]
     lib.emc2_voxel_image.argtypes = [vp, i32, i32, i32] + [vp] * 8
     lib.emc2_voxel_image_sampled.argtypes = [vp, i32, i32, i32] + [vp] * 9
+    lib.emc2_voxel_image_pooled.argtypes = [vp, i32, i32, i32] + [vp] * 6 + [i32, vp, vp, vp]
     lib.emc2_rulebook.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, ctypes.c_int64, vp]
     lib.emc2_pool_features.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.emc2_features_channels_last.argtypes = [vp, i32, vp, vp, vp]
@@ -177,6 +178,8 @@ def route_dispatch_static(config: Emc2Config, points: torch.Tensor, vis_mask: to
     lib = load_library()
     B, N, C = points.shape
     dev = points.device
+    if dev.type != "cuda" or dev.index != config.device:
+        raise ValueError(f"points live on {dev}, the configuration names CUDA device {config.device}")
     _check(points, torch.float32, (B, N, config.point_floats), "points", dev)
     _check(vis_mask, torch.uint8, (B, N), "vis_mask", dev)
     _check(gathered, torch.float32, (B, N, config.feat_c), "gathered", dev)
@@ -348,6 +351,29 @@ class Bridge:
                                                feat.data_ptr(), out["vox_img"].data_ptr(),
                                                out["vox_img_count"].data_ptr(), self._stream())
         self._raise(rc, "emc2_voxel_image_sampled")
+        return out
+
+    def voxel_image_pooled(self, vox: Dict[str, object], scale: int, uvd: torch.Tensor, cam: torch.Tensor,
+                           feat: torch.Tensor, p: int, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        """emc2_voxel_image_pooled: per-voxel image features from p x p window means of the unpooled maps."""
+        B, N = cam.shape
+        c = self.cfg
+        pv = vox["point_voxel"][scale]
+        counts = vox["counts"][scale]
+        cap = int(counts.shape[0])
+        _check(pv, torch.int32, (B, N), "point_voxel", self.device)
+        _check(uvd, torch.float32, (B, N, 3), "uvd", self.device)
+        _check(cam, torch.int8, (B, N), "cam", self.device)
+        _check(feat, torch.float32, (B, c.num_cameras, c.feat_h, c.feat_w, c.feat_c), "feat", self.device)
+        if out is None:
+            out = {"vox_img": torch.empty((cap, c.feat_c), dtype=torch.float32, device=self.device),
+                   "vox_img_count": torch.empty((cap,), dtype=torch.int32, device=self.device)}
+        nv = vox["num_voxels"]
+        rc = self.lib.emc2_voxel_image_pooled(self._h, B, N, cap, pv.data_ptr(), counts.data_ptr(),
+                                              nv.data_ptr() + 4 * scale, uvd.data_ptr(), cam.data_ptr(),
+                                              feat.data_ptr(), int(p), out["vox_img"].data_ptr(),
+                                              out["vox_img_count"].data_ptr(), self._stream())
+        self._raise(rc, "emc2_voxel_image_pooled")
         return out
 
     def rulebook(self, vox: Dict[str, object], scale: int, pair_capacity: Optional[int] = None,

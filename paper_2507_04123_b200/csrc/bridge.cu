@@ -8,7 +8,7 @@
 namespace emc2 {
 
 static const char* const kKernelNames[K_KINDS] = {
-    "vox_mark", "vox_count", "vox_prefix", "vox_rank", "vox_accum", "vox_finalize",
+    "vox_mark", "vox_count", "vox_prefix", "vox_rank", "vox_accum", "vox_over_find", "vox_over_fill", "vox_finalize",
     "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features",
     "vif_scan", "vif_fill", "vif_mean", "vif_sample", "occl_fill", "occl_splat", "occl_test",
     "channels_last", "rb_mark", "rb_count", "rb_scan", "rb_fill", "rb_clear"};
@@ -76,9 +76,6 @@ int validate(const emc2_config_t& c) {
         }
         if (cells * (uint64_t)c.max_batch > 0xFFFFFF00ull) return EMC2_ERR_BAD_CONFIG;
         if (g.max_points < 0) return EMC2_ERR_BAD_CONFIG;
-        // The per-voxel cap needs the per-cell point count, which only the count table holds.
-        if (g.max_points > 0 && cells * (uint64_t)c.max_batch > (uint64_t)kMaxTableCells)
-            return EMC2_ERR_BAD_CONFIG;
     }
     if (c.grid[1].dims[2] != 1) return EMC2_ERR_BAD_CONFIG;
     if (c.num_cameras < 1 || c.num_cameras > EMC2_MAX_CAMERAS) return EMC2_ERR_BAD_CONFIG;
@@ -395,6 +392,23 @@ int emc2_voxel_image_sampled(emc2_bridge_t* h, int32_t B, int32_t N, int32_t cap
     if (!guard.ok) return EMC2_ERR_CUDA;
     return launch_voxel_image(h, B, N, capacity, d_point_voxel, d_counts, d_num_voxels, nullptr, nullptr, d_uvd,
                               d_cam, d_feat, d_vox_img, d_vox_img_count, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int emc2_voxel_image_pooled(emc2_bridge_t* h, int32_t B, int32_t N, int32_t capacity, const int32_t* d_point_voxel,
+                            const int32_t* d_counts, const int32_t* d_num_voxels, const float* d_uvd,
+                            const int8_t* d_cam, const float* d_feat, int32_t p, float* d_vox_img,
+                            int32_t* d_vox_img_count, void* cuda_stream) {
+    int rc = check_call(h, B, N);
+    if (rc != EMC2_OK) return rc;
+    if (capacity < 0 || !d_num_voxels || !is_pow2(p)) return EMC2_ERR_INVALID_ARG;
+    if (B == 0 || N == 0 || capacity == 0) return EMC2_OK;
+    if (!d_point_voxel || !d_counts || !d_uvd || !d_cam || !d_feat || !d_vox_img || !d_vox_img_count)
+        return EMC2_ERR_INVALID_ARG;
+    if (!aligned16(d_feat) || !aligned16(d_vox_img)) return EMC2_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return EMC2_ERR_CUDA;
+    return launch_voxel_image(h, B, N, capacity, d_point_voxel, d_counts, d_num_voxels, nullptr, nullptr, d_uvd,
+                              d_cam, d_feat, d_vox_img, d_vox_img_count, static_cast<cudaStream_t>(cuda_stream), p);
 }
 
 int emc2_rulebook(emc2_bridge_t* h, int32_t scale, int32_t capacity, const int32_t* d_coords,

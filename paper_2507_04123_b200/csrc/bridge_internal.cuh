@@ -24,6 +24,8 @@ enum KernelKind {
     K_VOX_PREFIX,
     K_VOX_RANK,
     K_VOX_ACCUM,
+    K_VOX_OVER_FIND,
+    K_VOX_OVER_FILL,
     K_VOX_FINALIZE,
     K_PROJECT_GATHER,
     K_PROJECT_ROUTE,
@@ -194,7 +196,7 @@ int voxel_image_scan_max_blocks();
 int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t* d_point_voxel,
                        const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
                        const float* d_gathered, const float* d_uvd, const int8_t* d_cam, const float* d_feat,
-                       float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st);
+                       float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st, int pool = 1);
 int launch_rulebook(emc2_bridge* h, int scale, int capacity, const int32_t* d_coords, const int32_t* d_num_voxels,
                     int32_t* d_rule_offsets, int32_t* d_rule_in, int32_t* d_rule_out, long long pair_capacity,
                     cudaStream_t st);

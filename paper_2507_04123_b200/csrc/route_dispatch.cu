@@ -376,6 +376,8 @@ extern "C" int emc2_route_dispatch_static(const emc2_config_t* config, int32_t B
         for (int d = 0; d <= c.num_thresholds; ++d)
             if (c.lut[v][d] >= c.num_experts) return EMC2_ERR_BAD_CONFIG;
     if (B < 0 || N < 0 || B > EMC2_MAX_BATCH) return EMC2_ERR_INVALID_ARG;
+    // No frame that fits the scratch area is anywhere near this long; it also keeps the tile count in range.
+    if ((int64_t)N > (int64_t)EMC2_STATIC_SCRATCH_ENTRIES * kTile) return EMC2_ERR_TOO_LARGE;
     const int E = c.num_experts;
     const int tiles = (N + kTile - 1) / kTile;
     if ((int64_t)B * tiles * E > (int64_t)EMC2_STATIC_SCRATCH_ENTRIES) return EMC2_ERR_TOO_LARGE;

@@ -33,6 +33,8 @@ struct VifArgs {
     const float4* feat;         // feature maps (vif_sample)
     int N, K, Hf, Wf;
     float inv_stride, offset;
+    int pool, Hp, Wp;           // pool > 1: taps are p x p window means of the maps (Multiscale Pooling folded
+                                // into the sampling); Hp x Wp is the pooled map, inv_stride / offset describe it
     float4* vox_img;            // [capacity, cf4]
     int32_t* vox_cnt;           // [capacity]
     int* start;                 // [capacity] first list slot of each voxel
@@ -114,8 +116,11 @@ __global__ void __launch_bounds__(kThreads) vif_fill_kernel(VifArgs a) {
         if (a.vis) {
             entry = a.vis[i] ? (int)i : ~(int)i;
         } else {                                        // rows will be blended from the maps: keep the taps
-            rec = tap_record((int)(i / a.N), (int)a.cam[i], a.uvd[3 * i], a.uvd[3 * i + 1], a.K, a.Hf, a.Wf, a.cf4,
-                             a.inv_stride, a.offset);
+            // pooled: the record addresses a TEXEL of the pooled map (not a float4 of a row), see pooled_column
+            rec = a.pool > 1 ? tap_record((int)(i / a.N), (int)a.cam[i], a.uvd[3 * i], a.uvd[3 * i + 1], a.K, a.Hp, a.Wp, 1,
+                                          a.inv_stride, a.offset)
+                             : tap_record((int)(i / a.N), (int)a.cam[i], a.uvd[3 * i], a.uvd[3 * i + 1], a.K, a.Hf, a.Wf,
+                                          a.cf4, a.inv_stride, a.offset);
         }
         const int pos = a.start[m] + atomicAdd(&a.cursor[m], 1);
         // Inside the list whenever counts[] are the kept-point counts of pv[] (the voxelizer's outputs
@@ -145,7 +150,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_mean_kernel
         for (int u = 0; u < 2; ++u) {
             const bool ok = mm[u] < M;
             s0[u] = ok ? a.start[mm[u]] : 0;
-            n[u] = ok ? a.counts[mm[u]] : 0;
+            n[u] = ok ? min(a.counts[mm[u]], a.cursor[mm[u]]) : 0;   // never past what this call appended
         }
 #pragma unroll
         for (int u = 0; u < 2; ++u) first[u] = n[u] > 0 ? a.list[s0[u]] : -1;
@@ -185,10 +190,44 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_mean_kernel
     }
 }
 
+// Mean of the p x p window of map texels that pooled texel (ty, tx) of map `map` stands for, column c:
+// the same sum, in the same order, as pool_features_kernel (rows outer, columns inner, one multiply by
+// the reciprocal of the texel count), so the value is the pooled map's, bit for bit.
+__device__ __forceinline__ float4 window_mean(const VifArgs& a, uint32_t map, int ty, int tx, int c, int cf4) {
+    const int j0 = ty * a.pool, j1 = min(a.Hf, j0 + a.pool), i0 = tx * a.pool, i1 = min(a.Wf, i0 + a.pool);
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = j0; j < j1; ++j) {
+        const float4* row = a.feat + (((size_t)map * a.Hf + j) * a.Wf + i0) * cf4 + c;
+        for (int x = 0; x < i1 - i0; ++x) {
+            const float4 v = __ldg(row + (size_t)x * cf4);
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+    }
+    const float inv = 1.0f / (float)((j1 - j0) * (i1 - i0));
+    return make_float4(s.x * inv, s.y * inv, s.z * inv, s.w * inv);
+}
+
+// gather_column on the pooled map that is never materialised: the four taps are window means.
+__device__ __forceinline__ float4 pooled_column(const VifArgs& a, const uint4& rec, int c, int cf4) {
+    if (rec.x == kZeroRow) return make_float4(0.f, 0.f, 0.f, 0.f);
+    uint32_t t = rec.x;
+    const int x0 = (int)(t % (uint32_t)a.Wp);
+    t /= (uint32_t)a.Wp;
+    const int y0 = (int)(t % (uint32_t)a.Hp);
+    const uint32_t map = t / (uint32_t)a.Hp;
+    const int x1 = x0 + (int)(rec.y & 1u), y1 = y0 + (int)((rec.y >> 1) & 1u);
+    const float4 f00 = window_mean(a, map, y0, x0, c, cf4);
+    const float4 f01 = x1 != x0 ? window_mean(a, map, y0, x1, c, cf4) : f00;
+    const float4 f10 = y1 != y0 ? window_mean(a, map, y1, x0, c, cf4) : f00;
+    const float4 f11 = y1 != y0 ? (x1 != x0 ? window_mean(a, map, y1, x1, c, cf4) : f10) : f01;
+    return blend(f00, f01, f10, f11, __uint_as_float(rec.z), __uint_as_float(rec.w));
+}
+
 // vif_mean without the per-point rows: every listed point's row is blended from its four taps of
 // the feature maps here (the blend of the gather stage, from the point's pixel and camera), so the
 // [points, Cf] buffer is neither written nor read.  Same thread layout as vif_mean.
-template <int CF4>
+// kPooled: the taps are window means of the unpooled maps (emc2_voxel_image_pooled).
+template <int CF4, bool kPooled>
 __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_sample_kernel(VifArgs a) {
     if (*a.bad) return;
     const int M = voxels_in_use(a);
@@ -205,7 +244,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_sample_kern
         for (int u = 0; u < 2; ++u) {
             const bool ok = mm[u] < M;
             s0[u] = ok ? a.start[mm[u]] : 0;
-            n[u] = ok ? a.counts[mm[u]] : 0;
+            n[u] = ok ? min(a.counts[mm[u]], a.cursor[mm[u]]) : 0;   // never past what this call appended
             acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         // The first entries of the two voxels together, then the rest of each list, two at a time;
@@ -216,7 +255,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_sample_kern
             for (int u = 0; u < 2; ++u) rec[u] = n[u] > 0 ? a.recs[s0[u]] : make_uint4(kZeroRow, 0u, 0u, 0u);
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
-                acc[u] = gather_column(a.feat, rec[u], c, (uint32_t)cf4, row_stride);
+                acc[u] = kPooled ? pooled_column(a, rec[u], c, cf4) : gather_column(a.feat, rec[u], c, (uint32_t)cf4, row_stride);
                 seen[u] = rec[u].x != kZeroRow ? 1 : 0;
             }
         }
@@ -228,7 +267,8 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) vif_sample_kern
 #pragma unroll
                 for (int j = 0; j < 2; ++j) rec[j] = k + j < n[u] ? a.recs[s0[u] + k + j] : make_uint4(kZeroRow, 0u, 0u, 0u);
 #pragma unroll
-                for (int j = 0; j < 2; ++j) v[j] = gather_column(a.feat, rec[j], c, (uint32_t)cf4, row_stride);
+                for (int j = 0; j < 2; ++j)
+                    v[j] = kPooled ? pooled_column(a, rec[j], c, cf4) : gather_column(a.feat, rec[j], c, (uint32_t)cf4, row_stride);
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
                     if (rec[j].x == kZeroRow) continue;
@@ -265,7 +305,7 @@ int voxel_image_scan_max_blocks() {
 int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t* d_point_voxel,
                        const int32_t* d_counts, const int32_t* d_num_voxels, const uint8_t* d_vis_mask,
                        const float* d_gathered, const float* d_uvd, const int8_t* d_cam, const float* d_feat,
-                       float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st) {
+                       float* d_vox_img, int32_t* d_vox_img_count, cudaStream_t st, int pool) {
     const emc2_config_t& cfg = h->cfg;
     VifArgs a;
     a.pv = d_point_voxel; a.counts = d_counts; a.num_voxels = d_num_voxels; a.vis = d_vis_mask;
@@ -273,6 +313,13 @@ int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t
     a.cam = d_cam; a.uvd = d_uvd; a.feat = reinterpret_cast<const float4*>(d_feat);
     a.N = N; a.K = cfg.num_cameras; a.Hf = cfg.feat_h; a.Wf = cfg.feat_w;
     a.inv_stride = 1.0f / (float)cfg.feat_stride; a.offset = cfg.feat_offset;
+    a.pool = pool; a.Hp = cfg.feat_h; a.Wp = cfg.feat_w;
+    if (pool > 1) {
+        // The pooled map: texel J sits at the centre of its window, (J p + (p - 1) / 2) texels of stride s in.
+        a.Hp = (cfg.feat_h + pool - 1) / pool; a.Wp = (cfg.feat_w + pool - 1) / pool;
+        a.inv_stride = 1.0f / ((float)cfg.feat_stride * (float)pool);
+        a.offset = cfg.feat_offset + 0.5f * (float)(pool - 1) * (float)cfg.feat_stride;
+    }
     a.vox_img = reinterpret_cast<float4*>(d_vox_img); a.vox_cnt = d_vox_img_count;
     a.start = h->d_vif_start; a.cursor = h->d_vif_cursor; a.list = h->d_vif_list; a.part = h->d_vif_part;
     a.recs = h->d_vif_recs;
@@ -305,10 +352,14 @@ int launch_voxel_image(emc2_bridge* h, int B, int N, int capacity, const int32_t
         }
     } else {
         LaunchScope ls(h, K_VIF_SAMPLE, st);
-        switch (a.cf4) {
-            case 16: vif_sample_kernel<16><<<blocks, 16 * 16, 0, st>>>(a); break;
-            case 20: vif_sample_kernel<20><<<blocks, 16 * 20, 0, st>>>(a); break;
-            default: vif_sample_kernel<0><<<blocks, kThreads, 0, st>>>(a); break;
+        if (pool > 1) {
+            vif_sample_kernel<0, true><<<blocks, kThreads, 0, st>>>(a);
+        } else {
+            switch (a.cf4) {
+                case 16: vif_sample_kernel<16, false><<<blocks, 16 * 16, 0, st>>>(a); break;
+                case 20: vif_sample_kernel<20, false><<<blocks, 16 * 20, 0, st>>>(a); break;
+                default: vif_sample_kernel<0, false><<<blocks, kThreads, 0, st>>>(a); break;
+            }
         }
     }
     return check_cuda(h, cudaGetLastError());

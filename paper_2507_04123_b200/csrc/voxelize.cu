@@ -471,6 +471,65 @@ vox_accum_kernel(const float* __restrict__ pts, long long total, int N, AccumArg
     }
 }
 
+// ------------------------------------------------------------------ per-voxel cap on a bitmap scale
+// A bitmap store keeps no per-cell point count, so a voxel over its cap is only known once the points
+// are accumulated.  Two small passes then build what the table path gets from the rank scan:
+//   vox_over_find   a thread per voxel row: count > cap -> the voxel takes the next place j among the
+//                   over-cap voxels and the next `count` slots of the index list (warp-aggregated
+//                   tickets), and remembers j + 1 in the spare word of its accumulator;
+//   vox_over_fill   a thread per point: if its voxel is over the cap, the point's index goes into the
+//                   voxel's list.
+// vox_finalize then keeps the `cap` lowest indices of every list exactly as for a table scale.
+__global__ void __launch_bounds__(kThreads) vox_over_find_kernel(AccumArgs a, int sc) {
+    const ScaleDev& g = a.s[sc];
+    const int lane = threadIdx.x & 31;
+    const int M = min(g.totals[0], a.capacity[sc]);
+    for (int m0 = (blockIdx.x * kThreads + threadIdx.x) & ~31; m0 < M; m0 += gridDim.x * kThreads) {
+        const int m = m0 + lane;
+        const int n = m < M ? (int)g.acc[2 * (size_t)m + 1].y : 0;
+        const bool over = n > g.cap;
+        const unsigned who = __ballot_sync(0xFFFFFFFFu, over);
+        if (!who) continue;
+        int inc = over ? n : 0;                   // inclusive scan of the over-cap counts
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+            if (lane >= d) inc += y;
+        }
+        int j0 = 0, off0 = 0;
+        if (lane == 31) {
+            j0 = atomicAdd(&g.totals[1], __popc(who));
+            off0 = atomicAdd(&g.totals[2], inc);
+        }
+        j0 = __shfl_sync(0xFFFFFFFFu, j0, 31);
+        off0 = __shfl_sync(0xFFFFFFFFu, off0, 31);
+        if (!over) continue;
+        const int j = j0 + __popc(who & ((1u << lane) - 1u));
+        const int off = off0 + inc - n;
+        if ((uint32_t)j >= g.max_ovf || (uint32_t)(off + n) > g.max_list) continue;   // cannot happen with this batch's counts
+        g.ovf_vox[j] = m; g.ovf_off[j] = off; g.ovf_cell[j] = g.cell_list[m];
+        g.ovf_cursor[(size_t)j * kCursorStride] = 0;
+        reinterpret_cast<uint32_t*>(g.acc + 2 * (size_t)m + 1)[2] = (uint32_t)j + 1u;
+    }
+}
+
+template <int C>
+__global__ void __launch_bounds__(kThreads)
+vox_over_fill_kernel(const float* __restrict__ pts, long long total, int N, AccumArgs a, int sc) {
+    const ScaleDev& g = a.s[sc];
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < total; i += (long long)gridDim.x * kThreads) {
+        const float* p = pts + i * C;
+        const Slot s = slot_of(g, cell_of(g, p[0], p[1], p[2], (int)(i / N)));
+        if (s.m < 0 || s.m >= a.capacity[sc]) continue;
+        const uint32_t tag = reinterpret_cast<const uint32_t*>(g.acc + 2 * (size_t)s.m + 1)[2];
+        if (tag == 0u || tag > g.max_ovf) continue;
+        const int j = (int)tag - 1;
+        const int tk = atomicAdd(&g.ovf_cursor[(size_t)j * kCursorStride], 1);
+        const uint32_t pos = (uint32_t)(g.ovf_off[j] + tk);
+        if (pos < g.max_list) g.ovf_list[pos] = (int)i;
+    }
+}
+
 // ------------------------------------------------------------------ pass 4: rows, BEV, cleanup
 // Writes the output rows of n <= 32 voxels with consecutive rows mb, mb+1, ..., one per lane;
 // lane i holds the cell-list entry of row mb + i; `stage` is 1 KB of the warp's own shared memory.  Accumulators are read and mean rows written as
@@ -491,7 +550,9 @@ __device__ __forceinline__ void write_batch(const AccumArgs& a, int sc, int mb, 
     const bool active = lane < n;
     const bool table = g.mode == MODE_TABLE;
     const uint32_t cell = table ? (entry & 0x7FFFFFFFu) : entry;
-    const bool over = active && table && (entry >> 31) != 0u;
+    // Over the cap: a table store flags the cell in its list entry; a bitmap store has no per-cell count,
+    // there vox_over_find_kernel left the voxel's place among the over-cap voxels (+ 1) in a spare word.
+    const bool over = active && ((table && (entry >> 31) != 0u) || __float_as_uint(a1.z) != 0u);
     uint32_t r = cell, x, y, z;
     g.div[0].divmod(r, r, x);
     g.div[1].divmod(r, r, y);
@@ -682,6 +743,18 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     if (total > 0) {
         LaunchScope ls(h, K_VOX_ACCUM, st);
         vox_accum_kernel<C><<<ptiles, kThreads, 0, st>>>(d_points, total, N, aa);
+    }
+    for (int s = 0; s < 2 && total > 0; ++s) {
+        if (h->scale[s].mode != MODE_BITMAP || h->scale[s].cap <= 0) continue;
+        {
+            LaunchScope ls(h, K_VOX_OVER_FIND, st);
+            vox_over_find_kernel<<<4 * h->num_sms, kThreads, 0, st>>>(aa, s);
+        }
+        {
+            LaunchScope ls(h, K_VOX_OVER_FILL, st);
+            vox_over_fill_kernel<C><<<(int)min((long long)8 * h->num_sms, (total + kThreads - 1) / kThreads), kThreads, 0, st>>>(
+                d_points, total, N, aa, s);
+        }
     }
     if (total > 0) {
         // The number of voxels is only known on the device: a fixed grid strides over them.

@@ -65,6 +65,19 @@ def test_every_implementation_choice_matches_the_oracle(b200, oracle, tune):
     run_case(b200, oracle, w, batch=batch, repeat=2, tune=tune)
 
 
+def test_per_voxel_cap_on_the_fine_scale(b200, oracle):
+    """max_points on a grid too large for per-cell counts (the fine scale): keep-first-by-index, counts = kept,
+    means over the kept points, dropped points at -1 - as on the pillar scale."""
+    from dataclasses import replace
+    for base, n in ((gen.DENSE, 150_000), (gen.NUSCENES.with_shape(2, 80_000), None)):
+        w = base if n is None else base.with_shape(1, n)
+        w = replace(w, grids=(replace(w.grids[0], max_points=3), w.grids[1]))
+        ref, bufs = run_case(b200, oracle, w, repeat=2)
+        assert int((ref["vox0"]["counts"] == 3).sum()) > 100          # the cap binds on many voxels
+        assert int((ref["vox0"]["point_voxel"] < 0).sum()) > 0
+        run_case(b200, oracle, w, repeat=2, staged=True)
+
+
 def test_one_call_without_the_side_stream(b200, oracle):
     w = gen.NUSCENES.with_shape(2, 20000)
     batch = gen.make_batch(w)
@@ -278,6 +291,47 @@ def test_image_features_per_voxel(b200, oracle, cid, B, N):
     br.close()
 
 
+@pytest.mark.parametrize("p", [2, 4])
+def test_pooled_image_features_per_voxel(b200, oracle, p):
+    """Multiscale Pooling and the fusion by voxel as ONE path, in the paper's order: pool the maps, sample them
+    at the projected points, attach the rows to the voxels (zero rows where a voxel has no pixel).  The oracle
+    chain is pool -> gather(window-centre offset) -> voxel_image; the CUDA chain is emc2_pool_features -> a
+    handle for the pooled maps -> emc2_voxel_image_sampled, and emc2_voxel_image_pooled, which folds the
+    pooling into the sampling and must agree with it."""
+    from dataclasses import replace
+    for base in (gen.NUSCENES.with_shape(2, 40_000), gen.KITTI.with_shape(1, 30_000)):
+        batch = gen.make_batch(base)
+        d = to_dev(batch)
+        br0 = b200.Bridge(b200.config_from_workload(base))
+        pooled = br0.pool_features(d["feat"], p)
+        raw = br0.run(d["points"], d["proj"], d["feat"])         # unpooled handle: voxels, uvd, cam
+        br0.status()
+        w = replace(base, feat_stride=base.feat_stride * p, feat_offset=(p - 1) / 2 * base.feat_stride)
+        ref = oracle.bridge(w, dict(batch, feat=oracle.pool(batch["feat"], p)))
+        br = b200.Bridge(b200.config_from_workload(w))
+        bufs = br.run(d["points"], d["proj"], pooled)
+        br.status()
+        for s in range(2):
+            M = ref[f"vox{s}"]["num_voxels"]
+            want, cnt = oracle.voxel_image(ref[f"vox{s}"]["point_voxel"], M, ref["vis_mask"], ref["gathered"])
+            assert int((cnt == 0).sum()) > 0 and int((cnt > 1).sum()) > 0
+            outs = {"pool, then sample per voxel": br.voxel_image_sampled(bufs["vox"], s, bufs["pg"]["uvd"],
+                                                                          bufs["pg"]["cam"], pooled),
+                    "pool, gather per point, then mean per voxel": br.voxel_image(bufs["vox"], s, bufs["pg"]["vis_mask"],
+                                                                                  bufs["pg"]["gathered"]),
+                    "pooling folded into the sampling": br0.voxel_image_pooled(raw["vox"], s, raw["pg"]["uvd"],
+                                                                               raw["pg"]["cam"], d["feat"], p)}
+            br.status()
+            br0.status()
+            for name, out in outs.items():
+                assert np.array_equal(np_(out["vox_img_count"])[:M], cnt), (name, s)
+                ok, mx, nbad = close(np_(out["vox_img"])[:M], want)
+                assert ok, f"{name}, scale {s}, p {p}: max abs err {mx}, {nbad} outside tolerance"
+                assert not np_(out["vox_img"])[:M][cnt == 0].any(), name
+        br.close()
+        br0.close()
+
+
 def test_per_voxel_fusion_rejects_counts_of_another_batch(b200, oracle):
     # counts that add up to more than the points would make the per-voxel lists overrun their array:
     # the scan sees it, nothing is written and the status says so
@@ -302,6 +356,33 @@ def test_per_voxel_fusion_rejects_counts_of_another_batch(b200, oracle):
     br.status()
     M = int(bufs["vox"]["num_voxels"][0].item())             # rows past the voxels found are not written
     assert torch.equal(again["vox_img_count"][:M], good["vox_img_count"][:M])
+    br.close()
+
+
+def test_per_voxel_fusion_with_counts_moved_between_voxels_reads_only_what_it_appended(b200, oracle):
+    # counts with the right total but the wrong voxels (another scale's, or a stale buffer): a voxel must not
+    # walk past the entries this call appended for it, so every row is a mean of rows of THIS batch
+    w = gen.KITTI.with_shape(1, 20_000)
+    batch = gen.make_batch(w)
+    br = b200.Bridge(b200.config_from_workload(w))
+    d = to_dev(batch)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    br.status()
+    pg = bufs["pg"]
+    pg["gathered"].fill_(1.0)                                # every row of this batch is all ones
+    M = int(bufs["vox"]["num_voxels"][0].item())
+    wrong = {k: v for k, v in bufs["vox"].items()}
+    moved = bufs["vox"]["counts"][0].clone()
+    moved[:M] = torch.roll(moved[:M], 1)                     # same sum, other voxels
+    wrong["counts"] = [moved, bufs["vox"]["counts"][1]]
+    for call in (lambda: br.voxel_image(wrong, 0, pg["vis_mask"], pg["gathered"]),):
+        out = call()
+        assert br.status(raise_on_error=False) == b200.bridge.EMC2_OK
+        rows = out["vox_img"][:M]
+        cnt = out["vox_img_count"][:M]
+        assert bool(torch.isfinite(rows).all())
+        seen = cnt > 0
+        assert bool((rows[seen] == 1.0).all()) and bool((rows[~seen] == 0.0).all())
     br.close()
 
 
