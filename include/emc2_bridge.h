@@ -381,6 +381,14 @@ typedef enum {
     EMC2_TUNE_MARK_IN_PROJECTION = 1, /* emc2_bridge_run: 1 (default) = the projection kernel also marks the
                                    voxel cells of both scales (one pass over the points fewer in stage 1);
                                    0 = stage 1 marks them in a pass of its own, beside the projection */
+    EMC2_TUNE_DEDUP_FINE = 2,    /* how the voxels of grid[0] are deduplicated and ranked: 0 (default) = a
+                                   direct-addressed cell store (one bit per cell) ranked by prefix sums;
+                                   1 = an open-addressing hash table in device memory, sized by the points,
+                                   whose unique cell ids are then radix-sorted into canonical order;
+                                   2 = a radix sort of every point's (cell id, index).  Same outputs.
+                                   Selecting 1 or 2 allocates that design's scratch (this call may allocate;
+                                   emc2_bridge_scratch_bytes then includes it) */
+    EMC2_TUNE_DEDUP_PILLARS = 3, /* the same choice for grid[1] (default 0 = a direct per-cell count table) */
     EMC2_TUNE_KNOBS
 } emc2_tuning_t;
 int emc2_bridge_set_tuning(emc2_bridge_t* bridge, int32_t knob, int32_t value);

@@ -42,7 +42,10 @@ ABI_SYMBOLS = (
 # emc2_tuning_t
 TUNE_ROW_STORE = 0
 TUNE_MARK_IN_PROJECTION = 1
-TUNE_NAMES = {"row_store": TUNE_ROW_STORE, "mark_in_projection": TUNE_MARK_IN_PROJECTION}
+TUNE_DEDUP_FINE = 2
+TUNE_DEDUP_PILLARS = 3
+TUNE_NAMES = {"row_store": TUNE_ROW_STORE, "mark_in_projection": TUNE_MARK_IN_PROJECTION,
+              "dedup_fine": TUNE_DEDUP_FINE, "dedup_pillars": TUNE_DEDUP_PILLARS}
 
 
 class Emc2Grid(ctypes.Structure):

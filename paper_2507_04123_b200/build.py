@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libemc2_bridge.so")
-SOURCES = ["bridge.cu", "voxelize.cu", "project_gather.cu", "route_dispatch.cu", "voxel_image.cu", "occlusion.cu", "rulebook.cu"]
+SOURCES = ["bridge.cu", "voxelize.cu", "project_gather.cu", "route_dispatch.cu", "voxel_image.cu", "occlusion.cu", "rulebook.cu", "dedup_arms.cu"]
 HEADERS = [os.path.join(CSRC, "bridge_internal.cuh"), os.path.join(ROOT, "include", "emc2_bridge.h")]
 
 

@@ -8,7 +8,7 @@
 namespace emc2 {
 
 static const char* const kKernelNames[K_KINDS] = {
-    "vox_mark", "vox_count", "vox_prefix", "vox_rank", "vox_accum", "vox_over_find", "vox_over_fill", "vox_finalize",
+    "vox_mark", "vox_count", "vox_prefix", "vox_rank", "vox_accum", "vox_over_find", "vox_over_fill", "vox_finalize", "arm_keys", "arm_sort", "arm_hash", "arm_rank",
     "project_gather", "project_route", "gather_scatter", "route_hist", "route_scan", "dispatch_scatter", "scene_route", "pool_features",
     "vif_scan", "vif_fill", "vif_mean", "vif_sample", "occl_fill", "occl_splat", "occl_test",
     "channels_last", "rb_mark", "rb_count", "rb_scan", "rb_fill", "rb_clear"};
@@ -152,6 +152,8 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
             d.div[k] = make_fast_div((uint32_t)g.dims[k]);
         }
         d.cap = g.max_points;
+        d.design = 0;
+        d.point_rank = nullptr;
         d.cells = (uint32_t)((uint64_t)g.dims[0] * g.dims[1] * g.dims[2]);
         const uint64_t total_cells = (uint64_t)d.cells * c.max_batch;
         d.mode = total_cells <= (uint64_t)kMaxTableCells ? MODE_TABLE : MODE_BITMAP;
@@ -520,8 +522,19 @@ int emc2_bridge_set_overlap(emc2_bridge_t* h, int enable) {
 
 int emc2_bridge_set_tuning(emc2_bridge_t* h, int32_t knob, int32_t value) {
     if (!h || knob < 0 || knob >= EMC2_TUNE_KNOBS) return EMC2_ERR_INVALID_ARG;
-    static const int kMaxValue[EMC2_TUNE_KNOBS] = {2, 1};
+    static const int kMaxValue[EMC2_TUNE_KNOBS] = {2, 1, 2, 2};
     if (value < 0 || value > kMaxValue[knob]) return EMC2_ERR_INVALID_ARG;
+    if (knob == EMC2_TUNE_DEDUP_FINE || knob == EMC2_TUNE_DEDUP_PILLARS) {
+        const int s = knob == EMC2_TUNE_DEDUP_FINE ? 0 : 1;
+        if (value != 0) {                         // the other designs bring scratch of their own
+            DeviceGuard guard(h->cfg.device);
+            if (!guard.ok) return EMC2_ERR_CUDA;
+            const int rc = dedup_arm_alloc(h);
+            if (rc != EMC2_OK) return rc;
+        }
+        h->scale[s].design = value;
+        h->scale[s].point_rank = value ? h->arm.point_rank[s] : nullptr;
+    }
     h->tune[knob] = value;
     return EMC2_OK;
 }
@@ -553,6 +566,7 @@ int emc2_bridge_destroy(emc2_bridge_t* h) {
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->side) cudaStreamDestroy(h->side);
     if (h->slab && cudaFree(h->slab) != cudaSuccess) rc = EMC2_ERR_CUDA;
+    if (h->arm.slab && cudaFree(h->arm.slab) != cudaSuccess) rc = EMC2_ERR_CUDA;
     delete h;
     return rc;
 }
@@ -572,7 +586,7 @@ const char* emc2_status_string(int status) {
 }
 
 int emc2_bridge_last_cuda_error(const emc2_bridge_t* h) { return h ? h->last_cuda_error : 0; }
-size_t emc2_bridge_scratch_bytes(const emc2_bridge_t* h) { return h ? h->slab_bytes : 0; }
+size_t emc2_bridge_scratch_bytes(const emc2_bridge_t* h) { return h ? h->slab_bytes + h->arm.bytes : 0; }
 
 int emc2_bridge_kernel_kinds(void) { return K_KINDS; }
 const char* emc2_bridge_kernel_name(int kind) { return kind >= 0 && kind < K_KINDS ? kKernelNames[kind] : ""; }

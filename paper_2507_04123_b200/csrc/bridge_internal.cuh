@@ -27,6 +27,10 @@ enum KernelKind {
     K_VOX_OVER_FIND,
     K_VOX_OVER_FILL,
     K_VOX_FINALIZE,
+    K_ARM_KEYS,
+    K_ARM_SORT,
+    K_ARM_HASH,
+    K_ARM_RANK,
     K_PROJECT_GATHER,
     K_PROJECT_ROUTE,
     K_GATHER_SCATTER,
@@ -101,6 +105,9 @@ struct ScaleDev {
     uint32_t* ovf_cell;     // per cell over the cap j: its cell id
     int* ovf_vox;           // per cell over the cap j: its row m in the unique list
     int* ovf_list;          // global point indices of the points in cells over the cap
+    int design;             // dedup design of this scale: 0 = this direct-addressed store, 1 = hash, 2 = sort
+                            // (dedup_arms.cu); with 1 or 2 the store is not used and rows come from point_rank
+    const int* point_rank;  // design != 0: [points of the call] row of every point's voxel, -1 if outside
     int* totals;            // [0] voxels, [1] cells over the cap, [2] points in cells over the cap, [3] CTAs of the rank scan that found voxels
 };
 
@@ -109,6 +116,22 @@ struct RouteParams {
     int T, E;
     float thr2[EMC2_MAX_THRESHOLDS];    // squared thresholds
     uint8_t lut[16];                    // [visible ? 8 : 0] + number of thresholds reached -> expert
+};
+
+// Scratch of the alternative dedup designs (allocated when one is first selected).
+struct DedupArm {
+    void* slab = nullptr;
+    size_t bytes = 0;
+    uint32_t* keys[2] = {nullptr, nullptr};     // sort buffers (ping-pong): cell ids ...
+    uint32_t* vals[2] = {nullptr, nullptr};     // ... and point indices (hash design: the unique ids)
+    int* counts = nullptr;                      // [256][tiles] digit counts of a radix pass
+    int* row_tot = nullptr;                     // [256] totals per digit
+    int* tile_tot = nullptr;                    // run heads per tile
+    int* point_rank[2] = {nullptr, nullptr};    // per scale
+    uint32_t* tab_keys = nullptr;               // hash table: cell ids ...
+    int* tab_rows = nullptr;                    // ... and their rows
+    int* d_total = nullptr;
+    uint32_t slots = 0;
 };
 
 struct ProfRec {
@@ -140,7 +163,8 @@ struct emc2_bridge {
     int* d_rb_counts = nullptr;    // [27][voxel tiles] pairs per (offset, tile), and their prefix sums
     int* d_rb_base = nullptr;
     int max_tiles = 0;
-    int tune[EMC2_TUNE_KNOBS] = {0, 1};   // emc2_bridge_set_tuning
+    int tune[EMC2_TUNE_KNOBS] = {0, 1, 0, 0};   // emc2_bridge_set_tuning
+    emc2::DedupArm arm;
     int num_sms = 0;               // multiprocessors of the handle's device
     bool overlap = true;           // emc2_bridge_run puts stage 1 on `side`
     cudaStream_t side = nullptr;   // stream of stage 1 inside emc2_bridge_run
@@ -173,6 +197,9 @@ int launch_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t
                     int32_t* const d_counts[2], float* const d_mean[2], int32_t* const d_point_voxel[2],
                     const int32_t capacity[2], int32_t* d_num_voxels, float* d_bev, cudaStream_t st,
                     bool marked = false);
+int dedup_arm_alloc(emc2_bridge* h);
+int launch_dedup_arm(emc2_bridge* h, int s, int design, int B, int N, const float* d_points, int capacity,
+                     int32_t* d_num_voxels, cudaStream_t st);
 int launch_project_gather(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj,
                           const float* d_feat, float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam,
                           float* d_gathered, cudaStream_t st);
@@ -254,6 +281,7 @@ __device__ __forceinline__ void mark_point(const ScaleDev& s0, const ScaleDev& s
 #pragma unroll
     for (int sc = 0; sc < 2; ++sc) {
         const ScaleDev& g = sc ? s1 : s0;
+        if (g.design) continue;                   // another dedup design: no store to mark
         const uint32_t cell = cell_of(g, x, y, z, b);
         if (cell == 0xFFFFFFFFu) continue;
         // Results unused: these compile to reductions, which the thread does not wait for.

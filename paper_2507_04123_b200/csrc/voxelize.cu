@@ -44,10 +44,14 @@ struct Slot {
     int j;      // rank among cells over the cap, -1 if the cell is not over it
 };
 
-__device__ __forceinline__ Slot slot_of(const ScaleDev& g, uint32_t cell) {
+__device__ __forceinline__ Slot slot_of(const ScaleDev& g, uint32_t cell, long long point) {
     Slot s;
     s.m = -1; s.j = -1;
     if (cell == 0xFFFFFFFFu) return s;
+    if (g.design) {                               // hash / sort design: the row was computed per point
+        s.m = g.point_rank[point];
+        return s;
+    }
     if (g.mode == MODE_BITMAP) {
         const uint2 pr = *reinterpret_cast<const uint2*>(g.store + 2 * (size_t)(cell >> 5));
         s.m = (int)(pr.y + __popc(pr.x & ((1u << (cell & 31u)) - 1u)));
@@ -276,6 +280,7 @@ __global__ void __launch_bounds__(kPrefixThreads) vox_prefix_kernel(ScanArgs a) 
     __shared__ int tot[4];
     const int sc = blockIdx.x;
     const ScaleDev& g = a.s[sc];
+    if (g.design) return;                         // ranked by another design: its totals stand
     const int first = sc ? a.ctas0 : 0, n = sc ? a.ctas1 : a.ctas0;
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int per = (n + kPrefixThreads - 1) / kPrefixThreads;
@@ -437,7 +442,7 @@ vox_accum_kernel(const float* __restrict__ pts, long long total, int N, AccumArg
                     cx[sc][i] = ix; cy[sc][i] = iy; cz[sc][i] = iz;
                 }
             }
-            slot[sc][i] = slot_of(g, cell);
+            slot[sc][i] = slot_of(g, cell, g0 + t);
         }
     }
 #pragma unroll
@@ -519,7 +524,7 @@ vox_over_fill_kernel(const float* __restrict__ pts, long long total, int N, Accu
     const ScaleDev& g = a.s[sc];
     for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < total; i += (long long)gridDim.x * kThreads) {
         const float* p = pts + i * C;
-        const Slot s = slot_of(g, cell_of(g, p[0], p[1], p[2], (int)(i / N)));
+        const Slot s = slot_of(g, cell_of(g, p[0], p[1], p[2], (int)(i / N)), i);
         if (s.m < 0 || s.m >= a.capacity[sc]) continue;
         const uint32_t tag = reinterpret_cast<const uint32_t*>(g.acc + 2 * (size_t)s.m + 1)[2];
         if (tag == 0u || tag > g.max_ovf) continue;
@@ -671,7 +676,7 @@ vox_finalize_kernel(const float* __restrict__ pts, long long total, AccumArgs a,
         const ScaleDev& g = a.s[sc];
         const int n = min(32, (sc ? tot1 : tot0) - mb);
         const uint32_t entry = lane < n ? g.cell_list[mb + lane] : 0u;
-        if (lane < n) {
+        if (lane < n && !g.design) {
             if (g.mode == MODE_BITMAP) {
                 uint4* sp = reinterpret_cast<uint4*>(g.store + 8 * (size_t)(entry >> 7));
                 sp[0] = make_uint4(0u, 0u, 0u, 0u);
@@ -695,8 +700,11 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
     bool any_cap = false;
     for (int s = 0; s < 2; ++s) {
         sa.s[s] = h->scale[s];
-        aa.s[s] = h->scale[s];
-        const uint64_t cells = (uint64_t)B * h->scale[s].cells;
+        // A scale deduplicated by the hash or sort design has no store to scan; its voxel list is a plain
+        // list of cell ids, which the later passes treat like a bitmap scale's.
+        if (sa.s[s].design) sa.s[s].mode = MODE_BITMAP;
+        aa.s[s] = sa.s[s];
+        const uint64_t cells = sa.s[s].design ? 0 : (uint64_t)B * h->scale[s].cells;
         const uint64_t per_group = h->scale[s].mode == MODE_BITMAP ? kBitmapGroupCells : kTableGroupCells;
         sa.ngroups_used[s] = aa.ngroups_used[s] = (uint32_t)((cells + per_group - 1) / per_group);
         sa.capacity[s] = aa.capacity[s] = capacity[s];
@@ -728,6 +736,11 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
                                                            bev_vec ? bev_n >> 2 : 0);
         }
     }
+    for (int s = 0; s < 2; ++s) {
+        if (!h->scale[s].design) continue;
+        const int rc = launch_dedup_arm(h, s, h->scale[s].design, B, N, d_points, capacity[s], d_num_voxels, st);
+        if (rc != EMC2_OK) return rc;
+    }
     if (sa.ctas0 + sa.ctas1 > 0) {
         LaunchScope ls(h, K_VOX_COUNT, st);
         vox_count_kernel<<<sa.ctas0 + sa.ctas1, kThreads, 0, st>>>(sa);
@@ -745,7 +758,7 @@ int run_voxelize(emc2_bridge* h, int B, int N, const float* d_points, int32_t* c
         vox_accum_kernel<C><<<ptiles, kThreads, 0, st>>>(d_points, total, N, aa);
     }
     for (int s = 0; s < 2 && total > 0; ++s) {
-        if (h->scale[s].mode != MODE_BITMAP || h->scale[s].cap <= 0) continue;
+        if (aa.s[s].mode != MODE_BITMAP || h->scale[s].cap <= 0) continue;
         {
             LaunchScope ls(h, K_VOX_OVER_FIND, st);
             vox_over_find_kernel<<<4 * h->num_sms, kThreads, 0, st>>>(aa, s);
