@@ -76,6 +76,27 @@ def one_call_bytes(w, B, N, m0, m1, texels):
     return staged["voxelize"] + proj + kernel_bytes(w, B, N, texels)["gather_scatter"] + B * (w.num_experts + 1) * 4
 
 
+def bridge_fractions(own_bytes, staged_bytes, ms_step, staged_ms, peak, peak_kind):
+    """The bandwidth figures of the bench line.  Every time is paired with the bytes that path moves: the
+    one-call step with the one-call byte count (the headline), the three stage calls with the staged count.
+    The staged count over the one-call time is kept under a name that says what it is."""
+    own_gbs = own_bytes / (ms_step * 1e-3) / 1e9
+    staged_gbs = staged_bytes / (staged_ms * 1e-3) / 1e9
+    equiv_gbs = staged_bytes / (ms_step * 1e-3) / 1e9
+    return {
+        "one_call_bytes_per_step": own_bytes,
+        "bridge_own_gbs": own_gbs,
+        "bridge_frac_of_8tbs_own_bytes": own_gbs / NOMINAL_HBM_GBS,
+        f"bridge_frac_of_{peak_kind}_copy_own_bytes": own_gbs / peak,
+        "target_50pct_of_8tbs_met": bool(own_gbs / NOMINAL_HBM_GBS >= 0.5),
+        "staged_path": {"ms_per_step": staged_ms, "gbs": staged_gbs, "frac_of_8tbs": staged_gbs / NOMINAL_HBM_GBS,
+                        f"frac_of_{peak_kind}_copy": staged_gbs / peak},
+        "equivalent_staged_bandwidth": {"gbs": equiv_gbs, "frac_of_8tbs": equiv_gbs / NOMINAL_HBM_GBS,
+                                        "note": "bytes of the three stage calls divided by the one-call time; "
+                                                "the one-call path does not move all of them"},
+    }
+
+
 def distinct_texels(w, pg):
     """Distinct feature texels the gather touches, from the library's own uvd/cam outputs."""
     uvd, cam = pg["uvd"], pg["cam"]
@@ -447,10 +468,7 @@ def run_ours(args, w):
     ms_step = secs / args.steps * 1e3
     fps = world * B * args.steps / secs
     own_bytes = one_call_bytes(w, B, N, int(nv[0]), int(nv[1]), texels)
-    own_gbs = own_bytes / (ms_step * 1e-3) / 1e9          # bytes the one-call path moves over its own time
     staged_ms = staged_secs / args.steps * 1e3
-    staged_gbs = abytes["total"] / (staged_ms * 1e-3) / 1e9   # bytes of the three calls over their own time
-    equiv_gbs = abytes["total"] / (ms_step * 1e-3) / 1e9  # staged byte count over the one-call time
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         times = oracle_rate(w, target_s=12.0)
@@ -473,17 +491,8 @@ def run_ours(args, w):
         "graph_ms_per_step": graph_secs / args.steps * 1e3 if graph_secs is not None else None,
         "repeats": {"regions": len(regions), "ms_per_step_min": min(regions) / args.steps * 1e3,
                     "ms_per_step_median": ms_step, "ms_per_step_max": max(regions) / args.steps * 1e3},
-        "one_call_bytes_per_step": own_bytes,
-        "bridge_own_gbs": own_gbs,
-        "bridge_frac_of_8tbs_own_bytes": own_gbs / NOMINAL_HBM_GBS,
-        f"bridge_frac_of_{peak_kind}_copy_own_bytes": own_gbs / peak,
-        "target_50pct_of_8tbs_met": bool(own_gbs / NOMINAL_HBM_GBS >= 0.5),
+        **bridge_fractions(own_bytes, abytes["total"], ms_step, staged_ms, peak, peak_kind),
         "bridge_algorithmic_bytes_per_step": abytes,
-        "staged_path": {"ms_per_step": staged_ms, "gbs": staged_gbs, "frac_of_8tbs": staged_gbs / NOMINAL_HBM_GBS,
-                        f"frac_of_{peak_kind}_copy": staged_gbs / peak},
-        "equivalent_staged_bandwidth": {"gbs": equiv_gbs, "frac_of_8tbs": equiv_gbs / NOMINAL_HBM_GBS,
-                                        "note": "bytes of the three stage calls divided by the one-call time; "
-                                                "the one-call path does not move all of them"},
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_source": peak_kind,
                      "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "traffic_stale": traffic_stale,
                      "algorithmic_bytes_per_launch": kb[dom], "ms_per_launch": dom_ms},
@@ -496,6 +505,12 @@ def run_ours(args, w):
         "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
         "unique_voxels": [int(nv[0]), int(nv[1])], "distinct_texels": texels,
     }
+    if w.config_id == 2 and world == 1 and not args.no_other_workloads and args.pool <= 1 and not args.batch \
+            and not args.points:
+        # The KITTI-shaped batch and the dense frame, briefly (same call, same tuning), so that their numbers
+        # are in the same record as the headline workload's.
+        line["other_workloads"] = {gen.workload(c).name: short_run(pkg, gen.workload(c), local_rank, args.tune)
+                                   for c in (1, 3)}
     if args.tune:
         line["tuning"] = {k: v for k, v in args.tune}
     if timeline:
@@ -604,6 +619,30 @@ def run_ours(args, w):
     print(json.dumps(line), flush=True)
     if use_dist:
         dist.destroy_process_group()
+
+
+def short_run(pkg, w, device, tune, steps=20, repeats=3):
+    """One-call step time and own-byte fraction of another workload (no staged, host-buffer or CPU legs)."""
+    dev = torch.device("cuda", device)
+    batch = gen.make_batch(w)
+    d = {k: torch.from_numpy(v).to(dev) for k, v in batch.items()}
+    br = make_bridge(pkg, w, device, tune)
+    bufs = br.run(d["points"], d["proj"], d["feat"])
+    br.status()
+    nv = bufs["vox"]["num_voxels"].cpu().numpy()
+    own = one_call_bytes(w, w.B, w.N, int(nv[0]), int(nv[1]), distinct_texels(w, bufs["pg"]))
+    step = lambda: br.run(d["points"], d["proj"], d["feat"], bufs)
+    for _ in range(5):
+        step()
+    sync = lambda: torch.cuda.synchronize(dev)
+    regions = [time_steps(step, steps, sync, lambda: None) for _ in range(repeats)]
+    br.status()
+    br.close()
+    ms = float(np.median(regions)) / steps * 1e3
+    gbs = own / (ms * 1e-3) / 1e9
+    return {"frames_per_step": w.B, "points_per_frame": w.N, "ms_per_step": ms, "frames_per_s": w.B / (ms * 1e-3),
+            "mpoints_per_s": w.B * w.N / (ms * 1e-3) / 1e6, "one_call_bytes_per_step": own, "own_gbs": gbs,
+            "frac_of_8tbs_own_bytes": gbs / NOMINAL_HBM_GBS, "steps": steps, "regions": repeats}
 
 
 def run_sweep(args):

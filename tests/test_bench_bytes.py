@@ -39,3 +39,19 @@ def test_distinct_texels_counts_shared_taps_once():
     cam = torch.tensor([[0, 0, 0, -1]], dtype=torch.int8)
     # points 0 and 1 use texels (0..1, 0..1); point 2 uses (2..3, 0..1); the last point sees no camera
     assert bench.distinct_texels(w, {"uvd": uvd, "cam": cam}) == 8
+
+
+def test_every_bandwidth_figure_pairs_a_time_with_the_bytes_that_path_moves():
+    # 1,000 MB in 0.25 ms is 4,000 GB/s: half of 8 TB/s.  The staged count (1,400 MB) only counts against the
+    # staged time; over the one-call time it appears under a name that says so and is not the headline.
+    f = bench.bridge_fractions(own_bytes=1_000_000_000, staged_bytes=1_400_000_000, ms_step=0.25, staged_ms=0.4,
+                               peak=6500.0, peak_kind="measured")
+    assert f["one_call_bytes_per_step"] == 1_000_000_000
+    assert abs(f["bridge_own_gbs"] - 4000.0) < 1e-6
+    assert abs(f["bridge_frac_of_8tbs_own_bytes"] - 0.5) < 1e-12 and f["target_50pct_of_8tbs_met"] is True
+    assert abs(f["bridge_frac_of_measured_copy_own_bytes"] - 4000.0 / 6500.0) < 1e-12
+    assert abs(f["staged_path"]["gbs"] - 3500.0) < 1e-6 and abs(f["staged_path"]["frac_of_8tbs"] - 0.4375) < 1e-12
+    assert abs(f["equivalent_staged_bandwidth"]["frac_of_8tbs"] - 0.7) < 1e-12
+    assert "bridge_frac_of_8tbs" not in f and "bridge_gbs" not in f        # the ambiguous names are gone
+    slower = bench.bridge_fractions(1_000_000_000, 1_400_000_000, 0.26, 0.4, 6500.0, "measured")
+    assert slower["target_50pct_of_8tbs_met"] is False
