@@ -659,17 +659,20 @@ def run_sweep(args):
             bufs = br.run(d["points"], d["proj"], d["feat"])
             br.status()
             nv = bufs["vox"]["num_voxels"].cpu().numpy()
-            ab = algorithmic_bytes(w, B, N, int(nv[0]), int(nv[1]), distinct_texels(w, bufs["pg"]))
+            tex = distinct_texels(w, bufs["pg"])
+            ab = algorithmic_bytes(w, B, N, int(nv[0]), int(nv[1]), tex)
+            own = one_call_bytes(w, B, N, int(nv[0]), int(nv[1]), tex)
             step = lambda: br.run(d["points"], d["proj"], d["feat"], bufs)
             for _ in range(5):
                 step()
             steps = 20 if B * N < 4_000_000 else 8
             secs = time_steps(step, steps, lambda: torch.cuda.synchronize(dev), lambda: None)
             ms = secs / steps * 1e3
-            gbs = ab["total"] / (ms * 1e-3) / 1e9
+            gbs = own / (ms * 1e-3) / 1e9                   # the bytes the one-call path moves over its time
             rows.append({"N": N, "B": B, "ms_per_step": ms, "frames_per_s": B / (ms * 1e-3),
-                         "mpoints_per_s": B * N / (ms * 1e-3) / 1e6, "gbs": gbs, "frac_of_8tbs": gbs / NOMINAL_HBM_GBS,
-                         "bytes_per_point": ab["total"] / (B * N)})
+                         "mpoints_per_s": B * N / (ms * 1e-3) / 1e6, "own_gbs": gbs,
+                         "frac_of_8tbs_own_bytes": gbs / NOMINAL_HBM_GBS, "own_bytes_per_point": own / (B * N),
+                         "staged_bytes_per_point": ab["total"] / (B * N)})
             br.close()
             del d, bufs
             torch.cuda.empty_cache()

@@ -115,7 +115,11 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out);
  *   d_num_voxels     int32 [2]               number of unique voxels found per scale (true count
  *                                            even when it exceeds capacity[s])
  *   d_bev            float [B, C, Gy, Gx] of grid[1], or NULL: pillar means at (iy, ix), else 0
- * d_points is float [B, N, C].  Rows past num_voxels are left untouched.  If a scale finds more
+ * d_points is float [B, N, C].  Rows past num_voxels are left untouched.  All integer outputs
+ * (coordinates, counts, point rows, the number of voxels) are the same on every run; the means
+ * and the BEV image are sums of fp32 reductions whose order is not fixed, so they are
+ * reproducible to the comparison tolerance (1e-4 + 1e-5 |x|), not bit for bit.  The same holds
+ * for the rows of emc2_voxel_image and its variants.  If a scale finds more
  * voxels than capacity[s], rows past capacity are not written and EMC2_ERR_CAPACITY becomes
  * sticky.  d_coords, d_counts, d_mean and capacity are HOST arrays of two entries. */
 int emc2_voxelize(emc2_bridge_t* bridge, int32_t B, int32_t N, const float* d_points,
