@@ -381,7 +381,9 @@ typedef enum {
     EMC2_TUNE_ROW_STORE = 0,    /* how the one-call path stores feature rows: 0 = 128-bit stores from
                                    registers; 1 = rows staged in shared memory, ordered by expert, and written
                                    with bulk asynchronous copies (cp.async.bulk), both destinations; 2 = bulk
-                                   copies for the dispatched rows only */
+                                   copies for the dispatched rows only; 3 = 256-bit loads and stores
+                                   (eight channels per thread; needs feat_c % 8 == 0 and 32-byte aligned
+                                   buffers, else falls back to 0) */
     EMC2_TUNE_MARK_IN_PROJECTION = 1, /* emc2_bridge_run: 1 (default) = the projection kernel also marks the
                                    voxel cells of both scales (one pass over the points fewer in stage 1);
                                    0 = stage 1 marks them in a pass of its own, beside the projection */

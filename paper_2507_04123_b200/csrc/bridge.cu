@@ -522,7 +522,7 @@ int emc2_bridge_set_overlap(emc2_bridge_t* h, int enable) {
 
 int emc2_bridge_set_tuning(emc2_bridge_t* h, int32_t knob, int32_t value) {
     if (!h || knob < 0 || knob >= EMC2_TUNE_KNOBS) return EMC2_ERR_INVALID_ARG;
-    static const int kMaxValue[EMC2_TUNE_KNOBS] = {2, 1, 2, 2};
+    static const int kMaxValue[EMC2_TUNE_KNOBS] = {3, 1, 2, 2};
     if (value < 0 || value > kMaxValue[knob]) return EMC2_ERR_INVALID_ARG;
     if (knob == EMC2_TUNE_DEDUP_FINE || knob == EMC2_TUNE_DEDUP_PILLARS) {
         const int s = knob == EMC2_TUNE_DEDUP_FINE ? 0 : 1;

@@ -244,6 +244,13 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) gather_scatter_
     const size_t f0 = (size_t)b * a.N;        // first row of the frame
     const size_t g0 = f0 + i0;
     const int cf4 = CF4 > 0 ? CF4 : a.cf4;
+    // The tile's bases are requested first, together with the points' records: nothing below waits for
+    // a second round trip to memory before the rows start to move.
+    __shared__ int tbase[EMC2_MAX_EXPERTS];
+    if (t >= (int)blockDim.x - EMC2_MAX_EXPERTS) {
+        const int k = t - ((int)blockDim.x - EMC2_MAX_EXPERTS);
+        if (k < a.E) tbase[k] = a.tile_base[((size_t)b * a.tiles + tile) * a.E + k];
+    }
 
     // Stable rank inside the tile by ballots per expert, and the tap record of every point.
     int e = -1, rank = 0;
@@ -263,7 +270,7 @@ __global__ void __launch_bounds__(CF4 > 0 ? 16 * CF4 : kThreads) gather_scatter_
     if (t < npts) {
         int before = 0;
         for (int w = 0; w < warp; ++w) before += wcnt[w][e];
-        const int d = a.tile_base[((size_t)b * a.tiles + tile) * a.E + e] + before + rank;
+        const int d = tbase[e] + before + rank;
         sdest[t] = d;
         a.perm[f0 + d] = i0 + t;
     }
@@ -341,6 +348,11 @@ __global__ void __launch_bounds__(16 * CF4) gather_scatter_bulk_kernel(const __g
     const int npts = min(kTile, a.N - i0);
     const size_t f0 = (size_t)b * a.N;
     const size_t g0 = f0 + i0;
+    __shared__ int tbase[EMC2_MAX_EXPERTS];
+    if (t >= (int)blockDim.x - EMC2_MAX_EXPERTS) {
+        const int k = t - ((int)blockDim.x - EMC2_MAX_EXPERTS);
+        if (k < a.E) tbase[k] = a.tile_base[((size_t)b * a.tiles + tile) * a.E + k];
+    }
 
     int e = -1, rank = 0;
     if (t < kTile) {
@@ -360,7 +372,7 @@ __global__ void __launch_bounds__(16 * CF4) gather_scatter_bulk_kernel(const __g
         int before = 0, below = 0;
         for (int w = 0; w < warp; ++w) before += wcnt[w][e];
         for (int k = 0; k < e; ++k) below += wcnt[warp][k];
-        const int d = a.tile_base[((size_t)b * a.tiles + tile) * a.E + e] + before + rank;
+        const int d = tbase[e] + before + rank;
         sdest[t] = d;
         spos[t] = (uint8_t)(below + rank);
         a.perm[f0 + d] = i0 + t;
@@ -369,7 +381,7 @@ __global__ void __launch_bounds__(16 * CF4) gather_scatter_bulk_kernel(const __g
         const int w = t / a.E, k = t - w * a.E;
         int before = 0;
         for (int w2 = 0; w2 < w; ++w2) before += wcnt[w2][k];
-        wrow[w][k] = a.tile_base[((size_t)b * a.tiles + tile) * a.E + k] + before;
+        wrow[w][k] = tbase[k] + before;
     }
     __syncthreads();
 
@@ -422,6 +434,105 @@ __global__ void __launch_bounds__(16 * CF4) gather_scatter_bulk_kernel(const __g
     if (warp == 0) bulk_wait_read<0>();                   // shared memory must outlive the copies that read it
 }
 
+// ---- the same pass with 256-bit accesses (sm_100: ld/st.global.v8.f32)
+// A thread owns eight channels of a row instead of four: half as many load and store instructions
+// (and requests into the SM's memory pipeline) per byte moved, 32 rows x Cf/8 columns per round.
+// Needs Cf a multiple of 8 and 32-byte aligned maps and row buffers (checked at launch).
+struct F8 { float v[8]; };
+
+__device__ __forceinline__ F8 ldg8(const float* p) {
+    F8 r;
+    asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])
+                 : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void stcs8(float* p, const F8& r) {
+    asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
+                 : "memory");
+}
+
+// Blended channels [8c, 8c + 8) of the row described by `rec` (zeros for kZeroRow); same arithmetic as blend().
+__device__ __forceinline__ F8 gather_column8(const float* __restrict__ feat, const uint4& rec, int c, uint32_t cf4,
+                                             uint32_t row_stride) {
+    F8 o;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) o.v[k] = 0.f;
+    if (rec.x != kZeroRow) {
+        const float* p = feat + ((size_t)rec.x << 2) + 8 * c;
+        const size_t dx = (rec.y & 1u) ? (size_t)cf4 * 4 : 0, dy = (rec.y & 2u) ? (size_t)row_stride * 4 : 0;
+        const F8 f00 = ldg8(p), f01 = ldg8(p + dx), f10 = ldg8(p + dy), f11 = ldg8(p + dy + dx);
+        const float wx = __uint_as_float(rec.z), wy = __uint_as_float(rec.w);
+        const float ax = 1.0f - wx, ay = 1.0f - wy;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            o.v[k] = ay * (ax * f00.v[k] + wx * f01.v[k]) + wy * (ax * f10.v[k] + wx * f11.v[k]);
+    }
+    return o;
+}
+
+template <int C, int CF8>
+__global__ void __launch_bounds__(32 * CF8) gather_scatter_wide_kernel(const __grid_constant__ GsArgs a) {
+    __shared__ uint4 srow[kTile];
+    __shared__ int sdest[kTile];
+    __shared__ int wcnt[kTile / 32][EMC2_MAX_EXPERTS];
+    __shared__ int tbase[EMC2_MAX_EXPERTS];
+    const int b = blockIdx.y, tile = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int i0 = tile * kTile;
+    const int npts = min(kTile, a.N - i0);
+    const size_t f0 = (size_t)b * a.N;
+    const size_t g0 = f0 + i0;
+    constexpr int CF4 = 2 * CF8;
+    if (t >= (int)blockDim.x - EMC2_MAX_EXPERTS) {
+        const int k = t - ((int)blockDim.x - EMC2_MAX_EXPERTS);
+        if (k < a.E) tbase[k] = a.tile_base[((size_t)b * a.tiles + tile) * a.E + k];
+    }
+    int e = -1, rank = 0;
+    if (t < kTile) {
+        if (t < npts) {
+            e = (int)a.expert[g0 + t];
+            const float u = a.uvd[(g0 + t) * 3], v = a.uvd[(g0 + t) * 3 + 1];
+            srow[t] = tap_record(b, (int)a.cam[g0 + t], u, v, a.K, a.Hf, a.Wf, CF4, a.inv_stride, a.offset);
+        }
+        for (int k = 0; k < a.E; ++k) {
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, e == k);
+            if (e == k) rank = __popc(m & ((1u << lane) - 1u));
+            if (lane == 0) wcnt[warp][k] = __popc(m);
+        }
+    }
+    __syncthreads();
+    if (t < npts) {
+        int before = 0;
+        for (int w = 0; w < warp; ++w) before += wcnt[w][e];
+        const int d = tbase[e] + before + rank;
+        sdest[t] = d;
+        a.perm[f0 + d] = i0 + t;
+    }
+    __syncthreads();
+    const float* psrc = a.pts + g0 * C;
+    float* pdst = a.pts_out + f0 * C;
+    for (int i = t; i < npts * C; i += blockDim.x) {
+        const int r = i / C, c = i - r * C;
+        pdst[(size_t)sdest[r] * C + c] = __ldg(psrc + i);
+    }
+    const bool keep = a.gathered != nullptr;
+    float* out = reinterpret_cast<float*>(a.gathered) + g0 * (size_t)(8 * CF8);
+    float* fdst = reinterpret_cast<float*>(a.feat_out) + f0 * (size_t)(8 * CF8);
+    const float* feat = reinterpret_cast<const float*>(a.feat);
+    const uint32_t dyv = (uint32_t)a.Wf * CF4;
+    const int c = t % CF8, r0 = t / CF8;
+#pragma unroll 2
+    for (int j = 0; j < kTile / 32; ++j) {
+        const int r = r0 + 32 * j;
+        if (r >= npts) break;
+        const F8 o = gather_column8(feat, srow[r], c, (uint32_t)CF4, dyv);
+        if (keep) stcs8(out + (size_t)r * (8 * CF8) + 8 * c, o);
+        stcs8(fdst + (size_t)sdest[r] * (8 * CF8) + 8 * c, o);
+    }
+}
+
+
 template <int C>
 void launch_gs(emc2_bridge* h, const GsArgs& a, dim3 grid, cudaStream_t st) {
     LaunchScope ls(h, K_GATHER_SCATTER, st);
@@ -429,6 +540,10 @@ void launch_gs(emc2_bridge* h, const GsArgs& a, dim3 grid, cudaStream_t st) {
     if (mode == 1 && a.E < 31) {
         if (a.cf4 == 16) { gather_scatter_bulk_kernel<C, 16, true><<<grid, 16 * 16, 0, st>>>(a); return; }
         if (a.cf4 == 20) { gather_scatter_bulk_kernel<C, 20, true><<<grid, 16 * 20, 0, st>>>(a); return; }
+    } else if (mode == 3 && ((reinterpret_cast<uintptr_t>(a.feat) | reinterpret_cast<uintptr_t>(a.gathered) |
+                              reinterpret_cast<uintptr_t>(a.feat_out)) & 31) == 0) {
+        if (a.cf4 == 16) { gather_scatter_wide_kernel<C, 8><<<grid, 32 * 8, 0, st>>>(a); return; }
+        if (a.cf4 == 20) { gather_scatter_wide_kernel<C, 10><<<grid, 32 * 10, 0, st>>>(a); return; }
     } else if (mode == 2) {
         if (a.cf4 == 16) { gather_scatter_bulk_kernel<C, 16, false><<<grid, 16 * 16, 0, st>>>(a); return; }
         if (a.cf4 == 20) { gather_scatter_bulk_kernel<C, 20, false><<<grid, 16 * 20, 0, st>>>(a); return; }

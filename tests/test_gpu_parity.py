@@ -47,7 +47,7 @@ def test_ragged_shapes(b200, oracle, B, N):
         run_case(b200, oracle, base.with_shape(B, N), repeat=2, staged=(N % 2 == 0))
 
 
-TUNINGS = [(("row_store", 0),), (("row_store", 1),), (("row_store", 2),), (("mark_in_projection", 0),),
+TUNINGS = [(("row_store", 0),), (("row_store", 1),), (("row_store", 2),), (("row_store", 3),), (("mark_in_projection", 0),),
            (("mark_in_projection", 1),), (("dedup_fine", 1),), (("dedup_fine", 2),), (("dedup_pillars", 1),),
            (("dedup_pillars", 2),), (("dedup_fine", 2), ("dedup_pillars", 1)), (("dedup_fine", 1), ("dedup_pillars", 2))]
 
