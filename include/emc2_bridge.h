@@ -395,6 +395,10 @@ typedef enum {
                                    Selecting 1 or 2 allocates that design's scratch (this call may allocate;
                                    emc2_bridge_scratch_bytes then includes it) */
     EMC2_TUNE_DEDUP_PILLARS = 3, /* the same choice for grid[1] (default 0 = a direct per-cell count table) */
+    EMC2_TUNE_SPLIT_BATCH = 4,   /* emc2_bridge_run with the side stream and B >= 2: 1 = the batch is
+                                   projected in two halves, the second on the side stream beside the row
+                                   pass of the first; 0 (default) = all frames are projected before any row
+                                   moves */
     EMC2_TUNE_KNOBS
 } emc2_tuning_t;
 int emc2_bridge_set_tuning(emc2_bridge_t* bridge, int32_t knob, int32_t value);

@@ -44,8 +44,9 @@ TUNE_ROW_STORE = 0
 TUNE_MARK_IN_PROJECTION = 1
 TUNE_DEDUP_FINE = 2
 TUNE_DEDUP_PILLARS = 3
+TUNE_SPLIT_BATCH = 4
 TUNE_NAMES = {"row_store": TUNE_ROW_STORE, "mark_in_projection": TUNE_MARK_IN_PROJECTION,
-              "dedup_fine": TUNE_DEDUP_FINE, "dedup_pillars": TUNE_DEDUP_PILLARS}
+              "dedup_fine": TUNE_DEDUP_FINE, "dedup_pillars": TUNE_DEDUP_PILLARS, "split_batch": TUNE_SPLIT_BATCH}
 
 
 class Emc2Grid(ctypes.Structure):

@@ -229,6 +229,7 @@ int emc2_bridge_create(const emc2_config_t* config, emc2_bridge_t** out) {
     if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, prio_hi);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_half, cudaEventDisableTiming);
     if (e != cudaSuccess) { emc2_bridge_destroy(h); return EMC2_ERR_CUDA; }
     *out = h;
     return EMC2_OK;
@@ -335,22 +336,40 @@ int emc2_bridge_run(emc2_bridge_t* h, int32_t B, int32_t N, const float* d_point
     // One pass over the points serves the projection, the routing and the voxelizer's marking; the
     // rest of stage 1 then runs on the side stream beside the row traffic of stages 2 - 4.
     const bool fused_mark = rc2 == EMC2_OK && B > 0 && N > 0 && h->tune[EMC2_TUNE_MARK_IN_PROJECTION] != 0;
+    // With two or more frames the batch is taken in two halves: the rows of the first half start to
+    // move as soon as ITS points are projected, while the second half is projected on the side stream.
+    const int half0 = fused_mark && h->overlap && B >= 2 && h->tune[EMC2_TUNE_SPLIT_BATCH] != 0 ? B / 2 : B;
     if (fused_mark)
-        rc = launch_project_route(h, B, N, d_points, d_proj, d_uvd, d_vis_mask, d_cam, d_expert, true, d_bev, st);
+        rc = launch_project_route(h, 0, half0, N, d_points, d_proj, d_uvd, d_vis_mask, d_cam, d_expert, true, d_bev, B, st);
     if (rc == EMC2_OK && h->overlap) {
         e = cudaEventRecord(h->ev_fork, st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(h->side, h->ev_fork, 0);
         if (e != cudaSuccess) return check_cuda(h, e);
+    }
+    if (rc == EMC2_OK && half0 < B) {
+        rc = launch_project_route(h, half0, B - half0, N, d_points, d_proj, d_uvd, d_vis_mask, d_cam, d_expert, true,
+                                  nullptr, 0, h->side);
+        if (rc == EMC2_OK) {
+            e = cudaEventRecord(h->ev_half, h->side);
+            if (e != cudaSuccess) rc = check_cuda(h, e);
+        }
     }
     if (rc == EMC2_OK)
         rc = launch_voxelize(h, B, N, d_points, d_coords, d_counts, d_mean, d_point_voxel, capacity, d_num_voxels,
                              d_bev, vox_st, fused_mark);
     if (rc == EMC2_OK && rc2 == EMC2_OK && B > 0) {
         if (!fused_mark)
-            rc2 = launch_project_route(h, B, N, d_points, d_proj, d_uvd, d_vis_mask, d_cam, d_expert, false, nullptr, st);
+            rc2 = launch_project_route(h, 0, B, N, d_points, d_proj, d_uvd, d_vis_mask, d_cam, d_expert, false, nullptr, 0, st);
         if (rc2 == EMC2_OK)
-            rc2 = launch_scan_gather_scatter(h, B, N, d_points, d_feat, d_uvd, d_cam, d_gathered, d_expert, d_offsets,
-                                             d_perm, d_points_out, d_feat_out, st);
+            rc2 = launch_scan_gather_scatter(h, 0, half0, N, d_points, d_feat, d_uvd, d_cam, d_gathered, d_expert,
+                                             d_offsets, d_perm, d_points_out, d_feat_out, st);
+        if (rc2 == EMC2_OK && half0 < B) {
+            e = cudaStreamWaitEvent(st, h->ev_half, 0);
+            if (e != cudaSuccess) rc2 = check_cuda(h, e);
+            else
+                rc2 = launch_scan_gather_scatter(h, half0, B - half0, N, d_points, d_feat, d_uvd, d_cam, d_gathered,
+                                                 d_expert, d_offsets, d_perm, d_points_out, d_feat_out, st);
+        }
     }
     // Join even after an error, so that `cuda_stream` never runs ahead of stage 1.
     if (h->overlap) {
@@ -522,7 +541,7 @@ int emc2_bridge_set_overlap(emc2_bridge_t* h, int enable) {
 
 int emc2_bridge_set_tuning(emc2_bridge_t* h, int32_t knob, int32_t value) {
     if (!h || knob < 0 || knob >= EMC2_TUNE_KNOBS) return EMC2_ERR_INVALID_ARG;
-    static const int kMaxValue[EMC2_TUNE_KNOBS] = {3, 1, 2, 2};
+    static const int kMaxValue[EMC2_TUNE_KNOBS] = {3, 1, 2, 2, 1};
     if (value < 0 || value > kMaxValue[knob]) return EMC2_ERR_INVALID_ARG;
     if (knob == EMC2_TUNE_DEDUP_FINE || knob == EMC2_TUNE_DEDUP_PILLARS) {
         const int s = knob == EMC2_TUNE_DEDUP_FINE ? 0 : 1;
@@ -564,6 +583,7 @@ int emc2_bridge_destroy(emc2_bridge_t* h) {
     for (cudaEvent_t e : h->event_pool) cudaEventDestroy(e);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->ev_half) cudaEventDestroy(h->ev_half);
     if (h->side) cudaStreamDestroy(h->side);
     if (h->slab && cudaFree(h->slab) != cudaSuccess) rc = EMC2_ERR_CUDA;
     if (h->arm.slab && cudaFree(h->arm.slab) != cudaSuccess) rc = EMC2_ERR_CUDA;

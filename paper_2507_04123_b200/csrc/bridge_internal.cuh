@@ -163,12 +163,12 @@ struct emc2_bridge {
     int* d_rb_counts = nullptr;    // [27][voxel tiles] pairs per (offset, tile), and their prefix sums
     int* d_rb_base = nullptr;
     int max_tiles = 0;
-    int tune[EMC2_TUNE_KNOBS] = {0, 1, 0, 0};   // emc2_bridge_set_tuning
+    int tune[EMC2_TUNE_KNOBS] = {0, 1, 0, 0, 0};   // emc2_bridge_set_tuning
     emc2::DedupArm arm;
     int num_sms = 0;               // multiprocessors of the handle's device
     bool overlap = true;           // emc2_bridge_run puts stage 1 on `side`
     cudaStream_t side = nullptr;   // stream of stage 1 inside emc2_bridge_run
-    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_half = nullptr;
     int last_cuda_error = 0;
     bool profiling = false;
     int64_t launches[emc2::K_KINDS] = {0};
@@ -231,15 +231,15 @@ int launch_channels_last(emc2_bridge* h, int B, const float* d_planar, float* d_
 int launch_pool_features(emc2_bridge* h, int B, int p, const float* d_feat, float* d_pooled, cudaStream_t st);
 int launch_scene_route(emc2_bridge* h, int B, const int32_t* d_offsets, const uint8_t* priority, int min_points,
                        int32_t* d_scene_expert, cudaStream_t st);
-// Tile histograms (handle scratch) -> d_offsets and tile bases (handle scratch).
-void launch_route_scan(emc2_bridge* h, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st);
+// Tile histograms (handle scratch) of frames [b0, b0 + B) -> d_offsets (of frame b0 on) and tile bases.
+void launch_route_scan(emc2_bridge* h, int b0, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st);
 // Stages 2 - 4 in one pass over the feature rows (the one-call path), in two parts: projection +
 // routing per point (which, with `d_bev_to_zero`/`mark`, also marks the voxel cells of both scales
 // and zeroes the BEV image, so that stage 1 reads the points once less), then offsets + rows.
-int launch_project_route(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj, float* d_uvd,
-                         uint8_t* d_vis_mask, int8_t* d_cam, uint8_t* d_expert, bool mark, float* d_bev_to_zero,
-                         cudaStream_t st);
-int launch_scan_gather_scatter(emc2_bridge* h, int B, int N, const float* d_points, const float* d_feat,
+int launch_project_route(emc2_bridge* h, int b0, int B, int N, const float* d_points, const float* d_proj,
+                         float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam, uint8_t* d_expert, bool mark,
+                         float* d_bev_to_zero, int bev_frames, cudaStream_t st);
+int launch_scan_gather_scatter(emc2_bridge* h, int b0, int B, int N, const float* d_points, const float* d_feat,
                                const float* d_uvd, const int8_t* d_cam, float* d_gathered, const uint8_t* d_expert,
                                int32_t* d_offsets, int32_t* d_perm, float* d_points_out, float* d_feat_out,
                                cudaStream_t st);

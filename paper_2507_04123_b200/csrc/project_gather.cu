@@ -160,6 +160,7 @@ struct PrArgs {
     int N, tiles, K, H, W;
     float min_depth;
     RouteParams rp;
+    int frame0;           // kMark: frame index (in the whole batch) of this launch's first frame
     ScaleDev s0, s1;      // kMark: the voxel grids whose cells the points mark
     float4* bev;          // kMark: BEV image to zero (bev_n4 float4), or null
     size_t bev_n4;
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(kThreads) project_route_kernel(const __grid_co
         } else {
             x = __ldg(p); y = __ldg(p + 1); z = __ldg(p + 2);
         }
-        if (kMark) mark_point(a.s0, a.s1, x, y, z, b);
+        if (kMark) mark_point(a.s0, a.s1, x, y, z, a.frame0 + b);
         const Projected pr = project_point(sP, a.K, x, y, z, a.W, a.H, a.min_depth);
         suvd[t * 3] = pr.u; suvd[t * 3 + 1] = pr.v; suvd[t * 3 + 2] = pr.d;
         a.vis[g0 + t] = (uint8_t)pr.mask;
@@ -649,23 +650,28 @@ int launch_project_gather(emc2_bridge* h, int B, int N, const float* d_points, c
     return check_cuda(h, cudaGetLastError());
 }
 
-int launch_project_route(emc2_bridge* h, int B, int N, const float* d_points, const float* d_proj, float* d_uvd,
-                         uint8_t* d_vis_mask, int8_t* d_cam, uint8_t* d_expert, bool mark, float* d_bev_to_zero,
-                         cudaStream_t st) {
+// Frames [b0, b0 + B) of a batch whose buffers are given whole; `bev_frames` > 0: this launch also
+// zeroes the BEV image of that many frames.
+int launch_project_route(emc2_bridge* h, int b0, int B, int N, const float* d_points, const float* d_proj,
+                         float* d_uvd, uint8_t* d_vis_mask, int8_t* d_cam, uint8_t* d_expert, bool mark,
+                         float* d_bev_to_zero, int bev_frames, cudaStream_t st) {
     const emc2_config_t& c = h->cfg;
     const int tiles = (N + kTile - 1) / kTile;
     if (B == 0 || tiles == 0) return EMC2_OK;
     const dim3 grid(tiles, B);
+    const size_t p0 = (size_t)b0 * N;                      // first point of the range
     PrArgs pa;
-    pa.pts = d_points; pa.proj = d_proj; pa.uvd = d_uvd; pa.vis = d_vis_mask; pa.cam = d_cam;
-    pa.expert = d_expert; pa.tile_counts = h->d_tile_counts;
+    pa.pts = d_points + p0 * c.point_floats; pa.proj = d_proj + (size_t)b0 * c.num_cameras * 12;
+    pa.uvd = d_uvd + p0 * 3; pa.vis = d_vis_mask + p0; pa.cam = d_cam + p0;
+    pa.expert = d_expert + p0; pa.tile_counts = h->d_tile_counts + (size_t)b0 * tiles * c.num_experts;
     pa.N = N; pa.tiles = tiles; pa.K = c.num_cameras; pa.H = c.img_h; pa.W = c.img_w;
     pa.min_depth = c.min_depth;
     pa.rp = route_params(h);
+    pa.frame0 = b0;
     pa.s0 = h->scale[0]; pa.s1 = h->scale[1];
     pa.bev = nullptr; pa.bev_n4 = 0;
-    if (mark && d_bev_to_zero) {
-        const size_t bev_n = (size_t)B * c.point_floats * h->scale[1].dims[1] * h->scale[1].dims[0];
+    if (mark && d_bev_to_zero && bev_frames > 0) {
+        const size_t bev_n = (size_t)bev_frames * c.point_floats * h->scale[1].dims[1] * h->scale[1].dims[0];
         if (bev_n & 3) {
             cudaMemsetAsync(d_bev_to_zero, 0, bev_n * sizeof(float), st);
         } else {
@@ -686,7 +692,7 @@ int launch_project_route(emc2_bridge* h, int B, int N, const float* d_points, co
     return check_cuda(h, cudaGetLastError());
 }
 
-int launch_scan_gather_scatter(emc2_bridge* h, int B, int N, const float* d_points, const float* d_feat,
+int launch_scan_gather_scatter(emc2_bridge* h, int b0, int B, int N, const float* d_points, const float* d_feat,
                                const float* d_uvd, const int8_t* d_cam, float* d_gathered, const uint8_t* d_expert,
                                int32_t* d_offsets, int32_t* d_perm, float* d_points_out, float* d_feat_out,
                                cudaStream_t st) {
@@ -694,13 +700,18 @@ int launch_scan_gather_scatter(emc2_bridge* h, int B, int N, const float* d_poin
     if (B == 0) return EMC2_OK;
     const int tiles = (N + kTile - 1) / kTile;
     const dim3 grid(tiles > 0 ? tiles : 1, B);
-    launch_route_scan(h, B, tiles, N, d_offsets, st);
+    const int E = c.num_experts;
+    const size_t p0 = (size_t)b0 * N, t0 = (size_t)b0 * tiles * E;
+    launch_route_scan(h, b0, B, tiles, N, d_offsets + (size_t)b0 * (E + 1), st);
     if (tiles > 0) {
         GsArgs ga;
-        ga.pts = d_points; ga.uvd = d_uvd; ga.cam = d_cam; ga.expert = d_expert; ga.tile_base = h->d_tile_base;
-        ga.feat = reinterpret_cast<const float4*>(d_feat); ga.perm = d_perm; ga.pts_out = d_points_out;
-        ga.gathered = reinterpret_cast<float4*>(d_gathered); ga.feat_out = reinterpret_cast<float4*>(d_feat_out);
-        ga.N = N; ga.tiles = tiles; ga.E = c.num_experts; ga.K = c.num_cameras; ga.Hf = c.feat_h; ga.Wf = c.feat_w;
+        ga.pts = d_points + p0 * c.point_floats; ga.uvd = d_uvd + p0 * 3; ga.cam = d_cam + p0; ga.expert = d_expert + p0;
+        ga.tile_base = h->d_tile_base + t0;
+        ga.feat = reinterpret_cast<const float4*>(d_feat + (size_t)b0 * c.num_cameras * c.feat_h * c.feat_w * c.feat_c);
+        ga.perm = d_perm + p0; ga.pts_out = d_points_out + p0 * c.point_floats;
+        ga.gathered = d_gathered ? reinterpret_cast<float4*>(d_gathered + p0 * c.feat_c) : nullptr;
+        ga.feat_out = reinterpret_cast<float4*>(d_feat_out + p0 * c.feat_c);
+        ga.N = N; ga.tiles = tiles; ga.E = E; ga.K = c.num_cameras; ga.Hf = c.feat_h; ga.Wf = c.feat_w;
         ga.cf4 = c.feat_c / 4;
         ga.inv_stride = 1.0f / (float)c.feat_stride;
         ga.offset = c.feat_offset;

@@ -281,9 +281,11 @@ int launch_scene_route(emc2_bridge* h, int B, const int32_t* d_offsets, const ui
     return check_cuda(h, cudaGetLastError());
 }
 
-void launch_route_scan(emc2_bridge* h, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st) {
+void launch_route_scan(emc2_bridge* h, int b0, int B, int tiles, int N, int32_t* d_offsets, cudaStream_t st) {
     LaunchScope ls(h, K_ROUTE_SCAN, st);
-    route_scan_kernel<<<B, kScanThreads, 0, st>>>(h->d_tile_counts, h->d_tile_base, d_offsets, tiles, h->cfg.num_experts, N);
+    const size_t t0 = (size_t)b0 * tiles * h->cfg.num_experts;
+    route_scan_kernel<<<B, kScanThreads, 0, st>>>(h->d_tile_counts + t0, h->d_tile_base + t0, d_offsets, tiles,
+                                                  h->cfg.num_experts, N);
 }
 
 int launch_route_dispatch(emc2_bridge* h, int B, int N, const float* d_points, const uint8_t* d_vis_mask,

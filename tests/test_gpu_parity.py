@@ -48,7 +48,7 @@ def test_ragged_shapes(b200, oracle, B, N):
 
 
 TUNINGS = [(("row_store", 0),), (("row_store", 1),), (("row_store", 2),), (("row_store", 3),), (("mark_in_projection", 0),),
-           (("mark_in_projection", 1),), (("dedup_fine", 1),), (("dedup_fine", 2),), (("dedup_pillars", 1),),
+           (("mark_in_projection", 1),), (("split_batch", 0),), (("split_batch", 1),), (("dedup_fine", 1),), (("dedup_fine", 2),), (("dedup_pillars", 1),),
            (("dedup_pillars", 2),), (("dedup_fine", 2), ("dedup_pillars", 1)), (("dedup_fine", 1), ("dedup_pillars", 2))]
 
 
