@@ -94,3 +94,10 @@ def test_binding_refuses_to_run_without_cuda(pkg):
         pytest.skip("CUDA present")
     with pytest.raises(RuntimeError):
         pkg.Bridge(pkg.config_from_workload(gen.TINY))
+
+
+def test_tuning_and_timeline_reject_a_null_handle(pkg):
+    lib = pkg.load_library()
+    assert lib.emc2_bridge_set_tuning(None, 0, 0) == pkg.bridge.EMC2_ERR_INVALID_ARG
+    assert lib.emc2_bridge_profile_timeline(None, None, None, None, 0) == pkg.bridge.EMC2_ERR_INVALID_ARG
+    assert set(pkg.bridge.TUNE_NAMES.values()) == set(range(len(pkg.bridge.TUNE_NAMES)))

@@ -57,8 +57,9 @@ def test_every_implementation_choice_matches_the_oracle(b200, oracle, tune):
     """The alternatives behind emc2_bridge_set_tuning produce the same outputs: full tiles, ragged tiles,
     both feature widths, the dense frame (cap binds), and a frame with an expert that owns nothing."""
     for w in (gen.NUSCENES.with_shape(2, 20000), gen.KITTI.with_shape(3, 4099), gen.NUSCENES.with_shape(1, 31),
-              gen.DENSE.with_shape(1, 50000)):
+              gen.DENSE.with_shape(1, 50000), gen.KITTI.with_shape(1, 1)):
         run_case(b200, oracle, w, repeat=2, tune=tune)
+        run_case(b200, oracle, w, repeat=1, staged=True, tune=tune)
     w = gen.KITTI.with_shape(1, 3000)
     batch = gen.make_batch(w)
     batch["points"][..., 0] = np.abs(batch["points"][..., 0]) % 15.0     # everything nearer than 20 m
@@ -615,9 +616,12 @@ def test_single_expert_and_empty_expert(b200, oracle):
     assert (ref["offsets"][:, 2] == 0).all() and (ref["offsets"][:, 3] == w.N).all()
 
 
-def test_empty_inputs(b200):
+@pytest.mark.parametrize("design", [0, 1, 2], ids=["direct", "hash", "sort"])
+def test_empty_inputs(b200, design):
     w = gen.KITTI.with_shape(2, 64)
     br = b200.Bridge(b200.config_from_workload(w))
+    br.set_tuning("dedup_fine", design)
+    br.set_tuning("dedup_pillars", design)
     for B, N in ((0, 64), (2, 0)):
         pts = torch.zeros((B, N, 4), device="cuda")
         proj = torch.zeros((B, 1, 3, 4), device="cuda")
@@ -627,6 +631,7 @@ def test_empty_inputs(b200):
         assert np_(bufs["vox"]["num_voxels"]).tolist() == [0, 0]
         if B:
             assert (np_(bufs["rd"]["offsets"]) == 0).all()
+            assert not np_(bufs["vox"]["bev"]).any()       # an image without points is all zero
     br.close()
 
 
