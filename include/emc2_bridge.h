@@ -160,10 +160,12 @@ int emc2_route_dispatch(emc2_bridge_t* bridge, int32_t B, int32_t N, const float
  * of emc2_voxelize, emc2_project_gather and emc2_route_dispatch called in that order with the same
  * buffers.  Stages 2 - 4 run as one pass: the expert id is computed beside the projection, and
  * every feature row is blended once and stored both at its row of d_gathered and at its slot of
- * d_feat_out, so the rows are not read back.  Stage 1 does not depend on
- * stages 2 - 4, so the library runs it on a stream of its own (created with the handle, highest
- * priority) beside them: it starts once the work already queued on `cuda_stream` has finished,
- * and `cuda_stream` waits for it before the call's work counts as complete.  Seen from
+ * d_feat_out, so the rows are not read back.  The pass over the points that
+ * projects and routes them also marks their voxel cells, so stage 1 reads the points once less.
+ * The rest of stage 1 does not depend on stages 2 - 4, so the library runs it on a stream of its own
+ * (created with the handle, highest priority) beside them: it starts once that first pass, and with it
+ * the work already queued on `cuda_stream`, has finished, and `cuda_stream` waits for it before the
+ * call's work counts as complete.  Seen from
  * `cuda_stream` the call therefore behaves like the three calls, only shorter.  No allocation,
  * no host synchronisation.  d_gathered may be NULL for a caller who consumes only the dispatched
  * rows (d_feat_out with d_perm): the rows in point order are then not stored, which saves their
