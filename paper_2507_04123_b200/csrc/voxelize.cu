@@ -35,7 +35,7 @@ namespace {
 
 constexpr int kStatusCapacity = 1;
 constexpr int kStatusDirtyStore = 8;   // the cell store held more than one call's points can set
-constexpr int kPtsPerThread = 2;                      // independent points per thread (memory-level parallelism)
+constexpr int kPtsPerThread = 1;                      // points per thread of the two per-point passes (2 measured 1 - 3 % slower per step)
 constexpr int kBigTile = kThreads * kPtsPerThread;    // points per CTA in the two per-point passes
 
 // Where a point's cell sits in the unique list.
